@@ -1,0 +1,469 @@
+"""Pins of the CPU oracle against things other than itself: published test vectors, library
+routines (numpy.linalg, torch.optim), closed forms, invariants the paper states, brute force."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lordo_oracle as lo
+from oracle.lordo_oracle import (GLOBAL, LOCAL, OUTER_AVG, OUTER_NESTEROV, QHM_FULL, QHM_LOW, QHM_NONE, LordoOracle,
+                                 OracleConfig)
+
+RNG = np.random.default_rng(1234)
+
+
+def subspace_angle(A, B):
+    """Largest principal angle between the column spans of two orthonormal bases."""
+    s = np.linalg.svd(A.T @ B, compute_uv=False)
+    return float(np.arccos(np.clip(s.min(), -1.0, 1.0)))
+
+
+def make(mats, K=1, H=1, **kw):
+    kw.setdefault("state_dtype", "f64")
+    kw.setdefault("w_dtype", "f64")
+    kw.setdefault("e_dtype", "f64")
+    cfg = OracleConfig(mats=tuple(mats), K=K, H=H, **kw)
+    W0 = [RNG.standard_normal((m, n)) * 0.02 for m, n, _ in mats]
+    return cfg, W0
+
+
+# ------------------------------------------------------------------ integer generator (R14)
+
+def test_splitmix64_published_vectors():
+    # first three outputs of the public-domain splitmix64 generator seeded with 0
+    want = [0xE220A8397B1DCDAF, 0x6E789E6AA1B965F4, 0x06C45D188009454F]
+    got = lo.random_words(0, 3)
+    assert [int(x) for x in got] == want
+    assert [lo.mix64_int(lo._GOLDEN * (i + 1)) for i in range(3)] == want
+
+
+def test_vector_and_scalar_generators_agree_and_popcount():
+    key = lo.stream_key(7, lo.PURPOSE_OMEGA, 3, 2, 1)
+    w = lo.random_words(key, 1000)
+    for c in (0, 1, 17, 999):
+        assert int(w[c]) == lo.mix64_int(key + lo._GOLDEN * (c + 1))
+    pc = lo.popcount64(w)
+    assert [bin(int(x)).count("1") for x in w[:200]] == list(pc[:200])
+    # distinct streams differ
+    assert lo.stream_key(7, 2, 3, 2, 1) != lo.stream_key(7, 2, 3, 2, 0) != lo.stream_key(7, 2, 3, 1, 1)
+
+
+def test_random_matrix_moments():
+    M = lo.random_matrix(0, lo.PURPOSE_OMEGA, 0, 0, 0, 400, 256)
+    assert M.shape == (400, 256) and np.all(M == np.round(M)) and np.abs(M).max() <= 32
+    assert abs(M.mean()) < 0.05 and abs(M.var() - 16.0) < 0.3  # Binomial(64,1/2): variance 16
+    # row-major counter: element (i, j) is word i*cols + j
+    w = lo.random_words(lo.stream_key(0, lo.PURPOSE_OMEGA, 0, 0, 0), 400 * 256)
+    assert M[3, 5] == bin(int(w[3 * 256 + 5])).count("1") - 32
+
+
+def test_round_bf16_matches_torch():
+    x = np.concatenate([RNG.standard_normal(5000) * 10.0 ** RNG.integers(-6, 6, 5000),
+                        np.array([1.00390625, 1.01171875, -1.00390625, 0.0, 65280.0, 1e-40])])
+    want = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(lo.round_bf16(x), want)
+
+
+# ------------------------------------------------------------------ QR and the range finder (R1)
+
+@pytest.mark.parametrize("rows,r", [(8, 8), (50, 7), (300, 64)])
+def test_householder_matches_numpy_qr(rows, r):
+    Y = RNG.standard_normal((rows, r))
+    Q = lo.householder_qr_q(Y)
+    q, rr = np.linalg.qr(Y)
+    q = q * np.sign(np.diag(rr))[None, :]
+    assert np.abs(Q - q).max() < 1e-10
+    assert np.abs(Q.T @ Q - np.eye(r)).max() < 1e-12
+    R = Q.T @ Y
+    assert np.all(np.diag(R) > 0) and np.abs(np.tril(R, -1)).max() < 1e-10
+
+
+def test_householder_rank_deficient_is_finite_and_orthonormal():
+    Y = RNG.standard_normal((40, 3)) @ RNG.standard_normal((3, 8))
+    Y[:, 5] = 0.0
+    Q = lo.householder_qr_q(Y)
+    assert np.all(np.isfinite(Q)) and np.abs(Q.T @ Q - np.eye(8)).max() < 1e-10
+
+
+def test_initial_projection_orthonormal():
+    cfg, W0 = make([(96, 40, 16), (64, 64, 8)], K=2)
+    o = LordoOracle(cfg, W0)
+    for P in o.P:
+        assert np.abs(P.T @ P - np.eye(P.shape[1])).max() < 1e-5
+    cfgl, _ = make([(96, 40, 16)], K=2, variant=LOCAL)
+    ol = LordoOracle(cfgl, W0[:1])
+    assert ol.P[0].shape == (2, 96, 16) and np.array_equal(ol.P[0][1], np.eye(96, 16))
+
+
+@pytest.mark.parametrize("q", [0, 2])
+def test_exact_low_rank_gradient_is_reconstructed(q):
+    m, n, r = 64, 48, 8
+    cfg, W0 = make([(m, n, r)], K=1, variant=LOCAL, power_iters=q)
+    o = LordoOracle(cfg, W0)
+    G = [(RNG.standard_normal((m, r)) @ RNG.standard_normal((r, n)))[None]]
+    o.refresh_subspace(G)
+    P = o.P[0][0]
+    assert np.abs(P.T @ P - np.eye(r)).max() < 1e-5
+    assert np.linalg.norm(G[0][0] - P @ (P.T @ G[0][0])) / np.linalg.norm(G[0][0]) < 1e-5
+    o.inner_step(G, 1e-3, 0.9, 1.0, QHM_NONE)
+    assert np.abs(o.E[0]).max() < 1e-10 * np.abs(G[0]).max()
+
+
+@pytest.mark.parametrize("q", [0, 1, 2])
+def test_range_finder_angle_equals_closed_form(q):
+    """For S = U diag(s) V^T the span of (S S^T)^q S Omega is the span of U [I ; T] with
+    T = S2^(2q+1) Om2 Om1^-1 S1^-(2q+1), Om1 = V1^T Omega, Om2 = V2^T Omega, so the largest
+    principal angle to the top-r singular subspace (the paper's target, Q = U[:, :r]) has
+    tan(theta) = ||T||_2 exactly. It decays like (s_{r+1}/s_r)^(2q+1)."""
+    m, n, r = 80, 60, 6
+    U, _ = np.linalg.qr(RNG.standard_normal((m, m)))
+    V, _ = np.linalg.qr(RNG.standard_normal((n, n)))
+    sv = np.concatenate([np.linspace(10, 5, r), np.linspace(0.5, 0.05, n - r)])
+    S = (U[:, :n] * sv) @ V.T
+    Om = lo.random_matrix(0, lo.PURPOSE_OMEGA, 0, 0, 0, n, r)
+    P = lo.compute_projection(S, Om, q)
+    Om1, Om2 = V[:, :r].T @ Om, V[:, r:].T @ Om
+    e = 2 * q + 1
+    T = (sv[r:, None] ** e) * (Om2 @ np.linalg.inv(Om1)) / (sv[None, :r] ** e)
+    want = math.atan(np.linalg.norm(T, 2))
+    got = subspace_angle(P, U[:, :r])
+    assert abs(got - want) < 1e-6 * max(want, 1e-3) + 1e-9
+    Sx = (U[:, :r] * sv[:r]) @ V[:, :r].T  # exact rank r: the subspace is recovered exactly
+    assert subspace_angle(lo.compute_projection(Sx, Om, q), U[:, :r]) < 1e-6
+
+
+# ------------------------------------------------------------------ reductions to Adam
+
+def _adam_reference(W0, grads, lr, b1, b2, eps):
+    w = torch.tensor(W0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([w], lr=lr, betas=(b1, b2), eps=eps, weight_decay=0.0)
+    for g in grads:
+        w.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+    return w.detach().numpy()
+
+
+def test_identity_projection_reduces_to_adam():
+    m, n = 8, 12
+    cfg, W0 = make([(m, n, m)], K=1, H=1, variant=LOCAL, eps=1e-8, beta2=0.999)
+    o = LordoOracle(cfg, W0)  # Local: Q_0 = I
+    grads = [RNG.standard_normal((m, n)) for _ in range(6)]
+    for g in grads:
+        o.inner_step([g[None]], 3e-3, 0.9, 1.0, QHM_NONE)
+        o.outer_step()  # K = 1, averaging: must be the identity
+    want = _adam_reference(W0[0], grads, 3e-3, 0.9, 0.999, 1e-8)
+    assert np.abs(o.W[0][0] - want).max() < 1e-13
+    assert np.abs(o.E[0]).max() == 0.0
+
+
+def test_square_orthogonal_projection_is_adam_in_rotated_coordinates():
+    m, n = 10, 7
+    Qo, _ = np.linalg.qr(RNG.standard_normal((m, m)))
+    cfg, W0 = make([(m, n, m)], K=1, H=1)
+    o = LordoOracle(cfg, W0, P0=[Qo])
+    grads = [RNG.standard_normal((m, n)) for _ in range(5)]
+    for g in grads:
+        o.inner_step([g[None]], 1e-2, 0.8, 1.0, QHM_NONE)
+    want = Qo @ _adam_reference(Qo.T @ W0[0], [Qo.T @ g for g in grads], 1e-2, 0.8, 0.999, 1e-8)
+    assert np.abs(o.W[0][0] - want).max() < 1e-12
+
+
+# ------------------------------------------------------------------ brute force on 8x8
+
+def _brute_inner(W, E, P, u, v, G, s, lr, b1, b2, eps, omega, form, rho, ef):
+    """Direct loops over Algorithm 1's per-step lines for one worker; python floats only."""
+    m, n, r = len(W), len(W[0]), len(P[0])
+    nrm = math.sqrt(sum(G[i][j] ** 2 for i in range(m) for j in range(n)))
+    c = min(1.0, rho / (nrm + 1e-6)) if rho > 0 else 1.0
+    A = [[c * G[i][j] + (E[i][j] if ef else 0.0) for j in range(n)] for i in range(m)]
+    g = [[sum(P[i][a] * A[i][j] for i in range(m)) for j in range(n)] for a in range(r)]
+    En = [[A[i][j] - sum(P[i][a] * g[a][j] for a in range(r)) for j in range(n)] for i in range(m)] if ef else E
+    un = [[b1 * u[a][j] + (1 - b1) * g[a][j] for j in range(n)] for a in range(r)]
+    vn = [[b2 * v[a][j] + (1 - b2) * g[a][j] ** 2 for j in range(n)] for a in range(r)]
+    D = [[math.sqrt(vn[a][j] / (1 - b2 ** s)) + eps for j in range(n)] for a in range(r)]
+    uh = [[un[a][j] / (1 - b1 ** s) for j in range(n)] for a in range(r)]
+    Wn = [[0.0] * n for _ in range(m)]
+    for i in range(m):
+        for j in range(n):
+            if form == QHM_NONE:
+                upd = sum(P[i][a] * uh[a][j] / D[a][j] for a in range(r))
+            elif form == QHM_LOW:
+                upd = sum(P[i][a] * (omega * uh[a][j] + (1 - omega) * g[a][j]) / D[a][j] for a in range(r))
+            else:
+                mu = sum(D[a][j] for a in range(r)) / r
+                upd = (1 - omega) * c * G[i][j] / mu + omega * sum(P[i][a] * uh[a][j] / D[a][j] for a in range(r))
+            Wn[i][j] = W[i][j] - lr * upd
+    return Wn, En, un, vn
+
+
+@pytest.mark.parametrize("form", [QHM_NONE, QHM_LOW, QHM_FULL])
+@pytest.mark.parametrize("ef", [True, False])
+def test_brute_force_8x8_inner_and_outer(form, ef):
+    m = n = 8
+    r, K, H = 3, 2, 3
+    cfg, W0 = make([(m, n, r)], K=K, H=H, clip_rho=2.0, error_feedback=ef, outer=OUTER_NESTEROV, outer_lr=0.7,
+                   outer_momentum=0.9, beta2=0.95, eps=1e-6)
+    o = LordoOracle(cfg, W0)
+    P = o.P[0].tolist()
+    W = [W0[0].tolist() for _ in range(K)]
+    E = [[[0.0] * n for _ in range(m)] for _ in range(K)]
+    u = [[[0.0] * n for _ in range(r)] for _ in range(K)]
+    v = [[[0.0] * n for _ in range(r)] for _ in range(K)]
+    X0 = W0[0].tolist()
+    B = [[0.0] * n for _ in range(m)]
+    s = 0
+    for rnd in range(2):
+        for h in range(H):
+            G = RNG.standard_normal((K, m, n)) * (3.0 if h == 1 else 0.1)  # one step clips, others do not
+            o.inner_step([G], 0.01, 0.9, 0.7, form)
+            s += 1
+            for k in range(K):
+                W[k], E[k], u[k], v[k] = _brute_inner(W[k], E[k], P, u[k], v[k], G[k].tolist(), s, 0.01, 0.9, 0.95,
+                                                      1e-6, 0.7, form, 2.0, ef)
+            assert np.abs(o.W[0] - np.array(W)).max() < 1e-13
+            assert np.abs(o.E[0] - np.array(E)).max() < 1e-13
+            assert np.abs(o.v[0] - np.array(v)).max() < 1e-14
+        o.outer_step()
+        for a in range(r):
+            for j in range(n):
+                mu_, mv_ = sum(u[k][a][j] for k in range(K)) / K, sum(v[k][a][j] for k in range(K)) / K
+                for k in range(K):
+                    u[k][a][j], v[k][a][j] = mu_, mv_
+        for i in range(m):
+            for j in range(n):
+                d = X0[i][j] - sum(W[k][i][j] for k in range(K)) / K
+                B[i][j] = 0.9 * B[i][j] + d
+                X0[i][j] = X0[i][j] - 0.7 * (d + 0.9 * B[i][j])
+                for k in range(K):
+                    W[k][i][j] = X0[i][j]
+        assert np.abs(o.W[0] - np.array(W)).max() < 1e-13
+        assert np.abs(o.u[0] - np.array(u)).max() < 1e-14
+        assert np.abs(o.B[0] - np.array(B)).max() < 1e-13
+
+
+def test_brute_force_8x8_subspace_vs_svd():
+    m = n = 8
+    r = 2
+    U, _ = np.linalg.qr(RNG.standard_normal((m, m)))
+    V, _ = np.linalg.qr(RNG.standard_normal((n, n)))
+    S = (U * np.array([9, 7, 1e-3, 1e-3, 1e-3, 1e-3, 1e-3, 1e-3])) @ V.T
+    Usvd = np.linalg.svd(S)[0][:, :r]  # the paper's definition: Q = U[:, :r]
+    P = lo.compute_projection(S, lo.random_matrix(3, lo.PURPOSE_OMEGA, 0, 0, 0, n, r), 1)
+    assert subspace_angle(P, Usvd) < 1e-6
+
+
+def test_brute_force_rotation_8x8():
+    r, n, m = 3, 8, 8
+    P_old, _ = np.linalg.qr(RNG.standard_normal((m, r)))
+    P_new, _ = np.linalg.qr(RNG.standard_normal((m, r)))
+    u, v = RNG.standard_normal((r, n)), RNG.random((r, n))
+    b1, b2, s = 0.9, 0.99, 5
+    un, vn = lo.rotate_moments(u, v, P_new, P_old, b1, b2, s)
+    for a in range(r):
+        for j in range(n):
+            acc_u = acc_v = acc_ru = 0.0
+            for b in range(r):
+                rot = sum(P_new[i, a] * P_old[i, b] for i in range(m))
+                uh, vh = u[b, j] / (1 - b1 ** s), v[b, j] / (1 - b2 ** s)
+                acc_u += rot * u[b, j]
+                acc_ru += rot * uh
+                acc_v += rot * rot * (vh - uh * uh)
+            assert abs(un[a, j] - acc_u) < 1e-13
+            assert abs(vn[a, j] - (1 - b2 ** s) * abs(acc_v + acc_ru ** 2)) < 1e-13
+
+
+# ------------------------------------------------------------------ moment rotation (R4, R5)
+
+def test_rotation_identity_and_signed_permutation():
+    m, n, r = 20, 9, 5
+    P, _ = np.linalg.qr(RNG.standard_normal((m, r)))
+    u, v = RNG.standard_normal((r, n)), RNG.random((r, n)) + 1.0  # v_hat >= u_hat^2 not required
+    un, vn = lo.rotate_moments(u, v, P, P, 0.9, 0.999, 7)
+    assert np.abs(un - u).max() < 1e-13 and np.abs(vn - np.abs(v)).max() < 1e-12
+    perm = RNG.permutation(r)
+    sign = RNG.choice([-1.0, 1.0], r)
+    P2 = P[:, perm] * sign[None, :]
+    un, vn = lo.rotate_moments(u, v, P2, P, 0.9, 0.999, 7)
+    assert np.abs(un - sign[:, None] * u[perm]).max() < 1e-13
+    assert np.abs(vn - v[perm]).max() < 1e-12
+
+
+# ------------------------------------------------------------------ error feedback
+
+def test_error_feedback_invariants():
+    m, n, r = 24, 16, 4
+    cfg, W0 = make([(m, n, r)], K=1, clip_rho=0.0)
+    o = LordoOracle(cfg, W0)
+    o2 = LordoOracle(OracleConfig(**{**cfg.__dict__, "error_feedback": False}), W0)
+    P = o.P[0]
+    for t in range(4):
+        G = [RNG.standard_normal((1, m, n))]
+        o.inner_step(G, 1e-3, 0.9, 1.0, QHM_NONE)
+        o2.inner_step(G, 1e-3, 0.9, 1.0, QHM_NONE)
+        assert np.abs(P.T @ o.E[0][0]).max() < 1e-12  # E is orthogonal to the basis
+    # hence with a fixed basis the projected signal, and the whole trajectory, equal the one without EF
+    assert np.abs(o.W[0] - o2.W[0]).max() < 1e-12
+    assert np.abs(o.E[0]).max() > 0.1
+
+
+# ------------------------------------------------------------------ stagnation of the global rule
+
+@pytest.mark.parametrize("form,stagnates", [(QHM_NONE, True), (QHM_LOW, True), (QHM_FULL, False)])
+def test_global_projection_stagnates_without_full_rank_qhm(form, stagnates):
+    m, n, r, K, H = 32, 24, 4, 3, 5
+    cfg, W0 = make([(m, n, r)], K=K, H=H)
+    o = LordoOracle(cfg, W0)
+    P_before = o.P[0].copy()
+    for h in range(H):
+        o.inner_step([RNG.standard_normal((K, m, n))], 1e-2, 0.9, 0.9, form)
+    o.outer_step()
+    D = o.Delta[0]
+    resid = np.linalg.norm(D - P_before @ (P_before.T @ D)) / np.linalg.norm(D)
+    if stagnates:
+        assert resid < 1e-10 and np.linalg.matrix_rank(D, tol=1e-9) <= r
+        o.refresh_subspace(None, 0.9)
+        Rot = o.P[0].T @ P_before
+        mssv = np.sum(np.linalg.svd(Rot, compute_uv=False) ** 2) / r
+        assert subspace_angle(o.P[0], P_before) < 1e-6 and abs(mssv - 1.0) < 1e-9
+    else:
+        assert resid > 1e-2
+
+
+def test_local_pseudo_gradient_rank_bound():
+    m, n, r, K, H = 40, 36, 3, 4, 3
+    cfg, W0 = make([(m, n, r)], K=K, H=H, variant=LOCAL)
+    o = LordoOracle(cfg, W0)
+    for h in range(H):
+        G = [RNG.standard_normal((K, m, n))]
+        if h == 0:
+            o.refresh_subspace(G, 0.9)
+        o.inner_step(G, 1e-2, 0.9, 0.9, QHM_LOW)
+    o.outer_step()
+    sv = np.linalg.svd(o.Delta[0], compute_uv=False)
+    assert np.sum(sv > 1e-9 * sv[0]) == K * r  # rank(Delta) <= M * r, and generically equal
+
+
+# ------------------------------------------------------------------ outer step (R9, R10)
+
+def test_outer_average_and_unit_nesterov():
+    m, n, r, K = 6, 5, 2, 3
+    for kw in (dict(outer=OUTER_AVG), dict(outer=OUTER_NESTEROV, outer_lr=1.0, outer_momentum=0.0)):
+        cfg, W0 = make([(m, n, r)], K=K, H=1, **kw)
+        o = LordoOracle(cfg, W0)
+        o.W[0] = RNG.standard_normal((K, m, n))
+        mean = o.W[0].mean(axis=0)
+        o.outer_step()
+        assert np.abs(o.X0[0] - mean).max() < 1e-14 and np.abs(o.W[0] - mean[None]).max() < 1e-14
+        assert np.abs(o.Delta[0] - (W0[0] - mean)).max() < 1e-14
+
+
+def test_outer_nesterov_matches_torch_sgd():
+    m, n, r, K = 5, 4, 2, 2
+    cfg, W0 = make([(m, n, r)], K=K, H=1, outer=OUTER_NESTEROV, outer_lr=0.6, outer_momentum=0.9)
+    o = LordoOracle(cfg, W0)
+    w = torch.tensor(W0[0], dtype=torch.float64, requires_grad=True)
+    sgd = torch.optim.SGD([w], lr=0.6, momentum=0.9, nesterov=True, dampening=0.0)
+    for t in range(5):
+        drift = RNG.standard_normal((K, m, n)) * 0.1
+        o.W[0] = o.W[0] + drift  # workers move away from the anchor
+        delta = -(drift.mean(axis=0))
+        w.grad = torch.tensor(delta)
+        sgd.step()
+        o.outer_step()
+        assert np.abs(o.Delta[0] - delta).max() < 1e-14
+        assert np.abs(o.X0[0] - w.detach().numpy()).max() < 1e-13
+    # constant pseudo-gradient: B_j = Delta (1 - mu^j) / (1 - mu)
+    cfg2, W02 = make([(m, n, r)], K=1, H=1, outer=OUTER_NESTEROV, outer_lr=0.5, outer_momentum=0.8)
+    o2 = LordoOracle(cfg2, W02)
+    d = RNG.standard_normal((m, n))
+    for j in range(1, 6):
+        o2.W[0] = (o2.X0[0] - d)[None]
+        o2.outer_step()
+        assert np.abs(o2.B[0] - d * (1 - 0.8 ** j) / (1 - 0.8)).max() < 1e-13
+
+
+def test_single_worker_means_are_identities_and_state_sync():
+    m, n, r = 6, 7, 2
+    cfg, W0 = make([(m, n, r)], K=1, H=2)
+    o = LordoOracle(cfg, W0)
+    for _ in range(2):
+        o.inner_step([RNG.standard_normal((1, m, n))], 1e-2, 0.9, 1.0, QHM_NONE)
+    u, v, W = o.u[0].copy(), o.v[0].copy(), o.W[0].copy()
+    o.outer_step()
+    assert np.array_equal(o.u[0], u) and np.array_equal(o.v[0], v) and np.abs(o.W[0] - W).max() < 1e-16
+    cfg3, W03 = make([(m, n, r)], K=3, H=1, sync_u=True, sync_v=False)
+    o3 = LordoOracle(cfg3, W03)
+    o3.inner_step([RNG.standard_normal((3, m, n))], 1e-2, 0.9, 1.0, QHM_NONE)
+    u3, v3 = o3.u[0].copy(), o3.v[0].copy()
+    o3.outer_step()
+    assert np.abs(o3.u[0] - u3.mean(axis=0)[None]).max() < 1e-16 and np.array_equal(o3.v[0], v3)
+
+
+# ------------------------------------------------------------------ sign invariance
+
+def test_column_sign_flips_leave_weights_unchanged_but_rotations_do_not():
+    m, n, r = 16, 12, 4
+    cfg, W0 = make([(m, n, r)], K=1)
+    P, _ = np.linalg.qr(RNG.standard_normal((m, r)))
+    sign = np.array([1.0, -1.0, -1.0, 1.0])
+    Rq, _ = np.linalg.qr(RNG.standard_normal((r, r)))
+    oa, ob, oc = (LordoOracle(cfg, W0, P0=[p]) for p in (P, P * sign[None], P @ Rq))
+    for t in range(3):
+        G = [RNG.standard_normal((1, m, n))]
+        for o in (oa, ob, oc):
+            o.inner_step(G, 1e-2, 0.9, 0.8, QHM_FULL)
+    assert np.abs(oa.W[0] - ob.W[0]).max() < 1e-14
+    assert np.abs(oa.u[0] - sign[None, :, None] * ob.u[0]).max() < 1e-14
+    assert np.abs(oa.W[0] - oc.W[0]).max() > 1e-4
+
+
+# ------------------------------------------------------------------ clipping (R8)
+
+def test_clip_matches_torch_clip_grad_norm():
+    shapes = [(6, 5), (4, 9)]
+    K = 3
+    G = [RNG.standard_normal((K, a, b)) * sc for (a, b), sc in zip(shapes, (2.0, 0.5))]
+    G[0][2] *= 0.01
+    G[1][2] *= 0.01  # worker 2 stays under the radius
+    rho = 1.5
+    coef = lo.clip_coefficients(G, rho, 0)
+    for k in range(K):
+        params = [torch.nn.Parameter(torch.zeros(a, b, dtype=torch.float64)) for a, b in shapes]
+        for p, g in zip(params, G):
+            p.grad = torch.tensor(g[k])
+        total = torch.nn.utils.clip_grad_norm_(params, rho)
+        for i, p in enumerate(params):
+            assert np.abs(p.grad.numpy() - coef[i, k] * G[i][k]).max() < 1e-12
+        clipped = math.sqrt(sum(np.sum((coef[i, k] * G[i][k]) ** 2) for i in range(2)))
+        assert clipped <= rho * (1 + 1e-6)
+        assert coef[0, k] == coef[1, k]
+    assert coef[0, 2] == 1.0 and coef[0, 0] < 1.0
+    per_mat = lo.clip_coefficients(G, rho, 1)
+    assert per_mat[0, 0] != per_mat[1, 0]
+    assert np.all(lo.clip_coefficients(G, 0.0) == 1.0)
+
+
+# ------------------------------------------------------------------ storage accounting
+
+def test_state_size_matches_memory_table():
+    # Table "Memory overhead": parameters pq + projection pr + states 2rq (+ error buffer pq)
+    m, n, r, K = 12, 10, 3, 2
+    cfg, W0 = make([(m, n, r)], K=K, variant=LOCAL)
+    o = LordoOracle(cfg, W0)
+    per_worker = o.W[0][0].size + o.P[0][0].size + o.u[0][0].size + o.v[0][0].size
+    assert per_worker == m * n + m * r + 2 * r * n
+    assert o.E[0][0].size == m * n
+
+
+# ------------------------------------------------------------------ storage rounding modes
+
+def test_bf16_storage_rounds_once_per_step():
+    m, n, r = 8, 8, 2
+    cfg = OracleConfig(mats=((m, n, r),), K=1, H=1, w_dtype="bf16", e_dtype="bf16", state_dtype="f32")
+    W0 = [RNG.standard_normal((m, n)) * 0.02]
+    o = LordoOracle(cfg, W0)
+    o.inner_step([RNG.standard_normal((1, m, n))], 1e-2, 0.9, 1.0, QHM_NONE)
+    for arr in (o.W[0], o.E[0]):
+        assert np.array_equal(arr, lo.round_bf16(arr))
+    assert np.array_equal(o.u[0], o.u[0].astype(np.float32).astype(np.float64))
