@@ -1,0 +1,793 @@
+// Host layer of the LoRDO hot path: context, workspace carving, launch plans, the C ABI.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "lordo_kernels.h"
+
+using namespace lordo;
+
+namespace {
+
+constexpr int kMaxK = 64;
+
+enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3 };
+enum Phase { PH_SUBSPACE = 0, PH_ROTATE = 1, PH_COMMIT = 2 };
+
+struct PlanStep {
+  int type = ST_GEMM, phase = PH_SUBSPACE;
+  // gemm
+  int atrans = 0, dual = 0, a_square = 0, nprobs = 0;
+  long long prob_first = 0, tiles = 0;
+  // chol
+  const float* gram = nullptr;
+  float* lwork = nullptr;
+  float* rinv = nullptr;
+  int r = 0, batch = 0;
+  long long stride = 0;
+  // random fill
+  float* out = nullptr;
+  long long count = 0;
+  int purpose = 0, mat = 0, per_replica = 0;
+  // copy
+  void* dst = nullptr;
+  const void* src = nullptr;
+  size_t bytes = 0;
+};
+
+// Bump allocator over the workspace; with base == nullptr it only measures.
+struct Carver {
+  char* base;
+  size_t off = 0;
+  explicit Carver(void* b) : base(reinterpret_cast<char*>(b)) {}
+  template <class T>
+  T* take(size_t count) {
+    off = (off + 255) & ~size_t(255);
+    T* p = reinterpret_cast<T*>(base + off);  // base may be null: only offsets matter then
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+}  // namespace
+
+struct lordo_ctx {
+  lordo_config cfg;
+  std::vector<lordo_mat> mats;
+  std::vector<MatDev> h_mats;
+  int n_mats = 0, K = 0;
+
+  // device workspace pieces
+  MatDev* d_mats = nullptr;
+  long long *d_chunk_start = nullptr, *d_mom_start = nullptr, *d_wblk_start = nullptr, *d_sblk_start = nullptr;
+  const void** d_Gtab = nullptr;
+  double *d_partial = nullptr, *d_sumsq = nullptr;
+  float* d_coef = nullptr;
+  unsigned* d_status = nullptr;
+  GemmProblem* d_probs = nullptr;
+  float* d_scratch = nullptr;
+  long long total_chunks = 0, total_mom_tiles = 0, total_wblks = 0, total_sblks = 0;
+
+  // host plans
+  std::vector<GemmProblem> h_probs;
+  PlanStep inner_proj, inner_apply;
+  std::vector<PlanStep> refresh_steps, init_steps;
+
+  // pinned host staging
+  const void** h_Gtab = nullptr;  // pinned
+  unsigned* h_status = nullptr;   // pinned
+  std::vector<const void*> last_G;
+
+  // counters and call-order state
+  int64_t steps = 0, refreshes = 0, outers = 0, launches = 0;
+  int steps_in_round = 0;
+  bool after_outer = false;
+  std::string err;
+
+  // optional per-kernel-class timing (lordo_profile_enable)
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;
+  struct Span { int cls; cudaEvent_t a, b; };
+  std::vector<Span> spans;
+};
+
+namespace {
+
+int fail(lordo_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  return code;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate_config(const lordo_config* cfg, std::string& why) {
+  if (!cfg || !cfg->mats) { why = "null config or matrix list"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->n_mats < 1 || cfg->K < 1 || cfg->K > kMaxK || cfg->H < 1) { why = "n_mats, K (1..64) or H out of range"; return LORDO_ERR_INVALID_ARG; }
+  auto dt_ok = [](int d) { return d == LORDO_F32 || d == LORDO_BF16; };
+  if (!dt_ok(cfg->w_dtype) || !dt_ok(cfg->g_dtype) || !dt_ok(cfg->e_dtype)) { why = "unknown dtype"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->variant != LORDO_GLOBAL && cfg->variant != LORDO_LOCAL) { why = "unknown variant"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->outer != LORDO_OUTER_AVG && cfg->outer != LORDO_OUTER_NESTEROV) { why = "unknown outer optimizer"; return LORDO_ERR_INVALID_ARG; }
+  if (!(cfg->beta2 >= 0.f && cfg->beta2 < 1.f) || !(cfg->eps >= 0.f)) { why = "beta2 or eps out of range"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->power_iters < 0 || cfg->power_iters > 8) { why = "power_iters out of range (0..8)"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->clip_scope != 0 && cfg->clip_scope != 1) { why = "clip_scope must be 0 or 1"; return LORDO_ERR_INVALID_ARG; }
+  for (int i = 0; i < cfg->n_mats; ++i) {
+    const lordo_mat& a = cfg->mats[i];
+    if (a.m < 1 || a.n < 1 || a.r < 1) { why = "non-positive shape"; return LORDO_ERR_SHAPE; }
+    if (a.n % 8 != 0 || a.r % 8 != 0) { why = "n and r must be multiples of 8"; return LORDO_ERR_ALIGN; }
+    if (a.r > a.m || a.r > a.n) { why = "r must not exceed min(m, n)"; return LORDO_ERR_SHAPE; }
+    if (a.r > 4096) { why = "r above 4096 is not supported"; return LORDO_ERR_UNSUPPORTED; }
+  }
+  return LORDO_OK;
+}
+
+Operand plain(const void* p0, long long ld, int dt0 = LORDO_F32) {
+  Operand o;
+  std::memset(&o, 0, sizeof(o));
+  o.p0 = p0; o.ld = ld; o.dt0 = dt0; o.dt1 = LORDO_F32; o.kind = OP_PLAIN;
+  return o;
+}
+
+void prefix_arrays(const lordo_config& cfg, std::vector<long long>& chunk_start, std::vector<long long>& mom_start,
+                   std::vector<long long>& wblk, std::vector<long long>& sblk) {
+  const int n_mats = cfg.n_mats, K = cfg.K;
+  chunk_start.assign(n_mats + 1, 0); mom_start.assign(n_mats + 1, 0); wblk.assign(n_mats + 1, 0); sblk.assign(n_mats + 1, 0);
+  for (int i = 0; i < n_mats; ++i) {
+    const lordo_mat& a = cfg.mats[i];
+    const long long elems = a.m * a.n;
+    chunk_start[i + 1] = chunk_start[i] + (long long)K * ((elems + kSqChunk - 1) / kSqChunk);
+    mom_start[i + 1] = mom_start[i] + (long long)K * ((a.n + 127) / 128);
+    wblk[i + 1] = wblk[i] + (elems + 1023) / 1024;
+    sblk[i + 1] = sblk[i] + ((long long)a.r * a.n + 1023) / 1024;
+  }
+}
+
+// Builds everything that lives in the workspace. With ws == nullptr only the size is computed.
+size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
+  const lordo_config& cfg = c->cfg;
+  const int n_mats = cfg.n_mats, K = cfg.K;
+  const bool real = ws != nullptr && buf != nullptr;
+  const bool local = cfg.variant == LORDO_LOCAL;
+  const int q = cfg.power_iters;
+  Carver cv(ws);
+
+  c->d_mats = cv.take<MatDev>(n_mats);
+  c->d_chunk_start = cv.take<long long>(n_mats + 1);
+  c->d_mom_start = cv.take<long long>(n_mats + 1);
+  c->d_wblk_start = cv.take<long long>(n_mats + 1);
+  c->d_sblk_start = cv.take<long long>(n_mats + 1);
+  c->d_Gtab = cv.take<const void*>(n_mats);
+  c->d_status = cv.take<unsigned>(64);
+  c->d_sumsq = cv.take<double>((size_t)n_mats * K);
+  c->d_coef = cv.take<float>((size_t)n_mats * K);
+
+  std::vector<long long> chunk_start, mom_start, wblk, sblk;
+  prefix_arrays(cfg, chunk_start, mom_start, wblk, sblk);
+  size_t scratch_floats = 0;
+  for (int i = 0; i < n_mats; ++i) {
+    const lordo_mat& a = cfg.mats[i];
+    const long long maxd = a.m > a.n ? a.m : a.n;
+    const size_t nb = local ? K : 1;
+    const size_t per = (size_t)a.n * a.r + 2 * (size_t)a.m * a.r + (size_t)maxd * a.r + (q > 0 ? 2 * (size_t)a.n * a.r : 0) +
+                       4 * (size_t)a.r * a.r;
+    if (nb * per > scratch_floats) scratch_floats = nb * per;
+  }
+  c->total_chunks = chunk_start[n_mats];
+  c->total_mom_tiles = mom_start[n_mats];
+  c->total_wblks = wblk[n_mats];
+  c->total_sblks = sblk[n_mats];
+  c->d_partial = cv.take<double>((size_t)c->total_chunks);
+
+  c->h_mats.assign(n_mats, MatDev());
+  for (int i = 0; i < n_mats; ++i) {
+    const lordo_mat& a = cfg.mats[i];
+    MatDev& md = c->h_mats[i];
+    md.m = a.m; md.n = a.n; md.r = a.r; md.pad = 0;
+    md.ghat = cv.take<float>((size_t)K * a.r * a.n);
+    md.util = cv.take<float>((size_t)K * a.r * a.n);
+    md.dcol = cv.take<float>((size_t)K * a.n);
+    md.p_stride = local ? a.m * a.r : 0;
+    if (real) {
+      md.W = buf->W[i]; md.E = buf->E ? buf->E[i] : nullptr; md.P = buf->P[i]; md.u = buf->u[i]; md.v = buf->v[i];
+      md.X0 = buf->X0[i]; md.B = buf->B ? buf->B[i] : nullptr; md.Delta = buf->Delta[i];
+    }
+  }
+  c->d_scratch = cv.take<float>(scratch_floats);
+
+  // ---------------- launch plans ----------------
+  std::vector<GemmProblem>& P = c->h_probs;
+  P.clear();
+  auto begin_gemm = [&](int atrans, int dual, int a_square, int phase) {
+    PlanStep s;
+    s.type = ST_GEMM; s.atrans = atrans; s.dual = dual; s.a_square = a_square; s.phase = phase;
+    s.prob_first = (long long)P.size(); s.nprobs = 0; s.tiles = 0;
+    return s;
+  };
+  auto add_prob = [&](PlanStep& s, int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
+    GemmProblem g;
+    std::memset(&g, 0, sizeof(g));
+    g.M = M; g.N = N; g.Kd = Kd;
+    g.tiles_n = (N + 63) / 64;
+    g.tile_start = s.tiles;
+    g.A = A; g.B = B;
+    if (B2) g.B2 = *B2; else g.B2 = B;
+    g.epi = ep;
+    s.tiles += (long long)((M + 63) / 64) * g.tiles_n;
+    s.nprobs += 1;
+    P.push_back(g);
+  };
+  auto store_epi = [](float* C, long long ldc) {
+    Epilogue e;
+    std::memset(&e, 0, sizeof(e));
+    e.kind = EPI_STORE; e.C = C; e.ldc = ldc;
+    return e;
+  };
+
+  // inner step: g = P^T (c G + E)   and   E' = A - P g ; W' = W - lr (...)
+  c->inner_proj = begin_gemm(1, 0, 0, 0);
+  for (int i = 0; i < n_mats; ++i) {
+    const MatDev& md = c->h_mats[i];
+    for (int k = 0; k < K; ++k) {
+      Operand A = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
+      Operand B = plain(nullptr, md.n, cfg.g_dtype);
+      B.p0_ind = c->d_Gtab + i; B.p0_off = (long long)k * md.m * md.n;
+      B.s0_ptr = c->d_coef + (size_t)i * K + k;
+      if (cfg.error_feedback && real) {
+        B.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + (long long)k * md.m * md.n)
+                                        : (const void*)((const unsigned short*)md.E + (long long)k * md.m * md.n);
+        B.dt1 = cfg.e_dtype;
+      }
+      add_prob(c->inner_proj, md.r, (int)md.n, (int)md.m, A, B, nullptr, store_epi(md.ghat + (long long)k * md.r * md.n, md.n));
+    }
+  }
+  c->inner_apply = begin_gemm(0, 1, 0, 0);
+  for (int i = 0; i < n_mats; ++i) {
+    const MatDev& md = c->h_mats[i];
+    for (int k = 0; k < K; ++k) {
+      const long long wo = (long long)k * md.m * md.n;
+      Operand A = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
+      Operand B = plain(md.ghat + (long long)k * md.r * md.n, md.n);
+      Operand B2 = plain(md.util + (long long)k * md.r * md.n, md.n);
+      Epilogue e;
+      std::memset(&e, 0, sizeof(e));
+      e.kind = EPI_APPLY;
+      e.W = !real ? nullptr : cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
+      e.E = md.E ? (cfg.e_dtype == LORDO_F32 ? (void*)((float*)md.E + wo) : (void*)((unsigned short*)md.E + wo)) : nullptr;
+      e.G_ind = c->d_Gtab + i; e.G_off = wo;
+      e.dcol = md.dcol + (long long)k * md.n;
+      e.cptr = c->d_coef + (size_t)i * K + k;
+      add_prob(c->inner_apply, (int)md.m, (int)md.n, md.r, A, B, &B2, e);
+    }
+  }
+
+  // CholeskyQR2 of X (rows x r, batch of nb with stride sx) into O, through T.
+  auto cholqr2 = [&](std::vector<PlanStep>& plan, int phase, float* X, long long sx, float* T, long long st, float* O, long long so,
+                     long long rows, int r, int nb, float* gram, float* lw, float* rinv) {
+    float* src = X; long long ss = sx;
+    for (int pass = 0; pass < 2; ++pass) {
+      float* dst = pass == 0 ? T : O;
+      const long long sd = pass == 0 ? st : so;
+      PlanStep g = begin_gemm(1, 0, 0, phase);
+      for (int b = 0; b < nb; ++b) {
+        Operand A = plain(src + b * ss, r), B = plain(src + b * ss, r);
+        add_prob(g, r, r, (int)rows, A, B, nullptr, store_epi(gram + (long long)b * r * r, r));
+      }
+      plan.push_back(g);
+      PlanStep ch;
+      ch.type = ST_CHOL; ch.phase = phase; ch.gram = gram; ch.lwork = lw; ch.rinv = rinv; ch.r = r; ch.batch = nb; ch.stride = (long long)r * r;
+      plan.push_back(ch);
+      PlanStep ap = begin_gemm(0, 0, 0, phase);
+      for (int b = 0; b < nb; ++b) {
+        Operand A = plain(src + b * ss, r), B = plain(rinv + (long long)b * r * r, r);
+        add_prob(ap, (int)rows, r, r, A, B, nullptr, store_epi(dst + b * sd, r));
+      }
+      plan.push_back(ap);
+      src = dst; ss = sd;
+    }
+  };
+
+  c->refresh_steps.clear();
+  c->init_steps.clear();
+  for (int i = 0; i < n_mats; ++i) {
+    const MatDev& md = c->h_mats[i];
+    const long long m = md.m, n = md.n;
+    const int r = md.r;
+    const int nb = local ? K : 1;
+    const long long maxd = m > n ? m : n;
+    // scratch carve (batch-strided arrays)
+    float* s = c->d_scratch;
+    float* Om = s; s += (size_t)nb * n * r;
+    float* Ya = s; s += (size_t)nb * m * r;
+    float* Pn = s; s += (size_t)nb * m * r;
+    float* Yb = s; s += (size_t)nb * maxd * r;
+    float *Za = nullptr, *Zq = nullptr;
+    if (q > 0) { Za = s; s += (size_t)nb * n * r; Zq = s; s += (size_t)nb * n * r; }
+    float* gram = s; s += (size_t)nb * r * r;
+    float* lw = s; s += (size_t)nb * r * r;
+    float* rinv = s; s += (size_t)nb * r * r;
+    float* rot = s; s += (size_t)nb * r * r;
+
+    auto signal = [&](int b) {  // S of problem b: Delta (Global) or c_k G_k + E_k (Local), stored [m][n]
+      if (!local) return plain(md.Delta, n);
+      Operand A = plain(nullptr, n, cfg.g_dtype);
+      A.p0_ind = c->d_Gtab + i; A.p0_off = (long long)b * m * n;
+      A.s0_ptr = c->d_coef + (size_t)i * K + b;
+      if (cfg.error_feedback && real) {
+        A.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + (long long)b * m * n)
+                                        : (const void*)((const unsigned short*)md.E + (long long)b * m * n);
+        A.dt1 = cfg.e_dtype;
+      }
+      return A;
+    };
+    std::vector<PlanStep>& R = c->refresh_steps;
+    {
+      PlanStep f;
+      f.type = ST_RANDOM; f.phase = PH_SUBSPACE; f.out = Om; f.count = n * r; f.purpose = 2; f.mat = i; f.per_replica = local ? 1 : 0;
+      f.batch = nb;
+      R.push_back(f);
+    }
+    {  // Y = S Omega
+      PlanStep g = begin_gemm(0, 0, 0, PH_SUBSPACE);
+      for (int b = 0; b < nb; ++b) add_prob(g, (int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r));
+      R.push_back(g);
+    }
+    cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
+    for (int it = 0; it < q; ++it) {
+      {  // Z = S^T P'
+        PlanStep g = begin_gemm(1, 0, 0, PH_SUBSPACE);
+        for (int b = 0; b < nb; ++b) add_prob(g, (int)n, r, (int)m, signal(b), plain(Pn + (long long)b * m * r, r), nullptr, store_epi(Za + (long long)b * n * r, r));
+        R.push_back(g);
+      }
+      cholqr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n, r, nb, gram, lw, rinv);
+      {  // Y = S Z
+        PlanStep g = begin_gemm(0, 0, 0, PH_SUBSPACE);
+        for (int b = 0; b < nb; ++b) add_prob(g, (int)m, r, (int)n, signal(b), plain(Zq + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r));
+        R.push_back(g);
+      }
+      cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
+    }
+    {  // Rot = P'^T P
+      PlanStep g = begin_gemm(1, 0, 0, PH_ROTATE);
+      for (int b = 0; b < nb; ++b) add_prob(g, r, r, (int)m, plain(Pn + (long long)b * m * r, r), plain(md.P ? md.P + b * md.p_stride : nullptr, r), nullptr, store_epi(rot + (long long)b * r * r, r));
+      R.push_back(g);
+    }
+    {  // u', v' (into the transient g^ / U~ areas), then back
+      PlanStep g = begin_gemm(0, 1, 1, PH_ROTATE);
+      for (int k = 0; k < K; ++k) {
+        const long long so = (long long)k * r * n;
+        Operand A = plain(rot + (long long)(local ? k : 0) * r * r, r);
+        Operand B = plain(md.u ? md.u + so : nullptr, n); B.kind = OP_UHAT;
+        Operand B2 = plain(md.u ? md.u + so : nullptr, n); B2.kind = OP_VRES; B2.p1 = md.v ? md.v + so : nullptr;
+        Epilogue e;
+        std::memset(&e, 0, sizeof(e));
+        e.kind = EPI_ROTATE; e.u_out = md.ghat + so; e.v_out = md.util + so;
+        add_prob(g, r, (int)n, r, A, B, &B2, e);
+      }
+      R.push_back(g);
+      PlanStep cu, cv2;
+      cu.type = ST_COPY; cu.phase = PH_ROTATE; cu.dst = md.u; cu.src = md.ghat; cu.bytes = (size_t)K * r * n * sizeof(float);
+      cv2.type = ST_COPY; cv2.phase = PH_ROTATE; cv2.dst = md.v; cv2.src = md.util; cv2.bytes = (size_t)K * r * n * sizeof(float);
+      R.push_back(cu);
+      R.push_back(cv2);
+    }
+    {
+      PlanStep cp;
+      cp.type = ST_COPY; cp.phase = PH_COMMIT; cp.dst = md.P; cp.src = Pn; cp.bytes = (size_t)nb * m * r * sizeof(float);
+      R.push_back(cp);
+    }
+    if (!local) {  // P_0 = orthonormalised random m x r matrix
+      std::vector<PlanStep>& I = c->init_steps;
+      PlanStep f;
+      f.type = ST_RANDOM; f.out = Ya; f.count = m * r; f.purpose = 1; f.mat = i; f.per_replica = 0; f.batch = 1;
+      I.push_back(f);
+      cholqr2(I, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, md.P, m * r, m, r, 1, gram, lw, rinv);
+    }
+  }
+  c->d_probs = cv.take<GemmProblem>(P.size());
+
+  c->last_G.assign(n_mats, nullptr);
+  return (cv.off + 255) & ~size_t(255);
+}
+
+#define CUDA_OK(c, call)                                                                          \
+  do {                                                                                            \
+    cudaError_t e_ = (call);                                                                      \
+    if (e_ != cudaSuccess) return fail(c, LORDO_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
+  } while (0)
+
+int check_launch(lordo_ctx* c, const char* what) {
+  cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) return fail(c, LORDO_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+  return LORDO_OK;
+}
+
+// Kernel classes reported by lordo_profile_read.
+enum ProfClass { PC_CLIP = 0, PC_PROJECT = 1, PC_MOMENTS = 2, PC_APPLY = 3, PC_OUTER_STATES = 4, PC_OUTER_WEIGHTS = 5, PC_REFRESH = 6 };
+
+cudaEvent_t take_event(lordo_ctx* c) {
+  if (!c->ev_pool.empty()) { cudaEvent_t e = c->ev_pool.back(); c->ev_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct ProfScope {
+  lordo_ctx* c; cudaStream_t st; int cls; cudaEvent_t a = nullptr;
+  ProfScope(lordo_ctx* c_, cudaStream_t st_, int cls_) : c(c_), st(st_), cls(cls_) {
+    if (c->profiling) { a = take_event(c); cudaEventRecord(a, st); }
+  }
+  ~ProfScope() {
+    if (a) { cudaEvent_t b = take_event(c); cudaEventRecord(b, st); c->spans.push_back({cls, a, b}); }
+  }
+};
+
+GemmScalars base_scalars(const lordo_ctx* c) {
+  GemmScalars s;
+  std::memset(&s, 0, sizeof(s));
+  s.w_dt = c->cfg.w_dtype; s.e_dt = c->cfg.e_dtype; s.g_dt = c->cfg.g_dtype;
+  s.ef = c->cfg.error_feedback;
+  s.inv_bc1 = s.inv_bc2 = s.bc1 = s.bc2 = 1.f;
+  return s;
+}
+
+int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t st) {
+  switch (s.type) {
+    case ST_GEMM:
+      sc.a_square = s.a_square;
+      launch_gemm(c->d_probs + s.prob_first, s.nprobs, s.tiles, s.atrans, s.dual, sc, st);
+      c->launches += 1;
+      return check_launch(c, "gemm");
+    case ST_CHOL:
+      launch_chol_inverse(s.gram, s.lwork, s.rinv, s.r, s.batch, s.stride, c->d_status, st);
+      c->launches += 1;
+      return check_launch(c, "chol_inverse");
+    case ST_RANDOM: {
+      RandomKeys keys;
+      const long long index = s.purpose == 1 ? 0 : c->refreshes;
+      for (int b = 0; b < s.batch; ++b) keys.key[b] = stream_key(c->cfg.seed, s.purpose, s.mat, index, s.per_replica ? b : 0);
+      launch_fill_random(s.out, s.count, s.count, keys, s.batch, st);
+      c->launches += 1;
+      return check_launch(c, "fill_random");
+    }
+    case ST_COPY:
+      CUDA_OK(c, cudaMemcpyAsync(s.dst, s.src, s.bytes, cudaMemcpyDeviceToDevice, st));
+      return LORDO_OK;
+  }
+  return LORDO_OK;
+}
+
+// Makes the device copy of the gradient pointer table current.
+int set_gradients(lordo_ctx* c, const void* const* G, cudaStream_t st) {
+  bool same = true;
+  for (int i = 0; i < c->n_mats; ++i) {
+    if (!G[i]) return fail(c, LORDO_ERR_INVALID_ARG, "null gradient pointer");
+    if (!aligned16(G[i])) return fail(c, LORDO_ERR_ALIGN, "gradient pointer not 16-byte aligned");
+    if (G[i] != c->last_G[i]) same = false;
+  }
+  if (same) return LORDO_OK;
+  // the pinned table may still be read by an earlier copy on another stream: wait for this one
+  CUDA_OK(c, cudaStreamSynchronize(st));
+  for (int i = 0; i < c->n_mats; ++i) { c->h_Gtab[i] = G[i]; c->last_G[i] = G[i]; }
+  CUDA_OK(c, cudaMemcpyAsync(c->d_Gtab, c->h_Gtab, sizeof(void*) * c->n_mats, cudaMemcpyHostToDevice, st));
+  return LORDO_OK;
+}
+
+int run_clip(lordo_ctx* c, cudaStream_t st) {
+  if (!(c->cfg.clip_rho > 0.f)) return LORDO_OK;  // coefficients stay at 1
+  launch_sumsq_partial(c->d_mats, c->d_Gtab, c->d_chunk_start, c->n_mats, c->K, c->cfg.g_dtype, c->d_partial, c->total_chunks, st);
+  launch_clip_finalize(c->d_mats, c->d_chunk_start, c->n_mats, c->K, c->d_partial, c->cfg.clip_rho, c->cfg.clip_scope, c->d_coef,
+                       c->d_sumsq, c->d_status, st);
+  c->launches += 2;
+  return check_launch(c, "clip");
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+const char* lordo_status_string(int s) {
+  switch (s) {
+    case LORDO_OK: return "ok";
+    case LORDO_ERR_INVALID_ARG: return "invalid argument";
+    case LORDO_ERR_SHAPE: return "bad shape";
+    case LORDO_ERR_ALIGN: return "bad alignment";
+    case LORDO_ERR_STATE: return "call out of order";
+    case LORDO_ERR_NOMEM: return "workspace too small or host allocation failed";
+    case LORDO_ERR_CUDA: return "CUDA error";
+    case LORDO_ERR_NUMERIC: return "numerical flag set on the device";
+    case LORDO_ERR_UNSUPPORTED: return "unsupported configuration";
+  }
+  return "unknown status";
+}
+
+int lordo_query_workspace(const lordo_config* cfg, size_t* bytes) {
+  std::string why;
+  int rc = validate_config(cfg, why);
+  if (rc != LORDO_OK) return rc;
+  if (!bytes) return LORDO_ERR_INVALID_ARG;
+  lordo_ctx tmp;
+  tmp.cfg = *cfg;
+  tmp.n_mats = cfg->n_mats; tmp.K = cfg->K;
+  *bytes = build(&tmp, nullptr, nullptr);
+  return LORDO_OK;
+}
+
+int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspace, size_t workspace_bytes, void* stream,
+               lordo_ctx** out) {
+  std::string why;
+  int rc = validate_config(cfg, why);
+  if (rc != LORDO_OK) return rc;
+  if (!buf || !workspace || !out) return LORDO_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LORDO_ERR_ALIGN;
+  if (!buf->W || !buf->P || !buf->u || !buf->v || !buf->X0 || !buf->Delta) return LORDO_ERR_INVALID_ARG;
+  if (cfg->error_feedback && !buf->E) return LORDO_ERR_INVALID_ARG;
+  if (cfg->outer == LORDO_OUTER_NESTEROV && !buf->B) return LORDO_ERR_INVALID_ARG;
+  for (int i = 0; i < cfg->n_mats; ++i) {
+    const void* ptrs[8] = {buf->W[i], cfg->error_feedback ? buf->E[i] : (void*)16, buf->P[i], buf->u[i], buf->v[i], buf->X0[i],
+                           cfg->outer == LORDO_OUTER_NESTEROV ? (void*)buf->B[i] : (void*)16, buf->Delta[i]};
+    for (const void* p : ptrs) {
+      if (!p) return LORDO_ERR_INVALID_ARG;
+      if (!aligned16(p)) return LORDO_ERR_ALIGN;
+    }
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  lordo_ctx* c = new (std::nothrow) lordo_ctx;
+  if (!c) return LORDO_ERR_NOMEM;
+  c->cfg = *cfg;
+  c->mats.assign(cfg->mats, cfg->mats + cfg->n_mats);
+  c->cfg.mats = c->mats.data();
+  c->n_mats = cfg->n_mats; c->K = cfg->K;
+  const size_t need = build(c, buf, workspace);
+  if (need > workspace_bytes) { delete c; return LORDO_ERR_NOMEM; }
+
+  auto bail = [&](int code) { lordo_destroy(c); return code; };
+  if (cudaHostAlloc((void**)&c->h_Gtab, sizeof(void*) * c->n_mats, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
+  if (cudaHostAlloc((void**)&c->h_status, 256, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
+
+  std::vector<long long> cs, ms, wb, sb;
+  prefix_arrays(c->cfg, cs, ms, wb, sb);
+  const int nm = c->n_mats;
+#define INIT_CUDA(call) do { if ((call) != cudaSuccess) { cudaGetLastError(); return bail(LORDO_ERR_CUDA); } } while (0)
+  INIT_CUDA(cudaMemcpyAsync(c->d_mats, c->h_mats.data(), sizeof(MatDev) * nm, cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->d_chunk_start, cs.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->d_mom_start, ms.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->d_wblk_start, wb.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->d_sblk_start, sb.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemcpyAsync(c->d_probs, c->h_probs.data(), sizeof(GemmProblem) * c->h_probs.size(), cudaMemcpyHostToDevice, st));
+  INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
+  INIT_CUDA(cudaMemsetAsync(c->d_Gtab, 0, sizeof(void*) * nm, st));
+  INIT_CUDA(cudaStreamSynchronize(st));  // the host vectors above may now be reused
+
+  // Require block: replicas and anchor from W[0]; zero states; clip coefficients 1; P_0
+  launch_init_weights(c->d_mats, c->d_wblk_start, nm, c->total_wblks, c->K, c->cfg.w_dtype, st);
+  launch_fill_float(c->d_coef, (long long)nm * c->K, 1.f, st);
+  c->launches += 2;
+  for (int i = 0; i < nm; ++i) {
+    const MatDev& md = c->h_mats[i];
+    const size_t wn = (size_t)md.m * md.n, sn = (size_t)c->K * md.r * md.n;
+    if (md.E) INIT_CUDA(cudaMemsetAsync(md.E, 0, (size_t)c->K * wn * (c->cfg.e_dtype == LORDO_F32 ? 4 : 2), st));
+    INIT_CUDA(cudaMemsetAsync(md.u, 0, sn * 4, st));
+    INIT_CUDA(cudaMemsetAsync(md.v, 0, sn * 4, st));
+    if (md.B) INIT_CUDA(cudaMemsetAsync(md.B, 0, wn * 4, st));
+    INIT_CUDA(cudaMemsetAsync(md.Delta, 0, wn * 4, st));
+    if (c->cfg.variant == LORDO_LOCAL) {
+      launch_identity_projection(md.P, md.m, md.r, c->K, st);
+      c->launches += 1;
+    }
+  }
+  GemmScalars sc = base_scalars(c);
+  for (const PlanStep& s : c->init_steps) {
+    rc = run_plan_step(c, s, sc, st);
+    if (rc != LORDO_OK) return bail(rc);
+  }
+  INIT_CUDA(cudaStreamSynchronize(st));
+  if (cudaGetLastError() != cudaSuccess) return bail(LORDO_ERR_CUDA);
+#undef INIT_CUDA
+  *out = c;
+  return LORDO_OK;
+}
+
+int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, float omega, int form, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  if (!G) return fail(c, LORDO_ERR_INVALID_ARG, "G is null");
+  if (form != LORDO_QHM_NONE && form != LORDO_QHM_LOW && form != LORDO_QHM_FULL) return fail(c, LORDO_ERR_INVALID_ARG, "unknown QHM form");
+  if (!(beta1 >= 0.f && beta1 < 1.f) || !(omega >= 0.f && omega <= 1.f)) return fail(c, LORDO_ERR_INVALID_ARG, "beta1 or omega out of range");
+  if (c->steps_in_round >= c->cfg.H) return fail(c, LORDO_ERR_STATE, "H inner steps done: lordo_outer_step is due");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int rc = set_gradients(c, G, st);
+  if (rc != LORDO_OK) return rc;
+  {
+    ProfScope ps(c, st, PC_CLIP);
+    rc = run_clip(c, st);
+  }
+  if (rc != LORDO_OK) return rc;
+
+  const int64_t s = c->steps + 1;
+  const double bc1 = 1.0 - std::pow((double)beta1, (double)s), bc2 = 1.0 - std::pow((double)c->cfg.beta2, (double)s);
+  GemmScalars gs = base_scalars(c);
+  gs.lr = lr; gs.omega = omega; gs.form = form;
+  gs.inv_bc1 = (float)(1.0 / bc1); gs.inv_bc2 = (float)(1.0 / bc2); gs.bc1 = (float)bc1; gs.bc2 = (float)bc2;
+  StepScalars ss;
+  ss.lr = lr; ss.beta1 = beta1; ss.beta2 = c->cfg.beta2; ss.omega = omega; ss.eps = c->cfg.eps;
+  ss.inv_bc1 = gs.inv_bc1; ss.inv_bc2 = gs.inv_bc2; ss.form = form; ss.ef = c->cfg.error_feedback; ss.K = c->K;
+
+  {
+    ProfScope ps(c, st, PC_PROJECT);
+    rc = run_plan_step(c, c->inner_proj, gs, st);
+  }
+  if (rc != LORDO_OK) return rc;
+  {
+    ProfScope ps(c, st, PC_MOMENTS);
+    launch_moments(c->d_mats, c->d_mom_start, c->n_mats, c->total_mom_tiles, ss, st);
+  }
+  c->launches += 1;
+  rc = check_launch(c, "moments");
+  if (rc != LORDO_OK) return rc;
+  {
+    ProfScope ps(c, st, PC_APPLY);
+    rc = run_plan_step(c, c->inner_apply, gs, st);
+  }
+  if (rc != LORDO_OK) return rc;
+  c->steps = s;
+  c->steps_in_round += 1;
+  c->after_outer = false;
+  return LORDO_OK;
+}
+
+int lordo_inner_step_host(lordo_ctx* c, const void* const* G_host, void* const* G_stage, float lr, float beta1, float omega,
+                          int form, float* clip_out_host, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  if (!G_host || !G_stage) return fail(c, LORDO_ERR_INVALID_ARG, "null gradient table");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const size_t esz = c->cfg.g_dtype == LORDO_F32 ? 4 : 2;
+  for (int i = 0; i < c->n_mats; ++i) {
+    if (!G_host[i] || !G_stage[i]) return fail(c, LORDO_ERR_INVALID_ARG, "null gradient pointer");
+    const size_t bytes = (size_t)c->K * c->mats[i].m * c->mats[i].n * esz;
+    CUDA_OK(c, cudaMemcpyAsync(G_stage[i], G_host[i], bytes, cudaMemcpyHostToDevice, st));
+  }
+  int rc = lordo_inner_step(c, (const void* const*)G_stage, lr, beta1, omega, form, stream);
+  if (rc != LORDO_OK) return rc;
+  if (clip_out_host) CUDA_OK(c, cudaMemcpyAsync(clip_out_host, c->d_coef, sizeof(float) * c->K, cudaMemcpyDeviceToHost, st));
+  CUDA_OK(c, cudaStreamSynchronize(st));
+  return LORDO_OK;
+}
+
+int lordo_outer_step(lordo_ctx* c, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  if (c->steps_in_round != c->cfg.H) return fail(c, LORDO_ERR_STATE, "lordo_outer_step needs exactly H inner steps since the last one");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  const int which = (c->cfg.sync_u ? 1 : 0) | (c->cfg.sync_v ? 2 : 0);
+  if (which) {
+    ProfScope ps(c, st, PC_OUTER_STATES);
+    launch_outer_states(c->d_mats, c->d_sblk_start, c->n_mats, c->total_sblks, c->K, which, st);
+    c->launches += 1;
+  }
+  {
+    ProfScope ps(c, st, PC_OUTER_WEIGHTS);
+    launch_outer_weights(c->d_mats, c->d_wblk_start, c->n_mats, c->total_wblks, c->K, c->cfg.w_dtype, c->cfg.outer, c->cfg.outer_lr,
+                         c->cfg.outer_momentum, st);
+  }
+  c->launches += 1;
+  int rc = check_launch(c, "outer");
+  if (rc != LORDO_OK) return rc;
+  c->steps_in_round = 0;
+  c->outers += 1;
+  c->after_outer = true;
+  return LORDO_OK;
+}
+
+int lordo_refresh_subspace(lordo_ctx* c, const void* const* G, float beta1, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  const bool local = c->cfg.variant == LORDO_LOCAL;
+  if (!(beta1 >= 0.f && beta1 < 1.f)) return fail(c, LORDO_ERR_INVALID_ARG, "beta1 out of range");
+  if (local && !G) return fail(c, LORDO_ERR_INVALID_ARG, "Local refresh needs the gradients of the coming step");
+  if (!local && G) return fail(c, LORDO_ERR_INVALID_ARG, "Global refresh takes its signal from Delta: G must be NULL");
+  if (local && c->steps_in_round != 0) return fail(c, LORDO_ERR_STATE, "Local refresh only before the first inner step of a round");
+  if (!local && !c->after_outer) return fail(c, LORDO_ERR_STATE, "Global refresh only directly after lordo_outer_step");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int rc;
+  if (local) {
+    rc = set_gradients(c, G, st);
+    if (rc != LORDO_OK) return rc;
+    rc = run_clip(c, st);
+    if (rc != LORDO_OK) return rc;
+  }
+  GemmScalars gs = base_scalars(c);
+  const bool rotate = c->steps > 0;
+  if (rotate) {
+    const double bc1 = 1.0 - std::pow((double)beta1, (double)c->steps), bc2 = 1.0 - std::pow((double)c->cfg.beta2, (double)c->steps);
+    gs.inv_bc1 = (float)(1.0 / bc1); gs.inv_bc2 = (float)(1.0 / bc2); gs.bc1 = (float)bc1; gs.bc2 = (float)bc2;
+  }
+  {
+    ProfScope ps(c, st, PC_REFRESH);
+    for (const PlanStep& s : c->refresh_steps) {
+      if (s.phase == PH_ROTATE && !rotate) continue;
+      rc = run_plan_step(c, s, gs, st);
+      if (rc != LORDO_OK) return rc;
+    }
+  }
+  c->refreshes += 1;
+  c->after_outer = false;
+  return LORDO_OK;
+}
+
+int lordo_poll_status(lordo_ctx* c, void* stream, uint32_t* flags) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  CUDA_OK(c, cudaMemcpyAsync(c->h_status, c->d_status, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+  CUDA_OK(c, cudaStreamSynchronize(st));
+  CUDA_OK(c, cudaGetLastError());
+  if (flags) *flags = *c->h_status;
+  if (*c->h_status) return fail(c, LORDO_ERR_NUMERIC, "device flag word is non-zero");
+  return LORDO_OK;
+}
+
+int lordo_get_counters(const lordo_ctx* c, int64_t out[4]) {
+  if (!c || !out) return LORDO_ERR_INVALID_ARG;
+  out[0] = c->steps; out[1] = c->refreshes; out[2] = c->outers; out[3] = c->steps_in_round;
+  return LORDO_OK;
+}
+
+int lordo_set_counters(lordo_ctx* c, const int64_t in[4]) {
+  if (!c || !in) return LORDO_ERR_INVALID_ARG;
+  if (in[0] < 0 || in[1] < 0 || in[2] < 0 || in[3] < 0 || in[3] > c->cfg.H) return fail(c, LORDO_ERR_INVALID_ARG, "counter out of range");
+  c->steps = in[0]; c->refreshes = in[1]; c->outers = in[2]; c->steps_in_round = (int)in[3];
+  c->after_outer = false;
+  return LORDO_OK;
+}
+
+int lordo_clip_coefficients(const lordo_ctx* c, const float** device_ptr) {
+  if (!c || !device_ptr) return LORDO_ERR_INVALID_ARG;
+  *device_ptr = c->d_coef;
+  return LORDO_OK;
+}
+
+int64_t lordo_launch_count(const lordo_ctx* c) { return c ? c->launches : -1; }
+
+int lordo_profile_enable(lordo_ctx* c, int on) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  c->profiling = on != 0;
+  return LORDO_OK;
+}
+
+int lordo_profile_read(lordo_ctx* c, void* stream, float ms_out[8]) {
+  if (!c || !ms_out) return LORDO_ERR_INVALID_ARG;
+  CUDA_OK(c, cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(stream)));
+  for (int i = 0; i < 8; ++i) ms_out[i] = 0.f;
+  for (const lordo_ctx::Span& sp : c->spans) {
+    float ms = 0.f;
+    CUDA_OK(c, cudaEventElapsedTime(&ms, sp.a, sp.b));
+    ms_out[sp.cls] += ms;
+    c->ev_pool.push_back(sp.a);
+    c->ev_pool.push_back(sp.b);
+  }
+  c->spans.clear();
+  return LORDO_OK;
+}
+
+const char* lordo_last_error(const lordo_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+int lordo_destroy(lordo_ctx* c) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  if (c->h_Gtab) cudaFreeHost(c->h_Gtab);
+  if (c->h_status) cudaFreeHost(c->h_status);
+  for (const lordo_ctx::Span& sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  delete c;
+  return LORDO_OK;
+}
+
+int lordo_fill_random(uint64_t seed, int32_t purpose, int32_t mat, int64_t index, int32_t replica, int64_t rows, int64_t cols,
+                      float* out_dev, void* stream) {
+  if (!out_dev || rows < 1 || cols < 1) return LORDO_ERR_INVALID_ARG;
+  RandomKeys keys;
+  keys.key[0] = stream_key(seed, purpose, mat, index, replica);
+  launch_fill_random(out_dev, rows * cols, rows * cols, keys, 1, reinterpret_cast<cudaStream_t>(stream));
+  return cudaPeekAtLastError() == cudaSuccess ? LORDO_OK : LORDO_ERR_CUDA;
+}
+
+}  // extern "C"

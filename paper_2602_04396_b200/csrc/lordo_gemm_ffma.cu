@@ -1,0 +1,281 @@
+// Grouped fp32 FFMA GEMM with fused operand formation and epilogues: the fp32-accurate ("check
+// mode") realisation of every contraction of the path -- P^T(cG+E), P g, P U~, the sketch and
+// subspace-iteration products, Gram matrices, R^-1 application, Rot = P'^T P and the rotation of
+// the moments. 64 x 64 output tile, 16-deep k-slices, 256 threads, 4 x 4 outputs per thread.
+#include "lordo_kernels.h"
+
+namespace lordo {
+
+constexpr int BM = 64, BN = 64, BK = 16, PADS = 4;
+
+__device__ __forceinline__ const void* operand_base(const Operand& op) {
+  return op.p0_ind ? *op.p0_ind : op.p0;
+}
+
+// Four consecutive stored elements (row, col..col+3) of an operand, zero outside (rows, cols).
+__device__ __forceinline__ float4 operand_load4(const Operand& op, const void* base, float s0, const GemmScalars& sc, long long row,
+                                                long long col, long long rows, long long cols) {
+  float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (row >= rows || col >= cols) return o;
+  const long long idx = row * op.ld + col;
+  if (col + 3 < cols) {
+    const float4 a = load4(base, op.dt0, op.p0_off + idx);
+    if (op.kind == OP_PLAIN) {
+      o = make_float4(s0 * a.x, s0 * a.y, s0 * a.z, s0 * a.w);
+      if (op.p1) {
+        const float4 b = load4(op.p1, op.dt1, idx);
+        o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+      }
+    } else if (op.kind == OP_UHAT) {
+      o = make_float4(sc.inv_bc1 * a.x, sc.inv_bc1 * a.y, sc.inv_bc1 * a.z, sc.inv_bc1 * a.w);
+    } else {
+      const float4 b = load4(op.p1, op.dt1, idx);
+      const float ux = sc.inv_bc1 * a.x, uy = sc.inv_bc1 * a.y, uz = sc.inv_bc1 * a.z, uw = sc.inv_bc1 * a.w;
+      o = make_float4(sc.inv_bc2 * b.x - ux * ux, sc.inv_bc2 * b.y - uy * uy, sc.inv_bc2 * b.z - uz * uz,
+                      sc.inv_bc2 * b.w - uw * uw);
+    }
+    return o;
+  }
+  float t[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int e = 0; e < 4 && col + e < cols; ++e) {
+    const float a = load1(base, op.dt0, op.p0_off + idx + e);
+    if (op.kind == OP_PLAIN) {
+      t[e] = s0 * a + (op.p1 ? load1(op.p1, op.dt1, idx + e) : 0.f);
+    } else if (op.kind == OP_UHAT) {
+      t[e] = sc.inv_bc1 * a;
+    } else {
+      const float uh = sc.inv_bc1 * a;
+      t[e] = sc.inv_bc2 * load1(op.p1, op.dt1, idx + e) - uh * uh;
+    }
+  }
+  return make_float4(t[0], t[1], t[2], t[3]);
+}
+
+template <int ATRANS, int DUAL>
+__global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __restrict__ probs, int nprobs, GemmScalars sc) {
+  __shared__ __align__(16) float sA[BK][BM + PADS];
+  __shared__ __align__(16) float sB[BK][BN + PADS];
+  __shared__ __align__(16) float sB2[DUAL ? BK : 1][BN + PADS];
+
+  // locate the problem of this block
+  const long long blk = blockIdx.x;
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].tile_start <= blk) lo = mid; else hi = mid - 1;
+  }
+  const GemmProblem& pr = probs[lo];
+  const long long local = blk - pr.tile_start;
+  const int tile_m = (int)(local / pr.tiles_n), tile_n = (int)(local - (long long)tile_m * pr.tiles_n);
+  const int M = pr.M, N = pr.N, Kd = pr.Kd;
+  const long long m0 = (long long)tile_m * BM, n0 = (long long)tile_n * BN;
+
+  const void* baseA = operand_base(pr.A);
+  const void* baseB = operand_base(pr.B);
+  const void* baseB2 = DUAL ? operand_base(pr.B2) : nullptr;
+  const float sA0 = pr.A.s0_ptr ? *pr.A.s0_ptr : 1.f;
+  const float sB0 = pr.B.s0_ptr ? *pr.B.s0_ptr : 1.f;
+  float sB20 = 1.f;
+  if constexpr (DUAL) sB20 = pr.B2.s0_ptr ? *pr.B2.s0_ptr : 1.f;
+
+  const int t = threadIdx.x;
+  const int tx = t & 15, ty = t >> 4;
+  // B tile loader: one float4 per thread, row kk = t/16, columns (t%16)*4
+  const int bk = t >> 4, bc = (t & 15) * 4;
+  // A tile loader. ATRANS: as B (stored [Kd][M]). Otherwise stored [M][Kd]: row t/4, k (t%4)*4.
+  const int ar = ATRANS ? (t >> 4) : (t >> 2), ac = ATRANS ? (t & 15) * 4 : (t & 3) * 4;
+
+  float acc[4][4], acc2[DUAL ? 4 : 1][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      acc[i][j] = 0.f;
+      if constexpr (DUAL) acc2[i][j] = 0.f;
+    }
+
+  float4 ra, rb, rb2 = make_float4(0.f, 0.f, 0.f, 0.f);
+  auto fetch = [&](int k0) {
+    if (ATRANS) ra = operand_load4(pr.A, baseA, sA0, sc, k0 + ar, m0 + ac, Kd, M);
+    else ra = operand_load4(pr.A, baseA, sA0, sc, m0 + ar, k0 + ac, M, Kd);
+    rb = operand_load4(pr.B, baseB, sB0, sc, k0 + bk, n0 + bc, Kd, N);
+    if constexpr (DUAL) rb2 = operand_load4(pr.B2, baseB2, sB20, sc, k0 + bk, n0 + bc, Kd, N);
+  };
+  auto stash = [&]() {
+    if (ATRANS) {
+      *reinterpret_cast<float4*>(&sA[ar][ac]) = ra;
+    } else {
+      sA[ac + 0][ar] = ra.x; sA[ac + 1][ar] = ra.y; sA[ac + 2][ar] = ra.z; sA[ac + 3][ar] = ra.w;
+    }
+    *reinterpret_cast<float4*>(&sB[bk][bc]) = rb;
+    if constexpr (DUAL) *reinterpret_cast<float4*>(&sB2[bk][bc]) = rb2;
+  };
+
+  fetch(0);
+  for (int k0 = 0; k0 < Kd; k0 += BK) {
+    stash();
+    __syncthreads();
+    if (k0 + BK < Kd) fetch(k0 + BK);
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 a4 = *reinterpret_cast<const float4*>(&sA[kk][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&sB[kk][tx * 4]);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w};
+      const float b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+      if constexpr (DUAL) {
+        const float4 c4 = *reinterpret_cast<const float4*>(&sB2[kk][tx * 4]);
+        const float c[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float a2 = sc.a_square ? a[i] * a[i] : a[i];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc2[i][j] = fmaf(a2, c[j], acc2[i][j]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- epilogue: each thread owns rows m0+ty*4.., columns n0+tx*4..+3 (N is a multiple of 4)
+  const Epilogue& ep = pr.epi;
+  const long long col = n0 + tx * 4;
+  if (col >= N) return;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long row = m0 + ty * 4 + i;
+    if (row >= M) break;
+    if (ep.kind == EPI_STORE) {
+      *reinterpret_cast<float4*>(ep.C + row * ep.ldc + col) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    } else if (ep.kind == EPI_APPLY) {
+      if constexpr (DUAL) {
+        const long long idx = row * (long long)N + col;
+        const float c = *ep.cptr;
+        const float4 g = load4(*ep.G_ind, sc.g_dt, ep.G_off + idx);
+        const float4 w = load4(ep.W, sc.w_dt, idx);
+        float4 upd = make_float4(acc2[i][0], acc2[i][1], acc2[i][2], acc2[i][3]);
+        if (sc.form == LORDO_QHM_FULL) {
+          const float4 d = *reinterpret_cast<const float4*>(ep.dcol + col);
+          const float w1 = 1.f - sc.omega;
+          upd.x = w1 * (c * g.x) / d.x + sc.omega * upd.x;
+          upd.y = w1 * (c * g.y) / d.y + sc.omega * upd.y;
+          upd.z = w1 * (c * g.z) / d.z + sc.omega * upd.z;
+          upd.w = w1 * (c * g.w) / d.w + sc.omega * upd.w;
+        }
+        if (sc.ef) {
+          const float4 e = load4(ep.E, sc.e_dt, idx);
+          float4 en;
+          en.x = (c * g.x + e.x) - acc[i][0];
+          en.y = (c * g.y + e.y) - acc[i][1];
+          en.z = (c * g.z + e.z) - acc[i][2];
+          en.w = (c * g.w + e.w) - acc[i][3];
+          store4(ep.E, sc.e_dt, idx, en);
+        }
+        store4(ep.W, sc.w_dt, idx, make_float4(w.x - sc.lr * upd.x, w.y - sc.lr * upd.y, w.z - sc.lr * upd.z, w.w - sc.lr * upd.w));
+      }
+    } else {  // EPI_ROTATE: acc = Rot u^, acc2 = (Rot o Rot)(v^ - u^ o u^)
+      if constexpr (DUAL) {
+        const long long idx = row * (long long)N + col;
+        float4 un, vn;
+        un.x = sc.bc1 * acc[i][0]; un.y = sc.bc1 * acc[i][1]; un.z = sc.bc1 * acc[i][2]; un.w = sc.bc1 * acc[i][3];
+        vn.x = sc.bc2 * fabsf(acc2[i][0] + acc[i][0] * acc[i][0]);
+        vn.y = sc.bc2 * fabsf(acc2[i][1] + acc[i][1] * acc[i][1]);
+        vn.z = sc.bc2 * fabsf(acc2[i][2] + acc[i][2] * acc[i][2]);
+        vn.w = sc.bc2 * fabsf(acc2[i][3] + acc[i][3] * acc[i][3]);
+        *reinterpret_cast<float4*>(ep.u_out + idx) = un;
+        *reinterpret_cast<float4*>(ep.v_out + idx) = vn;
+      }
+    }
+  }
+}
+
+void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, const GemmScalars& sc,
+                 cudaStream_t st) {
+  const unsigned grid = (unsigned)total_tiles;
+  if (atrans && !dual) gemm_ffma_kernel<1, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+  else if (!atrans && !dual) gemm_ffma_kernel<0, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+  else if (!atrans && dual) gemm_ffma_kernel<0, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+  else gemm_ffma_kernel<1, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Cholesky of the Gram matrix + inverse of the triangular factor, one block per problem.
+// Left-looking column Cholesky, fp64 accumulation, L kept in global memory (L2-resident).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512) chol_inverse_kernel(const float* __restrict__ gram, float* __restrict__ lwork,
+                                                           float* __restrict__ rinv, int r, long long stride,
+                                                           unsigned* __restrict__ status) {
+  extern __shared__ float row_j[];  // r floats: row j of L (columns < j)
+  __shared__ float pivot_s;
+  __shared__ float maxdiag_s;
+  const float* A = gram + (long long)blockIdx.x * stride;
+  float* L = lwork + (long long)blockIdx.x * stride;
+  float* X = rinv + (long long)blockIdx.x * stride;
+  const int t = threadIdx.x, nt = blockDim.x;
+
+  if (t == 0) {
+    float md = 0.f;
+    for (int i = 0; i < r; ++i) md = fmaxf(md, fabsf(A[(long long)i * r + i]));
+    maxdiag_s = md;
+  }
+  __syncthreads();
+  const float floor_pivot = maxdiag_s > 0.f ? maxdiag_s * 1e-10f : 1.f;
+
+  for (int j = 0; j < r; ++j) {
+    for (int k = t; k < j; k += nt) row_j[k] = L[(long long)j * r + k];
+    __syncthreads();
+    // s_i = A[i][j] - sum_{k<j} L[i][k] L[j][k] for i >= j
+    for (int i = j + t; i < r; i += nt) {
+      const float* Li = L + (long long)i * r;
+      double s = (double)A[(long long)i * r + j];
+      for (int k = 0; k < j; ++k) s -= (double)Li[k] * (double)row_j[k];
+      if (i == j) {
+        float d = (float)s;
+        if (!(d > floor_pivot)) {  // also catches NaN
+          atomicOr(status, LORDO_FLAG_QR_BREAKDOWN);
+          d = floor_pivot;
+        }
+        pivot_s = sqrtf(d);
+      }
+      L[(long long)i * r + j] = (float)s;  // unscaled for now
+    }
+    __syncthreads();
+    const float piv = pivot_s;
+    for (int i = j + t; i < r; i += nt) {
+      float* Lij = L + (long long)i * r + j;
+      *Lij = (i == j) ? piv : (*Lij / piv);
+    }
+    __syncthreads();
+  }
+
+  // Linv: column c solved by thread c (forward substitution), kept transposed-free in X as
+  // X[i][c] = Linv[i][c]; afterwards rinv = Linv^T is produced in place through lwork.
+  for (int c = t; c < r; c += nt) {
+    for (int i = 0; i < c; ++i) X[(long long)i * r + c] = 0.f;
+    X[(long long)c * r + c] = 1.f / L[(long long)c * r + c];
+    for (int i = c + 1; i < r; ++i) {
+      const float* Li = L + (long long)i * r;
+      double s = 0.0;
+      for (int k = c; k < i; ++k) s += (double)Li[k] * (double)X[(long long)k * r + c];
+      X[(long long)i * r + c] = (float)(-s / (double)Li[i]);
+    }
+  }
+  __syncthreads();
+  // R^-1 = (L^-1)^T : transpose X through L's storage
+  for (long long e = t; e < (long long)r * r; e += nt) L[e] = X[e];
+  __syncthreads();
+  for (long long e = t; e < (long long)r * r; e += nt) {
+    const int i = (int)(e / r), c = (int)(e - (long long)i * r);
+    X[e] = L[(long long)c * r + i];
+  }
+}
+
+void launch_chol_inverse(const float* gram, float* lwork, float* rinv, int r, int batch, long long stride, unsigned* status,
+                         cudaStream_t st) {
+  chol_inverse_kernel<<<batch, 512, r * sizeof(float), st>>>(gram, lwork, rinv, r, stride, status);
+}
+
+}  // namespace lordo

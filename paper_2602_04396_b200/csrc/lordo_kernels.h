@@ -1,0 +1,90 @@
+// Internal interface between the host layer (lordo_api.cu) and the kernel files.
+#pragma once
+#include "lordo_common.cuh"
+
+namespace lordo {
+
+constexpr long long kSqChunk = 32768;  // elements per partial sum of squares
+
+struct RandomKeys {
+  unsigned long long key[64];
+};
+
+// ---------------------------------------------------------------------------------------------
+// Grouped fp32 GEMM with fused operand formation and epilogues (FFMA path).
+//   C[M x N] = A[M x Kd] * B[Kd x N]        (+ second accumulator: A' * B2, A' = A or A o A)
+// B, B2 are stored row-major [Kd][N]. A is stored [M][Kd] (ATRANS = 0) or [Kd][M] (ATRANS = 1).
+// ---------------------------------------------------------------------------------------------
+enum OperandKind {
+  OP_PLAIN = 0,  // (*s0_ptr) * p0[idx] + p1[idx]        (s0_ptr, p1 optional)
+  OP_UHAT = 1,   // inv_bc1 * p0[idx]                      bias-corrected first moment
+  OP_VRES = 2    // inv_bc2 * p1[idx] - (inv_bc1 * p0[idx])^2
+};
+
+struct Operand {
+  const void* p0;
+  const void* const* p0_ind;  // if set: p0 = *p0_ind (a per-call pointer table entry)
+  long long p0_off;           // element offset added to p0
+  const void* p1;
+  const float* s0_ptr;
+  long long ld;
+  int dt0, dt1, kind, pad;
+};
+
+enum EpilogueKind { EPI_STORE = 0, EPI_APPLY = 1, EPI_ROTATE = 2 };
+
+struct Epilogue {
+  int kind, pad;
+  float* C;         // STORE: C[row*ldc + col] = acc
+  long long ldc;
+  // APPLY (Algorithm 1: error-feedback line and the model update), row = weight row, col = column
+  void* W;
+  void* E;
+  const void* const* G_ind;
+  long long G_off;
+  const float* dcol;
+  const float* cptr;
+  // ROTATE (Algorithm 1: moment-rotation lines)
+  float* u_out;
+  float* v_out;
+};
+
+struct GemmProblem {
+  int M, N, Kd, tiles_n;
+  long long tile_start;  // first tile of this problem within its launch
+  Operand A, B, B2;
+  Epilogue epi;
+};
+
+struct GemmScalars {
+  float lr, omega, inv_bc1, inv_bc2, bc1, bc2;
+  int form, ef, w_dt, e_dt, g_dt, a_square;
+};
+
+void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, const GemmScalars& sc,
+                 cudaStream_t st);
+
+// Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
+// gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the
+// diagonal. lwork: r*r floats per problem. Strides in floats between batch entries.
+void launch_chol_inverse(const float* gram, float* lwork, float* rinv, int r, int batch, long long stride, unsigned* status,
+                         cudaStream_t st);
+
+// streaming kernels
+void launch_sumsq_partial(const MatDev* mats, const void* const* G, const long long* chunk_start, int n_mats, int K, int g_dt,
+                          double* partial, long long total_chunks, cudaStream_t st);
+void launch_clip_finalize(const MatDev* mats, const long long* chunk_start, int n_mats, int K, const double* partial, float rho,
+                          int scope, float* coef, double* sumsq, unsigned* status, cudaStream_t st);
+void launch_fill_float(float* p, long long count, float value, cudaStream_t st);
+void launch_moments(const MatDev* mats, const long long* tile_start, int n_mats, long long total_tiles, const StepScalars& sc,
+                    cudaStream_t st);
+void launch_outer_weights(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int w_dt,
+                          int outer, float eta_s, float mu_s, cudaStream_t st);
+void launch_outer_states(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int which,
+                         cudaStream_t st);
+void launch_init_weights(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int w_dt,
+                         cudaStream_t st);
+void launch_identity_projection(float* P, long long m, int r, int copies, cudaStream_t st);
+void launch_fill_random(float* out, long long count, long long batch_stride, const RandomKeys& keys, int batch, cudaStream_t st);
+
+}  // namespace lordo

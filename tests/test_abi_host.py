@@ -1,0 +1,65 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, validates configurations and sizes its workspace."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2602_04396_b200 import build as lbuild
+from paper_2602_04396_b200 import lordo
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    lbuild.build()
+    return lordo.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "lordo.h")).read()
+    declared = sorted(set(re.findall(r"LORDO_API\s+[\w\s\*]+?\b(lordo_\w+)\s*\(", header)))
+    assert len(declared) >= 15
+    assert sorted(lordo.EXPORTS) == declared
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings(lib):
+    assert lib.lordo_status_string(0) == b"ok"
+    assert b"order" in lib.lordo_status_string(4)
+
+
+def test_workspace_query_and_validation(lib):
+    cfg, _keep = lordo.make_config([(256, 256, 16)], 2, 4, clip_rho=1.0)
+    small = lordo.query_workspace(cfg)
+    cfg2, _keep2 = lordo.make_config([(256, 256, 16)] * 3, 2, 4, clip_rho=1.0)
+    assert lordo.query_workspace(cfg2) > small > 0
+    # g^ and U~ workspaces alone: 2 * K * r * n floats
+    assert small >= 2 * 2 * 16 * 256 * 4
+    bad = [
+        ([(256, 252, 16)], dict(), 3),           # n not a multiple of 8
+        ([(256, 256, 12)], dict(), 3),           # r not a multiple of 8
+        ([(16, 256, 32)], dict(), 2),            # r > m
+        ([(256, 256, 16)], dict(beta2=1.0), 1),  # beta2 out of range
+        ([(256, 256, 16)], dict(power_iters=9), 1),
+        ([(256, 256, 16)], dict(variant=5), 1),
+    ]
+    for mats, kw, code in bad:
+        cfg, _k = lordo.make_config(mats, 2, 4, **kw)
+        with pytest.raises(lordo.LordoError) as ei:
+            lordo.query_workspace(cfg)
+        assert ei.value.status == code
+    cfg, _k = lordo.make_config([(256, 256, 16)], 65, 4)
+    with pytest.raises(lordo.LordoError):
+        lordo.query_workspace(cfg)
+
+
+def test_null_arguments_are_rejected(lib):
+    assert lib.lordo_query_workspace(None, None) == 1
+    assert lib.lordo_inner_step(None, None, 0.1, 0.9, 0.9, 0, None) == 1
+    assert lib.lordo_outer_step(None, None) == 1
+    assert lib.lordo_destroy(None) == 1
+    assert lib.lordo_launch_count(None) == -1
