@@ -69,7 +69,8 @@ typedef enum { LORDO_OUTER_AVG = 0, LORDO_OUTER_NESTEROV = 1 } lordo_outer;     
 
 /* device status flags returned by lordo_poll_status */
 #define LORDO_FLAG_NONFINITE_GRAD 1u /* a gradient norm was NaN or Inf */
-#define LORDO_FLAG_QR_BREAKDOWN 2u   /* a Cholesky pivot in the QR was not positive (rank-deficient sketch) */
+#define LORDO_FLAG_QR_BREAKDOWN 2u   /* a column of a sketch was (numerically) dependent on the columns before it */
+#define LORDO_FLAG_DEVICE_TIMEOUT 4u /* a bounded wait inside a kernel gave up; results of that call are invalid */
 
 typedef struct {
   int64_t m, n; /* W is m x n */

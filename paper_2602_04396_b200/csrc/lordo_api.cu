@@ -70,6 +70,19 @@ struct lordo_ctx {
   float* d_scratch = nullptr;
   long long total_chunks = 0, total_mom_tiles = 0, total_wblks = 0, total_sblks = 0;
 
+  // tensor-core path of the inner step (check_mode == 0 and every r <= 256)
+  bool tc = false;
+  TcProblem* d_tc_probs = nullptr;
+  TcPrep* d_tc_prep = nullptr;
+  long long* d_prep_start = nullptr;
+  char* d_tc_bf16 = nullptr;  // all bf16 operand copies, zeroed once by lordo_init
+  size_t tc_bf16_bytes = 0;
+  long long tc_strips = 0, prep_blocks = 0;
+  int tc_rn_max = 0, tc_rk_max = 0;
+  std::vector<TcProblem> h_tc;
+  std::vector<TcPrep> h_prep;
+  std::vector<long long> h_prep_start;
+
   // host plans
   std::vector<GemmProblem> h_probs;
   PlanStep inner_proj, inner_apply;
@@ -194,6 +207,64 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     }
   }
   c->d_scratch = cv.take<float>(scratch_floats);
+
+  // ---------------- tensor-core operand copies and problem table ----------------
+  c->tc = cfg.check_mode == 0;
+  for (int i = 0; i < n_mats; ++i)
+    if (cfg.mats[i].r > 256) c->tc = false;  // larger ranks run on the fp32 path
+  c->h_tc.clear(); c->h_prep.clear(); c->h_prep_start.assign(1, 0);
+  c->tc_strips = 0; c->tc_rn_max = 0; c->tc_rk_max = 0;
+  if (c->tc) {
+    auto up = [](long long x, long long q) { return (x + q - 1) / q * q; };
+    (void)cv.take<char>(0);
+    const size_t bf16_begin = cv.off;
+    for (int i = 0; i < n_mats; ++i) {
+      const MatDev& md = c->h_mats[i];
+      const int r_k = (int)up(md.r, 64), r_n = (int)up(md.r, 16), m_k = (int)up(md.m, 64);
+      const int copies = local ? K : 1;
+      __nv_bfloat16* P16 = cv.take<__nv_bfloat16>((size_t)copies * m_k * r_k);
+      __nv_bfloat16* PT16 = cv.take<__nv_bfloat16>((size_t)copies * r_n * m_k);
+      __nv_bfloat16* gT16 = cv.take<__nv_bfloat16>((size_t)K * md.n * r_k);
+      __nv_bfloat16* uT16 = cv.take<__nv_bfloat16>((size_t)K * md.n * r_k);
+      if (r_n > c->tc_rn_max) c->tc_rn_max = r_n;
+      if (r_k > c->tc_rk_max) c->tc_rk_max = r_k;
+      for (int k = 0; k < copies; ++k) {
+        TcPrep pp;
+        std::memset(&pp, 0, sizeof(pp));
+        pp.P = md.P ? md.P + (long long)k * md.m * md.r : nullptr;
+        pp.P16 = P16 + (size_t)k * m_k * r_k; pp.PT16 = PT16 + (size_t)k * r_n * m_k;
+        pp.m = md.m; pp.r = md.r; pp.r_k = r_k; pp.m_k = m_k;
+        c->h_prep.push_back(pp);
+        c->h_prep_start.push_back(c->h_prep_start.back() + (md.m * md.r + 255) / 256);
+      }
+      for (int k = 0; k < K; ++k) {
+        const long long wo = (long long)k * md.m * md.n, so = (long long)k * md.r * md.n;
+        const int pk = local ? k : 0;
+        TcProblem tp;
+        std::memset(&tp, 0, sizeof(tp));
+        tp.strip_start = c->tc_strips;
+        tp.m = (int)md.m; tp.n = (int)md.n; tp.r = md.r; tp.r_k = r_k; tp.r_n = r_n; tp.m_k = m_k;
+        tp.PT16 = PT16 + (size_t)pk * r_n * m_k; tp.P16 = P16 + (size_t)pk * m_k * r_k;
+        tp.gT16 = gT16 + (size_t)k * md.n * r_k; tp.uT16 = uT16 + (size_t)k * md.n * r_k;
+        tp.u = md.u ? md.u + so : nullptr; tp.v = md.v ? md.v + so : nullptr;
+        tp.dcol = md.dcol + (long long)k * md.n;
+        if (real) {
+          tp.W = cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
+          tp.E = md.E ? (cfg.e_dtype == LORDO_F32 ? (void*)((float*)md.E + wo) : (void*)((unsigned short*)md.E + wo)) : nullptr;
+        }
+        tp.G_ind = c->d_Gtab + i; tp.G_off = wo;
+        tp.cptr = c->d_coef + (size_t)i * K + k;
+        c->h_tc.push_back(tp);
+        c->tc_strips += (md.n + 127) / 128;
+      }
+    }
+    c->d_tc_bf16 = ws ? reinterpret_cast<char*>(ws) + bf16_begin : nullptr;
+    c->tc_bf16_bytes = cv.off - bf16_begin;
+    c->prep_blocks = c->h_prep_start.back();
+    c->d_tc_probs = cv.take<TcProblem>(c->h_tc.size());
+    c->d_tc_prep = cv.take<TcPrep>(c->h_prep.size());
+    c->d_prep_start = cv.take<long long>(c->h_prep_start.size());
+  }
 
   // ---------------- launch plans ----------------
   std::vector<GemmProblem>& P = c->h_probs;
@@ -559,6 +630,13 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   INIT_CUDA(cudaMemcpyAsync(c->d_sblk_start, sb.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->d_probs, c->h_probs.data(), sizeof(GemmProblem) * c->h_probs.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
+  if (c->tc) {
+    INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));
+    INIT_CUDA(cudaMemsetAsync(c->d_tc_bf16, 0, c->tc_bf16_bytes, st));
+    INIT_CUDA(cudaMemcpyAsync(c->d_tc_probs, c->h_tc.data(), sizeof(TcProblem) * c->h_tc.size(), cudaMemcpyHostToDevice, st));
+    INIT_CUDA(cudaMemcpyAsync(c->d_tc_prep, c->h_prep.data(), sizeof(TcPrep) * c->h_prep.size(), cudaMemcpyHostToDevice, st));
+    INIT_CUDA(cudaMemcpyAsync(c->d_prep_start, c->h_prep_start.data(), 8 * c->h_prep_start.size(), cudaMemcpyHostToDevice, st));
+  }
   INIT_CUDA(cudaMemsetAsync(c->d_Gtab, 0, sizeof(void*) * nm, st));
   INIT_CUDA(cudaStreamSynchronize(st));  // the host vectors above may now be reused
 
@@ -583,6 +661,10 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   for (const PlanStep& s : c->init_steps) {
     rc = run_plan_step(c, s, sc, st);
     if (rc != LORDO_OK) return bail(rc);
+  }
+  if (c->tc) {
+    launch_prep_projection(c->d_tc_prep, c->d_prep_start, (int)c->h_prep.size(), c->prep_blocks, st);
+    c->launches += 1;
   }
   INIT_CUDA(cudaStreamSynchronize(st));
   if (cudaGetLastError() != cudaSuccess) return bail(LORDO_ERR_CUDA);
@@ -615,6 +697,26 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
   ss.lr = lr; ss.beta1 = beta1; ss.beta2 = c->cfg.beta2; ss.omega = omega; ss.eps = c->cfg.eps;
   ss.inv_bc1 = gs.inv_bc1; ss.inv_bc2 = gs.inv_bc2; ss.form = form; ss.ef = c->cfg.error_feedback; ss.K = c->K;
 
+  if (c->tc) {
+    ss.lr = lr;
+    {
+      ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
+      launch_project_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rn_max, ss, c->cfg.g_dtype, c->cfg.e_dtype,
+                        c->d_status, st);
+    }
+    {
+      ProfScope ps(c, st, PC_APPLY);
+      launch_apply_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rk_max, ss, c->cfg.g_dtype, c->cfg.e_dtype,
+                      c->cfg.w_dtype, c->d_status, st);
+    }
+    c->launches += 2;
+    rc = check_launch(c, "tensor-core inner step");
+    if (rc != LORDO_OK) return rc;
+    c->steps = s;
+    c->steps_in_round += 1;
+    c->after_outer = false;
+    return LORDO_OK;
+  }
   {
     ProfScope ps(c, st, PC_PROJECT);
     rc = run_plan_step(c, c->inner_proj, gs, st);
@@ -707,6 +809,12 @@ int lordo_refresh_subspace(lordo_ctx* c, const void* const* G, float beta1, void
     for (const PlanStep& s : c->refresh_steps) {
       if (s.phase == PH_ROTATE && !rotate) continue;
       rc = run_plan_step(c, s, gs, st);
+      if (rc != LORDO_OK) return rc;
+    }
+    if (c->tc) {  // bf16 operand copies of the new P
+      launch_prep_projection(c->d_tc_prep, c->d_prep_start, (int)c->h_prep.size(), c->prep_blocks, st);
+      c->launches += 1;
+      rc = check_launch(c, "prep_projection");
       if (rc != LORDO_OK) return rc;
     }
   }

@@ -2,6 +2,8 @@
 // mode") realisation of every contraction of the path -- P^T(cG+E), P g, P U~, the sketch and
 // subspace-iteration products, Gram matrices, R^-1 application, Rot = P'^T P and the rotation of
 // the moments. 64 x 64 output tile, 16-deep k-slices, 256 threads, 4 x 4 outputs per thread.
+// Products are formed and summed in fp32 inside a k-slice; the slice sums are carried across slices
+// in fp64, so a result is accurate to fp32 rounding whatever the contraction length.
 #include "lordo_kernels.h"
 
 namespace lordo {
@@ -86,12 +88,14 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
   const int ar = ATRANS ? (t >> 4) : (t >> 2), ac = ATRANS ? (t & 15) * 4 : (t & 3) * 4;
 
   float acc[4][4], acc2[DUAL ? 4 : 1][4];
+  double tot[4][4], tot2[DUAL ? 4 : 1][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       acc[i][j] = 0.f;
-      if constexpr (DUAL) acc2[i][j] = 0.f;
+      tot[i][j] = 0.0;
+      if constexpr (DUAL) { acc2[i][j] = 0.f; tot2[i][j] = 0.0; }
     }
 
   float4 ra, rb, rb2 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -137,8 +141,23 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
         }
       }
     }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        tot[i][j] += (double)acc[i][j];
+        acc[i][j] = 0.f;
+        if constexpr (DUAL) { tot2[i][j] += (double)acc2[i][j]; acc2[i][j] = 0.f; }
+      }
     __syncthreads();
   }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      acc[i][j] = (float)tot[i][j];
+      if constexpr (DUAL) acc2[i][j] = (float)tot2[i][j];
+    }
 
   // ---- epilogue: each thread owns rows m0+ty*4.., columns n0+tx*4..+3 (N is a multiple of 4)
   const Epilogue& ep = pr.epi;
@@ -222,7 +241,12 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const float* __restri
     maxdiag_s = md;
   }
   __syncthreads();
-  const float floor_pivot = maxdiag_s > 0.f ? maxdiag_s * 1e-10f : 1.f;
+  // A pivot is the squared distance of column j of the factored matrix from the span of the
+  // columns before it. Below kBreakdown times the column's own squared norm that distance is
+  // inside the rounding noise of an fp32 Gram matrix: the column is treated as dependent, the
+  // flag is raised and the pivot is clamped so that everything stays finite.
+  constexpr float kBreakdown = 3e-5f;
+  const float abs_floor = maxdiag_s > 0.f ? maxdiag_s * 1e-12f : 1.f;
 
   for (int j = 0; j < r; ++j) {
     for (int k = t; k < j; k += nt) row_j[k] = L[(long long)j * r + k];
@@ -234,6 +258,7 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const float* __restri
       for (int k = 0; k < j; ++k) s -= (double)Li[k] * (double)row_j[k];
       if (i == j) {
         float d = (float)s;
+        const float floor_pivot = fmaxf(kBreakdown * A[(long long)j * r + j], abs_floor);
         if (!(d > floor_pivot)) {  // also catches NaN
           atomicOr(status, LORDO_FLAG_QR_BREAKDOWN);
           d = floor_pivot;

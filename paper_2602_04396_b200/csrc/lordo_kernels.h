@@ -64,6 +64,45 @@ struct GemmScalars {
 void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, const GemmScalars& sc,
                  cudaStream_t st);
 
+// ---------------------------------------------------------------------------------------------
+// Tensor-core path of the inner step (bf16 operands, fp32 accumulation), see lordo_tc.cu.
+// One TcProblem per (matrix, worker); a launch covers `strips` 128-column strips in total.
+// ---------------------------------------------------------------------------------------------
+struct TcProblem {
+  long long strip_start;       // first strip of this problem within the launch
+  int m, n, r;
+  int r_k;                     // r rounded up to 64: k extent of P16, gT16, uT16
+  int r_n;                     // r rounded up to 16: rows of PT16
+  int m_k;                     // m rounded up to 64: k extent of PT16, rows of P16
+  const __nv_bfloat16* PT16;   // [r_n][m_k]  P^T, zero padded
+  const __nv_bfloat16* P16;    // [m_k][r_k]  P, zero padded
+  __nv_bfloat16* gT16;         // [n][r_k]    low-rank gradient, transposed
+  __nv_bfloat16* uT16;         // [n][r_k]    normalised low-rank update U~, transposed
+  float* u;                    // [r][n] of this worker
+  float* v;
+  float* dcol;                 // [n]
+  void* W;                     // [m][n] of this worker
+  void* E;
+  const void* const* G_ind;    // entry of the per-call gradient pointer table
+  long long G_off;             // element offset of this worker inside it
+  const float* cptr;           // clip coefficient
+};
+
+struct TcPrep {
+  const float* P;              // [m][r]
+  __nv_bfloat16* P16;
+  __nv_bfloat16* PT16;
+  long long m;
+  int r, r_k, m_k, pad;
+};
+
+cudaError_t tc_configure(int r_n_max, int r_k_max);
+void launch_prep_projection(const TcPrep* items, const long long* blk_start, int nitems, long long total_blocks, cudaStream_t st);
+void launch_project_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_n_max, const StepScalars& sc, int g_dt,
+                       int e_dt, unsigned* status, cudaStream_t st);
+void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_k_max, const StepScalars& sc, int g_dt,
+                     int e_dt, int w_dt, unsigned* status, cudaStream_t st);
+
 // Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
 // gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the
 // diagonal. lwork: r*r floats per problem. Strides in floats between batch entries.
