@@ -94,40 +94,71 @@ def test_nonfinite_gradient_sets_flag():
 FAST_TOL = 8 * 2.0 ** -9
 
 
-@pytest.mark.parametrize("shape", [(200, 136, 24), (320, 264, 72), (136, 520, 136), (704, 128, 256)])
+def _update_error(opt, orc, spec):
+    """|| (W - W0)_cuda - (W - W0)_oracle ||_F / || (W - W0)_oracle ||_F over all matrices."""
+    W0 = synth.init_weights(spec.wl, spec.seed)
+    num = den = 0.0
+    for i in range(len(W0)):
+        a = hz._np_state(opt.W[i]) - W0[i][None]
+        b = orc.W[i] - W0[i][None]
+        num += float(((a - b) ** 2).sum())
+        den += float((b ** 2).sum())
+    return (num / den) ** 0.5
+
+
+@pytest.mark.parametrize("shape", [(200, 136, 24), (320, 264, 72), (200, 520, 136), (704, 256, 256)])
 @pytest.mark.parametrize("form", [0, 1, 2])
 @pytest.mark.parametrize("variant", [0, 1])
 def test_fast_mode_inner_steps(shape, form, variant):
+    """eps is set to the size of a typical low-rank gradient entry, so that u^/(sqrt(v^)+eps) is a
+    smooth function of the gradient and the bf16 operand rounding shows up as a proportional error."""
     m, n, r = shape
     wl = _small(m=m, n=n, r=r, K=2, H=3, rounds=1, clip_rho=30.0)
-    spec = RunSpec(wl, variant=variant, form=form, refresh=False, lr=0.01, omega=0.9, check_mode=0)
+    spec = RunSpec(wl, variant=variant, form=form, refresh=False, lr=0.01, omega=0.9, check_mode=0, eps=0.05)
     opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
     st = hz.compare_states(opt, orc)
     assert opt.poll_status() == 0
-    # three steps of size <= lr * |U~| ~ lr: the weights may differ by FAST_TOL of that movement
-    rms_w = 0.02
-    assert st["W"] < FAST_TOL * 3 * 0.01 * 3 / rms_w and st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["E"] < FAST_TOL, st
+    assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["E"] < FAST_TOL, st
+    assert _update_error(opt, orc, spec) < FAST_TOL, _update_error(opt, orc, spec)
+    # three steps of size <= lr * |P U~| <= lr: the weights may differ by FAST_TOL of that movement
+    assert st["W"] < FAST_TOL * 3 * 0.01 / 0.02, st
+
+
+def test_fast_mode_adam_eps():
+    """With Adam's own eps = 1e-8 the first steps' update is sign-like, and an entry of the low-rank
+    gradient that is smaller than the bf16 rounding of its terms can land on the other sign; that is
+    a property of the arithmetic, so only the bulk of the update is compared."""
+    wl = _small(m=320, n=264, r=72, K=2, H=3, rounds=1, clip_rho=30.0)
+    spec = RunSpec(wl, variant=0, form=2, refresh=False, lr=0.01, omega=0.9, check_mode=0)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert opt.poll_status() == 0
+    assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["E"] < FAST_TOL, st
+    assert _update_error(opt, orc, spec) < 0.15
 
 
 def test_fast_mode_no_error_feedback_fp32_and_bf16():
     for dt in ("f32", "bf16"):
         wl = _small(m=264, n=392, r=40, K=3, H=2, rounds=2, clip_rho=30.0, w_dtype=dt, g_dtype=dt, e_dtype=dt)
-        spec = RunSpec(wl, variant=0, form=2, error_feedback=False, refresh=False, lr=0.01, omega=0.9, check_mode=0, outer=1)
+        spec = RunSpec(wl, variant=0, form=2, error_feedback=False, refresh=False, lr=0.01, omega=0.9, check_mode=0, outer=1,
+                       eps=0.05)
         opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
         st = hz.compare_states(opt, orc)
         assert opt.poll_status() == 0
-        assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["X0"] < 0.1, st
+        assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["X0"] < FAST_TOL * 4 * 0.01 / 0.02 + 4 * hz.BF16_EPS, st
 
 
 def test_fast_mode_full_loop_with_refresh():
-    """Whole loop in fast mode (refresh stays on the fp32 path): bases orthonormal, weights close."""
+    """Whole loop in fast mode. The refresh stays on the fp32 path, so each refresh, taken on the
+    CUDA path's own state, must match the oracle as tightly as in check mode."""
     wl = _small(m=264, n=200, r=32, K=2, H=2, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0)
     for variant, form in ((0, 2), (1, 1)):
         spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0)
-        opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
-        st = hz.compare_states(opt, orc)
+        opt, orc, worst = hz.run_lockstep_refresh(spec)
         assert opt.poll_status() == 0
-        assert st["P_orth"] < 1e-5 and st["W"] < 0.1, st
+        assert worst["P_angle"] < ANGLE_TOL and worst["P_orth"] < 1e-5 and worst["u"] < 1e-3 and worst["v"] < 1e-3, worst
+        for w in opt.W:
+            assert bool(torch.isfinite(w.float()).all())
 
 
 # ------------------------------------------------------------------ outer step
