@@ -209,7 +209,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   c->d_scratch = cv.take<float>(scratch_floats);
 
   // ---------------- tensor-core operand copies and problem table ----------------
-  c->tc = cfg.check_mode == 0;
+  c->tc = cfg.check_mode == 0 && cfg.g_dtype == cfg.w_dtype && (!cfg.error_feedback || cfg.e_dtype == cfg.w_dtype);
   for (int i = 0; i < n_mats; ++i)
     if (cfg.mats[i].r > 256) c->tc = false;  // larger ranks run on the fp32 path
   c->h_tc.clear(); c->h_prep.clear(); c->h_prep_start.assign(1, 0);
@@ -701,13 +701,13 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
     ss.lr = lr;
     {
       ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
-      launch_project_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rn_max, ss, c->cfg.g_dtype, c->cfg.e_dtype,
+      launch_project_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rn_max, ss, c->cfg.w_dtype == LORDO_BF16,
                         c->d_status, st);
     }
     {
       ProfScope ps(c, st, PC_APPLY);
-      launch_apply_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rk_max, ss, c->cfg.g_dtype, c->cfg.e_dtype,
-                      c->cfg.w_dtype, c->d_status, st);
+      launch_apply_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rk_max, ss, c->cfg.w_dtype == LORDO_BF16,
+                      c->d_status, st);
     }
     c->launches += 2;
     rc = check_launch(c, "tensor-core inner step");

@@ -98,10 +98,11 @@ struct TcPrep {
 
 cudaError_t tc_configure(int r_n_max, int r_k_max);
 void launch_prep_projection(const TcPrep* items, const long long* blk_start, int nitems, long long total_blocks, cudaStream_t st);
-void launch_project_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_n_max, const StepScalars& sc, int g_dt,
-                       int e_dt, unsigned* status, cudaStream_t st);
-void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_k_max, const StepScalars& sc, int g_dt,
-                     int e_dt, int w_dt, unsigned* status, cudaStream_t st);
+// bf16 != 0: G, E, W are all bf16; else all fp32 (mixed storage runs on the fp32 path).
+void launch_project_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_n_max, const StepScalars& sc, int bf16,
+                       unsigned* status, cudaStream_t st);
+void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_k_max, const StepScalars& sc, int bf16,
+                     unsigned* status, cudaStream_t st);
 
 // Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
 // gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the

@@ -23,7 +23,7 @@ namespace {
 
 constexpr int kStrip = 128;        // columns per strip = MMA M
 constexpr int kProjThreads = 288;  // 8 producer/epilogue warps + 1 MMA warp
-constexpr int kApplyEpiWarps = 16, kApplyProdWarps = 4;
+constexpr int kApplyEpiWarps = 16, kApplyProdWarps = 2;
 constexpr int kApplyThreads = (kApplyEpiWarps + kApplyProdWarps + 1) * 32;
 constexpr int kApplyRows = 64;     // rows of W per sweep step = MMA N
 
@@ -36,12 +36,29 @@ __device__ __forceinline__ int find_problem(const TcProblem* __restrict__ probs,
   return lo;
 }
 
-// two adjacent elements (row, col), (row, col+1) as floats
-__device__ __forceinline__ float2 load_pair(const void* base, int dt, long long idx) {
-  if (dt == LORDO_F32) return *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(base) + idx);
-  const uint32_t raw = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const unsigned short*>(base) + idx);
-  return make_float2(__uint_as_float(raw << 16), __uint_as_float(raw & 0xFFFF0000u));
-}
+// Storage type of G, E and W inside the tensor-core kernels: all bf16 or all fp32. Loads are kept
+// as raw values in registers (no use before the whole batch has been issued), converted afterwards.
+template <bool BF16>
+struct Elem;
+template <>
+struct Elem<true> {
+  using one = unsigned short;
+  using pair = uint32_t;
+  static __device__ __forceinline__ float cvt(one x) { return __uint_as_float(((uint32_t)x) << 16); }
+  static __device__ __forceinline__ float2 cvt2(pair x) { return make_float2(__uint_as_float(x << 16), __uint_as_float(x & 0xFFFF0000u)); }
+  static __device__ __forceinline__ one pack(float v) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    return *reinterpret_cast<const unsigned short*>(&h);
+  }
+};
+template <>
+struct Elem<false> {
+  using one = float;
+  using pair = float2;
+  static __device__ __forceinline__ float cvt(one x) { return x; }
+  static __device__ __forceinline__ float2 cvt2(pair x) { return x; }
+  static __device__ __forceinline__ one pack(float v) { return v; }
+};
 
 }  // namespace
 
@@ -65,8 +82,12 @@ __global__ void __launch_bounds__(256) prep_projection_kernel(const TcPrep* __re
 // ---------------------------------------------------------------------------------------------
 // project + moments
 // ---------------------------------------------------------------------------------------------
+template <bool BF16>
 __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcProblem* __restrict__ probs, int nprobs, StepScalars sc,
-                                                                  int g_dt, int e_dt, unsigned* __restrict__ status) {
+                                                                     unsigned* __restrict__ status) {
+  using EL = Elem<BF16>;
+  using one_t = typename EL::one;
+  using pair_t = typename EL::pair;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t full_bar[2], empty_bar[2], done_bar;
@@ -75,10 +96,10 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long strip = blockIdx.x;
-  const TcProblem& pr = probs[find_problem(probs, nprobs, strip)];
-  const int m = pr.m, n = pr.n, r = pr.r, r_n = pr.r_n;
-  const long long n0 = (strip - pr.strip_start) * kStrip;
-  const int nkb = pr.m_k / 64;
+  const TcProblem* __restrict__ prp = probs + find_problem(probs, nprobs, strip);
+  const int m = prp->m, n = prp->n, r = prp->r, r_n = prp->r_n, m_k = prp->m_k, r_k = prp->r_k;
+  const long long n0 = (strip - prp->strip_start) * kStrip;
+  const int nkb = m_k / 64;
   const uint32_t a_bytes = kStrip * 128, b_bytes = (uint32_t)r_n * 128, stage_bytes = a_bytes + ((b_bytes + 1023) & ~1023u);
   const uint32_t ncols = tmem_cols_pow2((uint32_t)r_n);
 
@@ -98,34 +119,40 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
     const int cp = tid & 63, kg = tid >> 6;  // column pair 0..63, k-group of 16 rows 0..3
     const long long col = n0 + 2 * cp;
     const bool col_ok = col < n;
-    const void* G = *pr.G_ind;
-    const float c = *pr.cptr;
+    const long long colc = col_ok ? col : (long long)n - 2;  // loads stay in bounds, results are masked
+    const one_t* __restrict__ Gp = reinterpret_cast<const one_t*>(*prp->G_ind) + prp->G_off;
     const bool have_e = sc.ef != 0;
+    const one_t* __restrict__ Ep = have_e ? reinterpret_cast<const one_t*>(prp->E) : Gp;
+    const float c = *prp->cptr;
+    const float es = have_e ? 1.f : 0.f;
+    const __nv_bfloat16* __restrict__ PT = prp->PT16;
+    const int pt_chunks = r_n * 8;
     bool ok = true;
     for (int kb = 0; kb < nkb && ok; ++kb) {
       const int s = kb & 1, use = kb >> 1;
+      pair_t rg[16], re[16];
+      const long long rbase = (long long)kb * 64 + kg * 16;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        long long row = rbase + j;
+        row = row < m ? row : (long long)m - 1;
+        const long long idx = row * n + colc;
+        rg[j] = *reinterpret_cast<const pair_t*>(Gp + idx);
+        re[j] = *reinterpret_cast<const pair_t*>(Ep + idx);
+      }
+      uint4 pt[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        int idx = tid + t * 256;
+        idx = idx < pt_chunks ? idx : pt_chunks - 1;
+        pt[t] = *reinterpret_cast<const uint4*>(PT + (long long)(idx >> 3) * m_k + kb * 64 + (idx & 7) * 8);
+      }
       float2 a[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const long long row = (long long)kb * 64 + kg * 16 + j;
-        float2 x = make_float2(0.f, 0.f);
-        if (col_ok && row < m) {
-          const long long idx = row * n + col;
-          const float2 g = load_pair(G, g_dt, pr.G_off + idx);
-          x = make_float2(c * g.x, c * g.y);
-          if (have_e) {
-            const float2 e = load_pair(pr.E, e_dt, idx);
-            x.x += e.x; x.y += e.y;
-          }
-        }
-        a[j] = x;
-      }
-      uint4 pt[8];
-      const int pt_chunks = r_n * 8;
-#pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        const int idx = tid + t * 256;
-        if (idx < pt_chunks) pt[t] = *reinterpret_cast<const uint4*>(pr.PT16 + (long long)(idx >> 3) * pr.m_k + kb * 64 + (idx & 7) * 8);
+        const float2 g = EL::cvt2(rg[j]), e = EL::cvt2(re[j]);
+        const float live = (col_ok && rbase + j < m) ? 1.f : 0.f;
+        a[j] = make_float2(live * (c * g.x + es * e.x), live * (c * g.y + es * e.y));
       }
       ok = mbar_wait(&empty_bar[s], (uint32_t)((use & 1) ^ 1), status);
       if (!ok) break;
@@ -148,7 +175,7 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
       }
       if (r_n > 256) {  // rows 256.. of the P^T tile (r up to 512)
         for (int idx = 2048 + tid; idx < pt_chunks; idx += 256) {
-          const uint4 v = *reinterpret_cast<const uint4*>(pr.PT16 + (long long)(idx >> 3) * pr.m_k + kb * 64 + (idx & 7) * 8);
+          const uint4 v = *reinterpret_cast<const uint4*>(PT + (long long)(idx >> 3) * m_k + kb * 64 + (idx & 7) * 8);
           *reinterpret_cast<uint4*>(sB + swz_chunk(idx >> 3, idx & 7)) = v;
         }
       }
@@ -162,21 +189,27 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
     const int q = warp & 3, half = warp >> 2;
     const long long ecol = n0 + q * 32 + lane;
     const bool e_ok = ok && ecol < n;
+    const long long ecolc = ecol < n ? ecol : (long long)n - 1;
+    float* __restrict__ up_ = prp->u;
+    float* __restrict__ vp_ = prp->v;
+    __nv_bfloat16* __restrict__ gT = prp->gT16 + ecolc * r_k;
+    __nv_bfloat16* __restrict__ uT = prp->uT16 + ecolc * r_k;
     const float b1 = sc.beta1, b2 = sc.beta2, w = sc.omega;
+    const bool low = sc.form == LORDO_QHM_LOW;
     float dsum = 0.f;
     for (int ch = half; ch < r_n / 16; ch += 2) {
-      float g[16];
-      tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 16), g);
       float u[16], v[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        const int row = ch * 16 + i;
-        const bool live = e_ok && row < r;
-        const long long idx = (long long)row * n + ecol;
-        u[i] = live ? pr.u[idx] : 0.f;
-        v[i] = live ? pr.v[idx] : 0.f;
+        int row = ch * 16 + i;
+        row = row < r ? row : r - 1;
+        const long long idx = (long long)row * n + ecolc;
+        u[i] = up_[idx];
+        v[i] = vp_[idx];
       }
-      uint32_t gp[8], up[8];
+      float g[16];
+      tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 16), g);
+      uint32_t gp[8], upk[8];
 #pragma unroll
       for (int i = 0; i < 16; i += 2) {
         float o[2];
@@ -188,30 +221,30 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
           const float vn = b2 * v[i + t] + (1.f - b2) * gg * gg;
           const float uh = un * sc.inv_bc1;
           const float D = sqrtf(vn * sc.inv_bc2) + sc.eps;
-          o[t] = (sc.form == LORDO_QHM_LOW) ? (w * uh + (1.f - w) * gg) / D : uh / D;
+          o[t] = low ? (w * uh + (1.f - w) * gg) / D : uh / D;
           if (e_ok && row < r) {
             const long long idx = (long long)row * n + ecol;
-            pr.u[idx] = un;
-            pr.v[idx] = vn;
+            up_[idx] = un;
+            vp_[idx] = vn;
             dsum += D;
           } else {
             o[t] = 0.f;
           }
         }
         gp[i >> 1] = pack2_bf16(g[i], g[i + 1]);
-        up[i >> 1] = pack2_bf16(o[0], o[1]);
+        upk[i >> 1] = pack2_bf16(o[0], o[1]);
       }
       if (e_ok) {
-        uint4* gd = reinterpret_cast<uint4*>(pr.gT16 + ecol * pr.r_k + ch * 16);
-        uint4* ud = reinterpret_cast<uint4*>(pr.uT16 + ecol * pr.r_k + ch * 16);
+        uint4* gd = reinterpret_cast<uint4*>(gT + ch * 16);
+        uint4* ud = reinterpret_cast<uint4*>(uT + ch * 16);
         gd[0] = make_uint4(gp[0], gp[1], gp[2], gp[3]); gd[1] = make_uint4(gp[4], gp[5], gp[6], gp[7]);
-        ud[0] = make_uint4(up[0], up[1], up[2], up[3]); ud[1] = make_uint4(up[4], up[5], up[6], up[7]);
+        ud[0] = make_uint4(upk[0], upk[1], upk[2], upk[3]); ud[1] = make_uint4(upk[4], upk[5], upk[6], upk[7]);
       }
     }
     if (sc.form == LORDO_QHM_FULL) {  // mu(D): mean over the rank axis, one value per column
       if (half == 1) dsum_s[q * 32 + lane] = dsum;
       asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (half == 0 && e_ok) pr.dcol[ecol] = (dsum + dsum_s[q * 32 + lane]) / (float)r;
+      if (half == 0 && e_ok) prp->dcol[ecol] = (dsum + dsum_s[q * 32 + lane]) / (float)r;
     }
   } else if (lane == 0) {
     // ---------------- MMA issue ---------------------------------------------------------------
@@ -242,8 +275,11 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
 // ---------------------------------------------------------------------------------------------
 // back-projection + error feedback + model update
 // ---------------------------------------------------------------------------------------------
+template <bool BF16>
 __global__ void __launch_bounds__(kApplyThreads, 1) apply_tc_kernel(const TcProblem* __restrict__ probs, int nprobs, StepScalars sc,
-                                                                    int g_dt, int e_dt, int w_dt, unsigned* __restrict__ status) {
+                                                                    unsigned* __restrict__ status) {
+  using EL = Elem<BF16>;
+  using one_t = typename EL::one;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t p_full[2], p_empty[2], acc_full[2], acc_empty[2];
@@ -251,9 +287,9 @@ __global__ void __launch_bounds__(kApplyThreads, 1) apply_tc_kernel(const TcProb
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const long long strip = blockIdx.x;
-  const TcProblem& pr = probs[find_problem(probs, nprobs, strip)];
-  const int m = pr.m, n = pr.n, r_k = pr.r_k;
-  const long long n0 = (strip - pr.strip_start) * kStrip;
+  const TcProblem* __restrict__ prp = probs + find_problem(probs, nprobs, strip);
+  const int m = prp->m, n = prp->n, r_k = prp->r_k;
+  const long long n0 = (strip - prp->strip_start) * kStrip;
   const int nkb = r_k / 64;
   const int nsteps = (m + kApplyRows - 1) / kApplyRows;
   const uint32_t x_bytes = (uint32_t)nkb * kStrip * 128;      // one resident operand (g^T or U~^T)
@@ -275,14 +311,34 @@ __global__ void __launch_bounds__(kApplyThreads, 1) apply_tc_kernel(const TcProb
   // resident operands: rows = the strip's columns, k = rank index (zero rows beyond n)
   {
     const int chunks_per_row = r_k / 8;
-    const int total = 2 * kStrip * chunks_per_row;
-    for (int idx = tid; idx < total; idx += kApplyThreads) {
-      const int which = idx >= kStrip * chunks_per_row;
-      const int rem = idx - which * kStrip * chunks_per_row;
-      const int row = rem / chunks_per_row, ch = rem - row * chunks_per_row;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (n0 + row < n) v = *reinterpret_cast<const uint4*>((which ? pr.uT16 : pr.gT16) + (n0 + row) * r_k + ch * 8);
-      *reinterpret_cast<uint4*>((which ? sX2 : sX1) + (ch >> 3) * (kStrip * 128) + swz_chunk(row, ch & 7)) = v;
+    const int per_op = kStrip * chunks_per_row;
+    const int total = 2 * per_op;
+    const __nv_bfloat16* __restrict__ g16 = prp->gT16;
+    const __nv_bfloat16* __restrict__ u16 = prp->uT16;
+    for (int base = tid; base < total; base += 4 * kApplyThreads) {
+      uint4 v[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        int idx = base + t * kApplyThreads;
+        idx = idx < total ? idx : total - 1;
+        const int which = idx >= per_op;
+        const int rem = idx - which * per_op;
+        const int row = rem / chunks_per_row, ch = rem - row * chunks_per_row;
+        long long grow = n0 + row;
+        grow = grow < n ? grow : (long long)n - 1;
+        v[t] = *reinterpret_cast<const uint4*>((which ? u16 : g16) + grow * r_k + ch * 8);
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int idx = base + t * kApplyThreads;
+        if (idx < total) {
+          const int which = idx >= per_op;
+          const int rem = idx - which * per_op;
+          const int row = rem / chunks_per_row, ch = rem - row * chunks_per_row;
+          const uint4 val = (n0 + row < n) ? v[t] : make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>((which ? sX2 : sX1) + (ch >> 3) * (kStrip * 128) + swz_chunk(row, ch & 7)) = val;
+        }
+      }
     }
   }
   fence_async_smem();
@@ -296,71 +352,70 @@ __global__ void __launch_bounds__(kApplyThreads, 1) apply_tc_kernel(const TcProb
     const int q = warp & 3, grp = warp >> 2;
     const long long col = n0 + q * 32 + lane;
     const bool col_ok = col < n;
-    const void* G = *pr.G_ind;
-    const float c = *pr.cptr;
+    const long long colc = col_ok ? col : (long long)n - 1;
+    const one_t* __restrict__ Gp = reinterpret_cast<const one_t*>(*prp->G_ind) + prp->G_off;
+    one_t* __restrict__ Wp = reinterpret_cast<one_t*>(prp->W);
+    const bool ef = sc.ef != 0;
+    one_t* __restrict__ Ep = ef ? reinterpret_cast<one_t*>(prp->E) : Wp;
+    const float c = *prp->cptr;
     const float lr = sc.lr, om = sc.omega;
-    const bool full = sc.form == LORDO_QHM_FULL, ef = sc.ef != 0;
-    const float cd = (full && col_ok) ? (1.f - om) * c / pr.dcol[col] : 0.f;
+    const bool full = sc.form == LORDO_QHM_FULL;
+    const float cd = full ? (1.f - om) * c / prp->dcol[colc] : 0.f;
+    const float a2w = full ? om : 1.f;
     bool ok = true;
     for (int t = 0; t < nsteps && ok; ++t) {
       const int b = t & 1;
       const long long row0 = (long long)t * kApplyRows + grp * 16;
-      float g[16], e[16], wv[16];
+      one_t rg[16], re[16], rw[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const bool live = col_ok && row0 + j < m;
-        const long long idx = (row0 + j) * n + col;
-        g[j] = live ? load1(G, g_dt, pr.G_off + idx) : 0.f;
-        e[j] = (live && ef) ? load1(pr.E, e_dt, idx) : 0.f;
-        wv[j] = live ? load1(pr.W, w_dt, idx) : 0.f;
+        long long row = row0 + j;
+        row = row < m ? row : (long long)m - 1;
+        const long long idx = row * n + colc;
+        rg[j] = Gp[idx];
+        re[j] = Ep[idx];
+        rw[j] = Wp[idx];
       }
       ok = mbar_wait(&acc_full[b], (uint32_t)((t >> 1) & 1), status);
       if (!ok) break;
       tc_fence_after_sync();
-      float a1[16], a2[16];
       const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 128 + grp * 16);
-      tmem_ld16(taddr, a1);
-      tmem_ld16(taddr + 64, a2);
+      float acc[16];
+      tmem_ld16(taddr, acc);  // (P g)^T
+      if (ef) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (col_ok && row0 + j < m) Ep[(row0 + j) * n + col] = EL::pack((c * EL::cvt(rg[j]) + EL::cvt(re[j])) - acc[j]);
+      }
+      tmem_ld16(taddr + 64, acc);  // (P U~)^T
       tc_fence_before_sync();
       mbar_arrive(&acc_empty[b]);
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        if (col_ok && row0 + j < m) {
-          const long long idx = (row0 + j) * n + col;
-          const float upd = full ? cd * g[j] + om * a2[j] : a2[j];
-          if (ef) store1(pr.E, e_dt, idx, (c * g[j] + e[j]) - a1[j]);
-          store1(pr.W, w_dt, idx, wv[j] - lr * upd);
-        }
-      }
+      for (int j = 0; j < 16; ++j)
+        if (col_ok && row0 + j < m)
+          Wp[(row0 + j) * n + col] = EL::pack(EL::cvt(rw[j]) - lr * (cd * EL::cvt(rg[j]) + a2w * acc[j]));
     }
   } else if (warp < kApplyEpiWarps + kApplyProdWarps) {
-    // ---------------- producers: rows of P for the next step ----------------------------------
+    // ---------------- producers: rows of P for the next step (asynchronous 16-byte copies) -----
     const int ptid = tid - kApplyEpiWarps * 32;
     const int chunks_per_row = r_k / 8;
-    const int total = kApplyRows * chunks_per_row;  // <= 2048 for r_k <= 256
+    const int total = kApplyRows * chunks_per_row;
+    const __nv_bfloat16* __restrict__ P16 = prp->P16;
     bool ok = true;
     for (int t = 0; t < nsteps && ok; ++t) {
       const int s = t & 1;
-      uint4 v[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int idx = ptid + i * (kApplyProdWarps * 32);
-        if (idx < total) {
-          const int row = idx / chunks_per_row, ch = idx - row * chunks_per_row;
-          v[i] = *reinterpret_cast<const uint4*>(pr.P16 + ((long long)t * kApplyRows + row) * r_k + ch * 8);
-        }
-      }
       ok = mbar_wait(&p_empty[s], (uint32_t)(((t >> 1) & 1) ^ 1), status);
       if (!ok) break;
-      unsigned char* dst = sP + s * p_bytes;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int idx = ptid + i * (kApplyProdWarps * 32);
-        if (idx < total) {
-          const int row = idx / chunks_per_row, ch = idx - row * chunks_per_row;
-          *reinterpret_cast<uint4*>(dst + (ch >> 3) * (kApplyRows * 128) + swz_chunk(row, ch & 7)) = v[i];
-        }
+      const uint32_t dst = smem_u32(sP + s * p_bytes);
+      for (int idx = ptid; idx < total; idx += kApplyProdWarps * 32) {
+        const int row = idx / chunks_per_row, ch = idx - row * chunks_per_row;
+        const __nv_bfloat16* src = P16 + ((long long)t * kApplyRows + row) * r_k + ch * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (ch >> 3) * (kApplyRows * 128) + swz_chunk(row, ch & 7)),
+                     "l"(src)
+                     : "memory");
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
       fence_async_smem();
       mbar_arrive(&p_full[s]);
     }
@@ -407,21 +462,27 @@ size_t apply_tc_smem(int r_k_max) {
 }
 
 cudaError_t tc_configure(int r_n_max, int r_k_max) {
-  cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)project_tc_smem(r_n_max));
+  cudaError_t e = cudaFuncSetAttribute(project_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)project_tc_smem(r_n_max));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(apply_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_tc_smem(r_k_max));
+  e = cudaFuncSetAttribute(project_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)project_tc_smem(r_n_max));
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(apply_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_tc_smem(r_k_max));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(apply_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apply_tc_smem(r_k_max));
 }
 
 void launch_prep_projection(const TcPrep* items, const long long* blk_start, int nitems, long long total_blocks, cudaStream_t st) {
   prep_projection_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(items, blk_start, nitems);
 }
-void launch_project_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_n_max, const StepScalars& sc, int g_dt,
-                       int e_dt, unsigned* status, cudaStream_t st) {
-  project_tc_kernel<<<(unsigned)total_strips, kProjThreads, project_tc_smem(r_n_max), st>>>(probs, nprobs, sc, g_dt, e_dt, status);
+void launch_project_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_n_max, const StepScalars& sc, int bf16,
+                       unsigned* status, cudaStream_t st) {
+  if (bf16) project_tc_kernel<true><<<(unsigned)total_strips, kProjThreads, project_tc_smem(r_n_max), st>>>(probs, nprobs, sc, status);
+  else project_tc_kernel<false><<<(unsigned)total_strips, kProjThreads, project_tc_smem(r_n_max), st>>>(probs, nprobs, sc, status);
 }
-void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_k_max, const StepScalars& sc, int g_dt,
-                     int e_dt, int w_dt, unsigned* status, cudaStream_t st) {
-  apply_tc_kernel<<<(unsigned)total_strips, kApplyThreads, apply_tc_smem(r_k_max), st>>>(probs, nprobs, sc, g_dt, e_dt, w_dt, status);
+void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_k_max, const StepScalars& sc, int bf16,
+                     unsigned* status, cudaStream_t st) {
+  if (bf16) apply_tc_kernel<true><<<(unsigned)total_strips, kApplyThreads, apply_tc_smem(r_k_max), st>>>(probs, nprobs, sc, status);
+  else apply_tc_kernel<false><<<(unsigned)total_strips, kApplyThreads, apply_tc_smem(r_k_max), st>>>(probs, nprobs, sc, status);
 }
 
 }  // namespace lordo
