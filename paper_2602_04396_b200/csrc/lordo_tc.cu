@@ -123,6 +123,8 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
     const one_t* __restrict__ Gp = reinterpret_cast<const one_t*>(*prp->G_ind) + prp->G_off;
     const bool have_e = sc.ef != 0;
     const one_t* __restrict__ Ep = have_e ? reinterpret_cast<const one_t*>(prp->E) : Gp;
+    const one_t* __restrict__ Gc = Gp + colc;
+    const one_t* __restrict__ Ec = Ep + colc;
     const float c = *prp->cptr;
     const float es = have_e ? 1.f : 0.f;
     const __nv_bfloat16* __restrict__ PT = prp->PT16;
@@ -131,14 +133,21 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
     for (int kb = 0; kb < nkb && ok; ++kb) {
       const int s = kb & 1, use = kb >> 1;
       pair_t rg[16], re[16];
-      const long long rbase = (long long)kb * 64 + kg * 16;
+      const int rbase = kb * 64 + kg * 16;
+      if (rbase + 16 <= m) {
+        const size_t base = (size_t)rbase * (size_t)n;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        long long row = rbase + j;
-        row = row < m ? row : (long long)m - 1;
-        const long long idx = row * n + colc;
-        rg[j] = *reinterpret_cast<const pair_t*>(Gp + idx);
-        re[j] = *reinterpret_cast<const pair_t*>(Ep + idx);
+        for (int j = 0; j < 16; ++j) {
+          rg[j] = *reinterpret_cast<const pair_t*>(Gc + base + (size_t)(unsigned)(j * n));
+          re[j] = *reinterpret_cast<const pair_t*>(Ec + base + (size_t)(unsigned)(j * n));
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const size_t off = (size_t)(unsigned)min(rbase + j, m - 1) * (size_t)n;
+          rg[j] = *reinterpret_cast<const pair_t*>(Gc + off);
+          re[j] = *reinterpret_cast<const pair_t*>(Ec + off);
+        }
       }
       uint4 pt[8];
 #pragma unroll
@@ -184,7 +193,7 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
     }
 
     // ---------------- epilogue: moments on this thread's column ------------------------------
-    if (ok) ok = mbar_wait(&done_bar, 0u, status);
+    if (ok) ok = mbar_wait<64>(&done_bar, 0u, status);
     tc_fence_after_sync();
     const int q = warp & 3, half = warp >> 2;
     const long long ecol = n0 + q * 32 + lane;
@@ -201,9 +210,7 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
       float u[16], v[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
-        int row = ch * 16 + i;
-        row = row < r ? row : r - 1;
-        const long long idx = (long long)row * n + ecolc;
+        const size_t idx = (size_t)(unsigned)min(ch * 16 + i, r - 1) * (size_t)n + (size_t)ecolc;
         u[i] = up_[idx];
         v[i] = vp_[idx];
       }
@@ -223,7 +230,7 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
           const float D = sqrtf(vn * sc.inv_bc2) + sc.eps;
           o[t] = low ? (w * uh + (1.f - w) * gg) / D : uh / D;
           if (e_ok && row < r) {
-            const long long idx = (long long)row * n + ecol;
+            const size_t idx = (size_t)(unsigned)row * (size_t)n + (size_t)ecol;
             up_[idx] = un;
             vp_[idx] = vn;
             dsum += D;
@@ -362,38 +369,63 @@ __global__ void __launch_bounds__(kApplyThreads, 1) apply_tc_kernel(const TcProb
     const bool full = sc.form == LORDO_QHM_FULL;
     const float cd = full ? (1.f - om) * c / prp->dcol[colc] : 0.f;
     const float a2w = full ? om : 1.f;
+    const one_t* __restrict__ Gc = Gp + colc;
+    one_t* __restrict__ Ec = Ep + colc;
+    one_t* __restrict__ Wc = Wp + colc;
     bool ok = true;
     for (int t = 0; t < nsteps && ok; ++t) {
       const int b = t & 1;
-      const long long row0 = (long long)t * kApplyRows + grp * 16;
+      const int row0 = t * kApplyRows + grp * 16;
+      const bool whole = row0 + 16 <= m;
+      const size_t base = (size_t)(unsigned)min(row0, m - 1) * (size_t)n;
       one_t rg[16], re[16], rw[16];
+      if (whole) {
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        long long row = row0 + j;
-        row = row < m ? row : (long long)m - 1;
-        const long long idx = row * n + colc;
-        rg[j] = Gp[idx];
-        re[j] = Ep[idx];
-        rw[j] = Wp[idx];
+        for (int j = 0; j < 16; ++j) {
+          const size_t off = base + (size_t)(unsigned)(j * n);
+          rg[j] = Gc[off];
+          re[j] = Ec[off];
+          rw[j] = Wc[off];
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const size_t off = (size_t)(unsigned)min(row0 + j, m - 1) * (size_t)n;
+          rg[j] = Gc[off];
+          re[j] = Ec[off];
+          rw[j] = Wc[off];
+        }
       }
-      ok = mbar_wait(&acc_full[b], (uint32_t)((t >> 1) & 1), status);
+      ok = mbar_wait<40>(&acc_full[b], (uint32_t)((t >> 1) & 1), status);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * 128 + grp * 16);
       float acc[16];
       tmem_ld16(taddr, acc);  // (P g)^T
-      if (ef) {
+      if (ef && col_ok) {
+        if (whole) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (col_ok && row0 + j < m) Ep[(row0 + j) * n + col] = EL::pack((c * EL::cvt(rg[j]) + EL::cvt(re[j])) - acc[j]);
+          for (int j = 0; j < 16; ++j) Ec[base + (size_t)(unsigned)(j * n)] = EL::pack((c * EL::cvt(rg[j]) + EL::cvt(re[j])) - acc[j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (row0 + j < m) Ec[base + (size_t)(unsigned)(j * n)] = EL::pack((c * EL::cvt(rg[j]) + EL::cvt(re[j])) - acc[j]);
+        }
       }
       tmem_ld16(taddr + 64, acc);  // (P U~)^T
       tc_fence_before_sync();
       mbar_arrive(&acc_empty[b]);
+      if (col_ok) {
+        if (whole) {
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        if (col_ok && row0 + j < m)
-          Wp[(row0 + j) * n + col] = EL::pack(EL::cvt(rw[j]) - lr * (cd * EL::cvt(rg[j]) + a2w * acc[j]));
+          for (int j = 0; j < 16; ++j)
+            Wc[base + (size_t)(unsigned)(j * n)] = EL::pack(EL::cvt(rw[j]) - lr * (cd * EL::cvt(rg[j]) + a2w * acc[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (row0 + j < m) Wc[base + (size_t)(unsigned)(j * n)] = EL::pack(EL::cvt(rw[j]) - lr * (cd * EL::cvt(rg[j]) + a2w * acc[j]));
+        }
+      }
     }
   } else if (warp < kApplyEpiWarps + kApplyProdWarps) {
     // ---------------- producers: rows of P for the next step (asynchronous 16-byte copies) -----

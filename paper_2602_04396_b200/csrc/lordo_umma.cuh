@@ -40,10 +40,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Returns false (after setting *timed_out) if the phase did not complete within the limit.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* timed_out) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
+    if (kSleepNs > 0) __nanosleep(kSleepNs);  // keeps many pollers out of the issue slots of the working warps
     if (clock64() - t0 > kWaitLimitCycles) {
       atomicOr(timed_out, LORDO_FLAG_DEVICE_TIMEOUT);
       return false;
