@@ -16,25 +16,38 @@ constexpr int kMaxK = 64;
 enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3 };
 enum Phase { PH_SUBSPACE = 0, PH_ROTATE = 1, PH_COMMIT = 2 };
 
+// One launch of the refresh / init / inner-step plans. The entries it works on are a contiguous
+// range [first, first + count) of the table of its type (GEMM problems, Cholesky problems, ...).
 struct PlanStep {
   int type = ST_GEMM, phase = PH_SUBSPACE;
-  // gemm
-  int atrans = 0, dual = 0, a_square = 0, nprobs = 0;
-  long long prob_first = 0, tiles = 0;
-  // chol
-  const float* gram = nullptr;
-  float* lwork = nullptr;
-  float* rinv = nullptr;
-  int r = 0, batch = 0;
-  long long stride = 0;
-  // random fill
-  float* out = nullptr;
-  long long count = 0;
-  int purpose = 0, mat = 0, per_replica = 0;
-  // copy
-  void* dst = nullptr;
-  const void* src = nullptr;
-  size_t bytes = 0;
+  int atrans = 0, dual = 0, a_square = 0;  // gemm
+  int r_max = 0;                           // chol
+  int p0 = 0;                              // random: 1 = initial projection (draw index 0), 0 = sketch (index = refresh count)
+  long long first = 0, tiles = 0;          // tiles: gemm tiles or 256-thread blocks
+  int count = 0;
+};
+
+// Collects, slot by slot, the entries of many matrices that run the same sequence of steps, so
+// that each step of the sequence becomes one launch over all of them.
+struct SlotBuilder {
+  struct Slot {
+    PlanStep st;
+    std::vector<GemmProblem> g;
+    std::vector<CholProblem> ch;
+    std::vector<RandProblem> rn;
+    std::vector<CopyProblem> cp;
+  };
+  std::vector<Slot> slots;
+  size_t cur = 0;
+  void rewind() { cur = 0; }
+  Slot& next(int type, int phase, int atrans = 0, int dual = 0, int a_square = 0, int p0 = 0) {
+    if (cur == slots.size()) {
+      Slot sl;
+      sl.st.type = type; sl.st.phase = phase; sl.st.atrans = atrans; sl.st.dual = dual; sl.st.a_square = a_square; sl.st.p0 = p0;
+      slots.push_back(sl);
+    }
+    return slots[cur++];
+  }
 };
 
 // Bump allocator over the workspace; with base == nullptr it only measures.
@@ -67,6 +80,9 @@ struct lordo_ctx {
   float* d_coef = nullptr;
   unsigned* d_status = nullptr;
   GemmProblem* d_probs = nullptr;
+  CholProblem* d_chols = nullptr;
+  RandProblem* d_rands = nullptr;
+  CopyProblem* d_copies = nullptr;
   float* d_scratch = nullptr;
   long long total_chunks = 0, total_mom_tiles = 0, total_wblks = 0, total_sblks = 0;
 
@@ -85,6 +101,9 @@ struct lordo_ctx {
 
   // host plans
   std::vector<GemmProblem> h_probs;
+  std::vector<CholProblem> h_chols;
+  std::vector<RandProblem> h_rands;
+  std::vector<CopyProblem> h_copies;
   PlanStep inner_proj, inner_apply;
   std::vector<PlanStep> refresh_steps, init_steps;
 
@@ -177,14 +196,27 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
 
   std::vector<long long> chunk_start, mom_start, wblk, sblk;
   prefix_arrays(cfg, chunk_start, mom_start, wblk, sblk);
+  // Refresh scratch: matrices are processed in groups whose scratch fits kRefreshScratchFloats;
+  // every step of the refresh is one launch over a whole group.
+  constexpr size_t kRefreshScratchFloats = size_t(1) << 30;  // 4 GiB
+  std::vector<size_t> mat_scratch(n_mats);
+  std::vector<int> group_of(n_mats);
   size_t scratch_floats = 0;
-  for (int i = 0; i < n_mats; ++i) {
-    const lordo_mat& a = cfg.mats[i];
-    const long long maxd = a.m > a.n ? a.m : a.n;
-    const size_t nb = local ? K : 1;
-    const size_t per = (size_t)a.n * a.r + 2 * (size_t)a.m * a.r + (size_t)maxd * a.r + (q > 0 ? 2 * (size_t)a.n * a.r : 0) +
-                       4 * (size_t)a.r * a.r;
-    if (nb * per > scratch_floats) scratch_floats = nb * per;
+  {
+    size_t acc = 0;
+    int grp = 0;
+    for (int i = 0; i < n_mats; ++i) {
+      const lordo_mat& a = cfg.mats[i];
+      const long long maxd = a.m > a.n ? a.m : a.n;
+      const size_t nb = local ? K : 1;
+      const size_t per = (size_t)a.n * a.r + 2 * (size_t)a.m * a.r + (size_t)maxd * a.r + (q > 0 ? 2 * (size_t)a.n * a.r : 0) +
+                         4 * (size_t)a.r * a.r;
+      mat_scratch[i] = nb * per;
+      if (acc > 0 && acc + mat_scratch[i] > kRefreshScratchFloats) { ++grp; acc = 0; }
+      group_of[i] = grp;
+      acc += mat_scratch[i];
+      if (acc > scratch_floats) scratch_floats = acc;
+    }
   }
   c->total_chunks = chunk_start[n_mats];
   c->total_mom_tiles = mom_start[n_mats];
@@ -268,25 +300,16 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
 
   // ---------------- launch plans ----------------
   std::vector<GemmProblem>& P = c->h_probs;
-  P.clear();
-  auto begin_gemm = [&](int atrans, int dual, int a_square, int phase) {
-    PlanStep s;
-    s.type = ST_GEMM; s.atrans = atrans; s.dual = dual; s.a_square = a_square; s.phase = phase;
-    s.prob_first = (long long)P.size(); s.nprobs = 0; s.tiles = 0;
-    return s;
-  };
-  auto add_prob = [&](PlanStep& s, int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
+  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear();
+  auto gemm_prob = [&](int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
     GemmProblem g;
     std::memset(&g, 0, sizeof(g));
     g.M = M; g.N = N; g.Kd = Kd;
     g.tiles_n = (N + 63) / 64;
-    g.tile_start = s.tiles;
     g.A = A; g.B = B;
     if (B2) g.B2 = *B2; else g.B2 = B;
     g.epi = ep;
-    s.tiles += (long long)((M + 63) / 64) * g.tiles_n;
-    s.nprobs += 1;
-    P.push_back(g);
+    return g;
   };
   auto store_epi = [](float* C, long long ldc) {
     Epilogue e;
@@ -294,168 +317,198 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     e.kind = EPI_STORE; e.C = C; e.ldc = ldc;
     return e;
   };
+  // Turns the slots of a builder into launches, appending their entries to the tables.
+  auto flatten = [&](SlotBuilder& sb, std::vector<PlanStep>& out) {
+    for (SlotBuilder::Slot& sl : sb.slots) {
+      PlanStep st = sl.st;
+      if (st.type == ST_GEMM) {
+        st.first = (long long)P.size(); st.count = (int)sl.g.size(); st.tiles = 0;
+        for (GemmProblem& g : sl.g) {
+          g.tile_start = st.tiles;
+          st.tiles += (long long)((g.M + 63) / 64) * g.tiles_n;
+          P.push_back(g);
+        }
+      } else if (st.type == ST_CHOL) {
+        st.first = (long long)c->h_chols.size(); st.count = (int)sl.ch.size(); st.r_max = 0;
+        for (const CholProblem& x : sl.ch) { if (x.r > st.r_max) st.r_max = x.r; c->h_chols.push_back(x); }
+      } else if (st.type == ST_RANDOM) {
+        st.first = (long long)c->h_rands.size(); st.count = (int)sl.rn.size(); st.tiles = 0;
+        for (RandProblem& x : sl.rn) { x.blk_start = st.tiles; st.tiles += (x.count + 255) / 256; c->h_rands.push_back(x); }
+      } else {
+        st.first = (long long)c->h_copies.size(); st.count = (int)sl.cp.size(); st.tiles = 0;
+        for (CopyProblem& x : sl.cp) { x.blk_start = st.tiles; st.tiles += (x.chunks + 1023) / 1024; c->h_copies.push_back(x); }
+      }
+      out.push_back(st);
+    }
+  };
+  auto add_copy = [](SlotBuilder& sb, int phase, void* dst, const void* src, size_t bytes) {
+    CopyProblem cp;
+    cp.dst = dst; cp.src = src; cp.chunks = (long long)(bytes / 16); cp.blk_start = 0;
+    sb.next(ST_COPY, phase).cp.push_back(cp);
+  };
 
   // inner step: g = P^T (c G + E)   and   E' = A - P g ; W' = W - lr (...)
-  c->inner_proj = begin_gemm(1, 0, 0, 0);
-  for (int i = 0; i < n_mats; ++i) {
-    const MatDev& md = c->h_mats[i];
-    for (int k = 0; k < K; ++k) {
-      Operand A = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
-      Operand B = plain(nullptr, md.n, cfg.g_dtype);
-      B.p0_ind = c->d_Gtab + i; B.p0_off = (long long)k * md.m * md.n;
-      B.s0_ptr = c->d_coef + (size_t)i * K + k;
-      if (cfg.error_feedback && real) {
-        B.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + (long long)k * md.m * md.n)
-                                        : (const void*)((const unsigned short*)md.E + (long long)k * md.m * md.n);
-        B.dt1 = cfg.e_dtype;
+  {
+    SlotBuilder sb;
+    for (int i = 0; i < n_mats; ++i) {
+      const MatDev& md = c->h_mats[i];
+      for (int k = 0; k < K; ++k) {
+        sb.rewind();
+        const long long wo = (long long)k * md.m * md.n;
+        Operand A = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
+        Operand B = plain(nullptr, md.n, cfg.g_dtype);
+        B.p0_ind = c->d_Gtab + i; B.p0_off = wo;
+        B.s0_ptr = c->d_coef + (size_t)i * K + k;
+        if (cfg.error_feedback && real) {
+          B.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + wo) : (const void*)((const unsigned short*)md.E + wo);
+          B.dt1 = cfg.e_dtype;
+        }
+        sb.next(ST_GEMM, 0, 1, 0, 0).g.push_back(gemm_prob(md.r, (int)md.n, (int)md.m, A, B, nullptr, store_epi(md.ghat + (long long)k * md.r * md.n, md.n)));
+        Operand B1 = plain(md.ghat + (long long)k * md.r * md.n, md.n);
+        Operand B2 = plain(md.util + (long long)k * md.r * md.n, md.n);
+        Epilogue e;
+        std::memset(&e, 0, sizeof(e));
+        e.kind = EPI_APPLY;
+        e.W = !real ? nullptr : cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
+        e.E = md.E ? (cfg.e_dtype == LORDO_F32 ? (void*)((float*)md.E + wo) : (void*)((unsigned short*)md.E + wo)) : nullptr;
+        e.G_ind = c->d_Gtab + i; e.G_off = wo;
+        e.dcol = md.dcol + (long long)k * md.n;
+        e.cptr = c->d_coef + (size_t)i * K + k;
+        sb.next(ST_GEMM, 0, 0, 1, 0).g.push_back(gemm_prob((int)md.m, (int)md.n, md.r, A, B1, &B2, e));
       }
-      add_prob(c->inner_proj, md.r, (int)md.n, (int)md.m, A, B, nullptr, store_epi(md.ghat + (long long)k * md.r * md.n, md.n));
     }
-  }
-  c->inner_apply = begin_gemm(0, 1, 0, 0);
-  for (int i = 0; i < n_mats; ++i) {
-    const MatDev& md = c->h_mats[i];
-    for (int k = 0; k < K; ++k) {
-      const long long wo = (long long)k * md.m * md.n;
-      Operand A = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
-      Operand B = plain(md.ghat + (long long)k * md.r * md.n, md.n);
-      Operand B2 = plain(md.util + (long long)k * md.r * md.n, md.n);
-      Epilogue e;
-      std::memset(&e, 0, sizeof(e));
-      e.kind = EPI_APPLY;
-      e.W = !real ? nullptr : cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
-      e.E = md.E ? (cfg.e_dtype == LORDO_F32 ? (void*)((float*)md.E + wo) : (void*)((unsigned short*)md.E + wo)) : nullptr;
-      e.G_ind = c->d_Gtab + i; e.G_off = wo;
-      e.dcol = md.dcol + (long long)k * md.n;
-      e.cptr = c->d_coef + (size_t)i * K + k;
-      add_prob(c->inner_apply, (int)md.m, (int)md.n, md.r, A, B, &B2, e);
-    }
+    std::vector<PlanStep> two;
+    flatten(sb, two);
+    c->inner_proj = two[0];
+    c->inner_apply = two[1];
   }
 
   // CholeskyQR2 of X (rows x r, batch of nb with stride sx) into O, through T.
-  auto cholqr2 = [&](std::vector<PlanStep>& plan, int phase, float* X, long long sx, float* T, long long st, float* O, long long so,
+  auto cholqr2 = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so,
                      long long rows, int r, int nb, float* gram, float* lw, float* rinv) {
     float* src = X; long long ss = sx;
     for (int pass = 0; pass < 2; ++pass) {
       float* dst = pass == 0 ? T : O;
       const long long sd = pass == 0 ? st : so;
-      PlanStep g = begin_gemm(1, 0, 0, phase);
+      SlotBuilder::Slot& g = sb.next(ST_GEMM, phase, 1, 0, 0);
       for (int b = 0; b < nb; ++b) {
         Operand A = plain(src + b * ss, r), B = plain(src + b * ss, r);
-        add_prob(g, r, r, (int)rows, A, B, nullptr, store_epi(gram + (long long)b * r * r, r));
+        g.g.push_back(gemm_prob(r, r, (int)rows, A, B, nullptr, store_epi(gram + (long long)b * r * r, r)));
       }
-      plan.push_back(g);
-      PlanStep ch;
-      ch.type = ST_CHOL; ch.phase = phase; ch.gram = gram; ch.lwork = lw; ch.rinv = rinv; ch.r = r; ch.batch = nb; ch.stride = (long long)r * r;
-      plan.push_back(ch);
-      PlanStep ap = begin_gemm(0, 0, 0, phase);
+      SlotBuilder::Slot& ch = sb.next(ST_CHOL, phase);
+      for (int b = 0; b < nb; ++b) {
+        CholProblem cp;
+        cp.gram = gram + (long long)b * r * r; cp.lwork = lw + (long long)b * r * r; cp.rinv = rinv + (long long)b * r * r; cp.r = r; cp.pad = 0;
+        ch.ch.push_back(cp);
+      }
+      SlotBuilder::Slot& ap = sb.next(ST_GEMM, phase, 0, 0, 0);
       for (int b = 0; b < nb; ++b) {
         Operand A = plain(src + b * ss, r), B = plain(rinv + (long long)b * r * r, r);
-        add_prob(ap, (int)rows, r, r, A, B, nullptr, store_epi(dst + b * sd, r));
+        ap.g.push_back(gemm_prob((int)rows, r, r, A, B, nullptr, store_epi(dst + b * sd, r)));
       }
-      plan.push_back(ap);
       src = dst; ss = sd;
     }
   };
 
   c->refresh_steps.clear();
   c->init_steps.clear();
-  for (int i = 0; i < n_mats; ++i) {
-    const MatDev& md = c->h_mats[i];
-    const long long m = md.m, n = md.n;
-    const int r = md.r;
-    const int nb = local ? K : 1;
-    const long long maxd = m > n ? m : n;
-    // scratch carve (batch-strided arrays)
-    float* s = c->d_scratch;
-    float* Om = s; s += (size_t)nb * n * r;
-    float* Ya = s; s += (size_t)nb * m * r;
-    float* Pn = s; s += (size_t)nb * m * r;
-    float* Yb = s; s += (size_t)nb * maxd * r;
-    float *Za = nullptr, *Zq = nullptr;
-    if (q > 0) { Za = s; s += (size_t)nb * n * r; Zq = s; s += (size_t)nb * n * r; }
-    float* gram = s; s += (size_t)nb * r * r;
-    float* lw = s; s += (size_t)nb * r * r;
-    float* rinv = s; s += (size_t)nb * r * r;
-    float* rot = s; s += (size_t)nb * r * r;
+  const int n_groups = n_mats ? group_of[n_mats - 1] + 1 : 0;
+  for (int grp = 0; grp < n_groups; ++grp) {
+    SlotBuilder R, I;
+    size_t goff = 0;
+    for (int i = 0; i < n_mats; ++i) {
+      if (group_of[i] != grp) continue;
+      R.rewind(); I.rewind();
+      const MatDev& md = c->h_mats[i];
+      const long long m = md.m, n = md.n;
+      const int r = md.r;
+      const int nb = local ? K : 1;
+      const long long maxd = m > n ? m : n;
+      // scratch carve of this matrix inside its group (batch-strided arrays)
+      float* s = c->d_scratch + goff;
+      goff += mat_scratch[i];
+      float* Om = s; s += (size_t)nb * n * r;
+      float* Ya = s; s += (size_t)nb * m * r;
+      float* Pn = s; s += (size_t)nb * m * r;
+      float* Yb = s; s += (size_t)nb * maxd * r;
+      float *Za = nullptr, *Zq = nullptr;
+      if (q > 0) { Za = s; s += (size_t)nb * n * r; Zq = s; s += (size_t)nb * n * r; }
+      float* gram = s; s += (size_t)nb * r * r;
+      float* lw = s; s += (size_t)nb * r * r;
+      float* rinv = s; s += (size_t)nb * r * r;
+      float* rot = s; s += (size_t)nb * r * r;
 
-    auto signal = [&](int b) {  // S of problem b: Delta (Global) or c_k G_k + E_k (Local), stored [m][n]
-      if (!local) return plain(md.Delta, n);
-      Operand A = plain(nullptr, n, cfg.g_dtype);
-      A.p0_ind = c->d_Gtab + i; A.p0_off = (long long)b * m * n;
-      A.s0_ptr = c->d_coef + (size_t)i * K + b;
-      if (cfg.error_feedback && real) {
-        A.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + (long long)b * m * n)
-                                        : (const void*)((const unsigned short*)md.E + (long long)b * m * n);
-        A.dt1 = cfg.e_dtype;
+      auto signal = [&](int b) {  // S of problem b: Delta (Global) or c_k G_k + E_k (Local), stored [m][n]
+        if (!local) return plain(md.Delta, n);
+        Operand A = plain(nullptr, n, cfg.g_dtype);
+        A.p0_ind = c->d_Gtab + i; A.p0_off = (long long)b * m * n;
+        A.s0_ptr = c->d_coef + (size_t)i * K + b;
+        if (cfg.error_feedback && real) {
+          A.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + (long long)b * m * n)
+                                          : (const void*)((const unsigned short*)md.E + (long long)b * m * n);
+          A.dt1 = cfg.e_dtype;
+        }
+        return A;
+      };
+      {
+        SlotBuilder::Slot& f = R.next(ST_RANDOM, PH_SUBSPACE);
+        for (int b = 0; b < nb; ++b) {
+          RandProblem rp;
+          rp.out = Om + (long long)b * n * r; rp.count = n * r; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
+          f.rn.push_back(rp);
+        }
       }
-      return A;
-    };
-    std::vector<PlanStep>& R = c->refresh_steps;
-    {
-      PlanStep f;
-      f.type = ST_RANDOM; f.phase = PH_SUBSPACE; f.out = Om; f.count = n * r; f.purpose = 2; f.mat = i; f.per_replica = local ? 1 : 0;
-      f.batch = nb;
-      R.push_back(f);
-    }
-    {  // Y = S Omega
-      PlanStep g = begin_gemm(0, 0, 0, PH_SUBSPACE);
-      for (int b = 0; b < nb; ++b) add_prob(g, (int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r));
-      R.push_back(g);
-    }
-    cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
-    for (int it = 0; it < q; ++it) {
-      {  // Z = S^T P'
-        PlanStep g = begin_gemm(1, 0, 0, PH_SUBSPACE);
-        for (int b = 0; b < nb; ++b) add_prob(g, (int)n, r, (int)m, signal(b), plain(Pn + (long long)b * m * r, r), nullptr, store_epi(Za + (long long)b * n * r, r));
-        R.push_back(g);
-      }
-      cholqr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n, r, nb, gram, lw, rinv);
-      {  // Y = S Z
-        PlanStep g = begin_gemm(0, 0, 0, PH_SUBSPACE);
-        for (int b = 0; b < nb; ++b) add_prob(g, (int)m, r, (int)n, signal(b), plain(Zq + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r));
-        R.push_back(g);
+      {  // Y = S Omega
+        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
+        for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
       }
       cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
-    }
-    {  // Rot = P'^T P
-      PlanStep g = begin_gemm(1, 0, 0, PH_ROTATE);
-      for (int b = 0; b < nb; ++b) add_prob(g, r, r, (int)m, plain(Pn + (long long)b * m * r, r), plain(md.P ? md.P + b * md.p_stride : nullptr, r), nullptr, store_epi(rot + (long long)b * r * r, r));
-      R.push_back(g);
-    }
-    {  // u', v' (into the transient g^ / U~ areas), then back
-      PlanStep g = begin_gemm(0, 1, 1, PH_ROTATE);
-      for (int k = 0; k < K; ++k) {
-        const long long so = (long long)k * r * n;
-        Operand A = plain(rot + (long long)(local ? k : 0) * r * r, r);
-        Operand B = plain(md.u ? md.u + so : nullptr, n); B.kind = OP_UHAT;
-        Operand B2 = plain(md.u ? md.u + so : nullptr, n); B2.kind = OP_VRES; B2.p1 = md.v ? md.v + so : nullptr;
-        Epilogue e;
-        std::memset(&e, 0, sizeof(e));
-        e.kind = EPI_ROTATE; e.u_out = md.ghat + so; e.v_out = md.util + so;
-        add_prob(g, r, (int)n, r, A, B, &B2, e);
+      for (int it = 0; it < q; ++it) {
+        {  // Z = S^T P'
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, r, (int)m, signal(b), plain(Pn + (long long)b * m * r, r), nullptr, store_epi(Za + (long long)b * n * r, r)));
+        }
+        cholqr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n, r, nb, gram, lw, rinv);
+        {  // Y = S Z
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Zq + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
+        }
+        cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
       }
-      R.push_back(g);
-      PlanStep cu, cv2;
-      cu.type = ST_COPY; cu.phase = PH_ROTATE; cu.dst = md.u; cu.src = md.ghat; cu.bytes = (size_t)K * r * n * sizeof(float);
-      cv2.type = ST_COPY; cv2.phase = PH_ROTATE; cv2.dst = md.v; cv2.src = md.util; cv2.bytes = (size_t)K * r * n * sizeof(float);
-      R.push_back(cu);
-      R.push_back(cv2);
+      {  // Rot = P'^T P
+        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_ROTATE, 1, 0, 0);
+        for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob(r, r, (int)m, plain(Pn + (long long)b * m * r, r), plain(md.P ? md.P + b * md.p_stride : nullptr, r), nullptr, store_epi(rot + (long long)b * r * r, r)));
+      }
+      {  // u', v' (into the transient g^ / U~ areas), then back
+        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_ROTATE, 0, 1, 1);
+        for (int k = 0; k < K; ++k) {
+          const long long so = (long long)k * r * n;
+          Operand A = plain(rot + (long long)(local ? k : 0) * r * r, r);
+          Operand B = plain(md.u ? md.u + so : nullptr, n); B.kind = OP_UHAT;
+          Operand B2 = plain(md.u ? md.u + so : nullptr, n); B2.kind = OP_VRES; B2.p1 = md.v ? md.v + so : nullptr;
+          Epilogue e;
+          std::memset(&e, 0, sizeof(e));
+          e.kind = EPI_ROTATE; e.u_out = md.ghat + so; e.v_out = md.util + so;
+          g.g.push_back(gemm_prob(r, (int)n, r, A, B, &B2, e));
+        }
+        add_copy(R, PH_ROTATE, md.u, md.ghat, (size_t)K * r * n * sizeof(float));
+        add_copy(R, PH_ROTATE, md.v, md.util, (size_t)K * r * n * sizeof(float));
+      }
+      add_copy(R, PH_COMMIT, md.P, Pn, (size_t)nb * m * r * sizeof(float));
+      if (!local) {  // P_0 = orthonormalised random m x r matrix
+        RandProblem rp;
+        rp.out = Ya; rp.count = m * r; rp.blk_start = 0; rp.purpose = 1; rp.mat = i; rp.replica = 0; rp.pad = 0;
+        I.next(ST_RANDOM, PH_SUBSPACE, 0, 0, 0, 1).rn.push_back(rp);
+        cholqr2(I, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, md.P, m * r, m, r, 1, gram, lw, rinv);
+      }
     }
-    {
-      PlanStep cp;
-      cp.type = ST_COPY; cp.phase = PH_COMMIT; cp.dst = md.P; cp.src = Pn; cp.bytes = (size_t)nb * m * r * sizeof(float);
-      R.push_back(cp);
-    }
-    if (!local) {  // P_0 = orthonormalised random m x r matrix
-      std::vector<PlanStep>& I = c->init_steps;
-      PlanStep f;
-      f.type = ST_RANDOM; f.out = Ya; f.count = m * r; f.purpose = 1; f.mat = i; f.per_replica = 0; f.batch = 1;
-      I.push_back(f);
-      cholqr2(I, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, md.P, m * r, m, r, 1, gram, lw, rinv);
-    }
+    flatten(R, c->refresh_steps);
+    flatten(I, c->init_steps);
   }
   c->d_probs = cv.take<GemmProblem>(P.size());
+  c->d_chols = cv.take<CholProblem>(c->h_chols.size() + 1);
+  c->d_rands = cv.take<RandProblem>(c->h_rands.size() + 1);
+  c->d_copies = cv.take<CopyProblem>(c->h_copies.size() + 1);
 
   c->last_G.assign(n_mats, nullptr);
   return (cv.off + 255) & ~size_t(255);
@@ -503,27 +556,25 @@ GemmScalars base_scalars(const lordo_ctx* c) {
 }
 
 int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t st) {
+  if (s.count == 0) return LORDO_OK;
   switch (s.type) {
     case ST_GEMM:
       sc.a_square = s.a_square;
-      launch_gemm(c->d_probs + s.prob_first, s.nprobs, s.tiles, s.atrans, s.dual, sc, st);
+      launch_gemm(c->d_probs + s.first, s.count, s.tiles, s.atrans, s.dual, sc, st);
       c->launches += 1;
       return check_launch(c, "gemm");
     case ST_CHOL:
-      launch_chol_inverse(s.gram, s.lwork, s.rinv, s.r, s.batch, s.stride, c->d_status, st);
+      launch_chol_inverse(c->d_chols + s.first, s.count, s.r_max, c->d_status, st);
       c->launches += 1;
       return check_launch(c, "chol_inverse");
-    case ST_RANDOM: {
-      RandomKeys keys;
-      const long long index = s.purpose == 1 ? 0 : c->refreshes;
-      for (int b = 0; b < s.batch; ++b) keys.key[b] = stream_key(c->cfg.seed, s.purpose, s.mat, index, s.per_replica ? b : 0);
-      launch_fill_random(s.out, s.count, s.count, keys, s.batch, st);
+    case ST_RANDOM:
+      launch_fill_random_grouped(c->d_rands + s.first, s.count, s.tiles, c->cfg.seed, s.p0 ? 0 : c->refreshes, st);
       c->launches += 1;
       return check_launch(c, "fill_random");
-    }
     case ST_COPY:
-      CUDA_OK(c, cudaMemcpyAsync(s.dst, s.src, s.bytes, cudaMemcpyDeviceToDevice, st));
-      return LORDO_OK;
+      launch_copy_grouped(c->d_copies + s.first, s.count, s.tiles, st);
+      c->launches += 1;
+      return check_launch(c, "copy");
   }
   return LORDO_OK;
 }
@@ -629,6 +680,9 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   INIT_CUDA(cudaMemcpyAsync(c->d_wblk_start, wb.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->d_sblk_start, sb.data(), 8 * (nm + 1), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemcpyAsync(c->d_probs, c->h_probs.data(), sizeof(GemmProblem) * c->h_probs.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_chols.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_chols, c->h_chols.data(), sizeof(CholProblem) * c->h_chols.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_rands.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_rands, c->h_rands.data(), sizeof(RandProblem) * c->h_rands.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_copies.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_copies, c->h_copies.data(), sizeof(CopyProblem) * c->h_copies.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
   if (c->tc) {
     INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));

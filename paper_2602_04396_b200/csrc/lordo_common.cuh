@@ -106,7 +106,7 @@ __host__ __device__ __forceinline__ unsigned long long mix64(unsigned long long 
 }
 constexpr unsigned long long kGolden = 0x9E3779B97F4A7C15ull;
 
-inline unsigned long long stream_key(unsigned long long seed, int purpose, int mat, long long index, int replica) {
+__host__ __device__ inline unsigned long long stream_key(unsigned long long seed, int purpose, int mat, long long index, int replica) {
   unsigned long long k = mix64(seed + kGolden);
   const unsigned long long f[4] = {(unsigned long long)purpose, (unsigned long long)mat, (unsigned long long)index,
                                    (unsigned long long)replica};

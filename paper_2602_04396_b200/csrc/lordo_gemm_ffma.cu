@@ -224,15 +224,15 @@ void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, in
 // Cholesky of the Gram matrix + inverse of the triangular factor, one block per problem.
 // Left-looking column Cholesky, fp64 accumulation, L kept in global memory (L2-resident).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(512) chol_inverse_kernel(const float* __restrict__ gram, float* __restrict__ lwork,
-                                                           float* __restrict__ rinv, int r, long long stride,
-                                                           unsigned* __restrict__ status) {
+__global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __restrict__ probs, unsigned* __restrict__ status) {
   extern __shared__ float row_j[];  // r floats: row j of L (columns < j)
   __shared__ float pivot_s;
   __shared__ float maxdiag_s;
-  const float* A = gram + (long long)blockIdx.x * stride;
-  float* L = lwork + (long long)blockIdx.x * stride;
-  float* X = rinv + (long long)blockIdx.x * stride;
+  const CholProblem pb = probs[blockIdx.x];
+  const int r = pb.r;
+  const float* A = pb.gram;
+  float* L = pb.lwork;
+  float* X = pb.rinv;
   const int t = threadIdx.x, nt = blockDim.x;
 
   if (t == 0) {
@@ -298,9 +298,8 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const float* __restri
   }
 }
 
-void launch_chol_inverse(const float* gram, float* lwork, float* rinv, int r, int batch, long long stride, unsigned* status,
-                         cudaStream_t st) {
-  chol_inverse_kernel<<<batch, 512, r * sizeof(float), st>>>(gram, lwork, rinv, r, stride, status);
+void launch_chol_inverse(const CholProblem* probs, int nprobs, int r_max, unsigned* status, cudaStream_t st) {
+  chol_inverse_kernel<<<nprobs, 512, r_max * sizeof(float), st>>>(probs, status);
 }
 
 }  // namespace lordo

@@ -107,8 +107,29 @@ void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips,
 // Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
 // gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the
 // diagonal. lwork: r*r floats per problem. Strides in floats between batch entries.
-void launch_chol_inverse(const float* gram, float* lwork, float* rinv, int r, int batch, long long stride, unsigned* status,
-                         cudaStream_t st);
+struct CholProblem {
+  const float* gram;
+  float* lwork;
+  float* rinv;
+  int r, pad;
+};
+void launch_chol_inverse(const CholProblem* probs, int nprobs, int r_max, unsigned* status, cudaStream_t st);
+
+// Grouped helpers of the refresh: random sketches and device-to-device copies for many matrices
+// in one launch each. blk_start is the first 256-thread block of the entry within the launch.
+struct RandProblem {
+  float* out;
+  long long count, blk_start;
+  int purpose, mat, replica, pad;
+};
+struct CopyProblem {
+  void* dst;
+  const void* src;
+  long long chunks, blk_start;  // 16-byte chunks
+};
+void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long total_blocks, unsigned long long seed, long long index,
+                                cudaStream_t st);
+void launch_copy_grouped(const CopyProblem* probs, int nprobs, long long total_blocks, cudaStream_t st);
 
 // streaming kernels
 void launch_sumsq_partial(const MatDev* mats, const void* const* G, const long long* chunk_start, int n_mats, int K, int g_dt,

@@ -248,9 +248,54 @@ __global__ void __launch_bounds__(256) fill_random_kernel(float* __restrict__ ou
   out[(long long)blockIdx.y * batch_stride + c] = (float)(__popcll(w) - 32);
 }
 
+// The same generator for many matrices in one launch; the key of each is derived on the device.
+__global__ void __launch_bounds__(256) fill_random_grouped_kernel(const RandProblem* __restrict__ probs, int nprobs,
+                                                                  unsigned long long seed, long long index) {
+  const long long blk = blockIdx.x;
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].blk_start <= blk) lo = mid; else hi = mid - 1;
+  }
+  const RandProblem pb = probs[lo];
+  const long long c = (blk - pb.blk_start) * 256 + threadIdx.x;
+  if (c >= pb.count) return;
+  const unsigned long long key = stream_key(seed, pb.purpose, pb.mat, index, pb.replica);
+  const unsigned long long w = mix64(key + kGolden * (unsigned long long)(c + 1));
+  pb.out[c] = (float)(__popcll(w) - 32);
+}
+
+// Device-to-device copies of many buffers in one launch (16-byte chunks).
+__global__ void __launch_bounds__(256) copy_grouped_kernel(const CopyProblem* __restrict__ probs, int nprobs) {
+  const long long blk = blockIdx.x;
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].blk_start <= blk) lo = mid; else hi = mid - 1;
+  }
+  const CopyProblem pb = probs[lo];
+  const long long c = ((blk - pb.blk_start) * 256 + threadIdx.x) * 4;
+  const uint4* __restrict__ src = reinterpret_cast<const uint4*>(pb.src);
+  uint4* __restrict__ dst = reinterpret_cast<uint4*>(pb.dst);
+  uint4 v[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (c + i < pb.chunks) v[i] = src[c + i];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (c + i < pb.chunks) dst[c + i] = v[i];
+}
+
 // ---------------------------------------------------------------------------------------------
 // host launchers
 // ---------------------------------------------------------------------------------------------
+void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long total_blocks, unsigned long long seed, long long index,
+                                cudaStream_t st) {
+  fill_random_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs, seed, index);
+}
+void launch_copy_grouped(const CopyProblem* probs, int nprobs, long long total_blocks, cudaStream_t st) {
+  copy_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs);
+}
 void launch_sumsq_partial(const MatDev* mats, const void* const* G, const long long* chunk_start, int n_mats, int K, int g_dt,
                           double* partial, long long total_chunks, cudaStream_t st) {
   sumsq_partial_kernel<<<(unsigned)total_chunks, 256, 0, st>>>(mats, G, chunk_start, n_mats, K, g_dt, partial);
