@@ -157,13 +157,13 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 def oracle_sample(wl, variant_name: str):
     """Returns (sample workload, description). One matrix of the most common shape class with all
-    K replicas, a round of 2 inner steps + outer step + refresh."""
+    K replicas, a round of up to 6 inner steps + outer step + refresh."""
     from paper_2602_04396_b200 import synth
     shapes = {}
     for mat in wl.mats:
         shapes[mat] = shapes.get(mat, 0) + 1
     mat = max(shapes, key=lambda s: (shapes[s], -s[0] * s[1]))
-    H = min(wl.H, 2)
+    H = min(wl.H, 6)
     sample = synth.scaled(wl, mats=[mat], H=H, rounds=1)
     desc = (f"1 matrix {mat[0]}x{mat[1]} r{mat[2]} of {len(wl.mats)}, all K={wl.K} replicas, one round of "
             f"{H} inner steps + outer step + refresh, {variant_name} rule")
