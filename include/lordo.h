@@ -201,6 +201,35 @@ LORDO_API int lordo_destroy(lordo_ctx* ctx);
 LORDO_API int lordo_fill_random(uint64_t seed, int32_t purpose, int32_t mat, int64_t index, int32_t replica, int64_t rows,
                       int64_t cols, float* out_dev, void* stream);
 
+/*
+ * (The paper has no counterpart for this entry point; it is a convenience of this library.)
+ *
+ * Clip coefficient c = min(1, rho / (||G||_2 + 1e-6)) of ONE gradient array, computed without any
+ * device allocation: no context, no workspace. It is meant for callers that must not or cannot
+ * allocate device memory at the point where they need the coefficient -- code running while a
+ * memory pool is frozen or nearly exhausted, a plug-in that was handed fixed buffers by its host
+ * framework, a monitoring hook that may not disturb the allocator of the job it watches.
+ * The reduction's partial sums live in a fixed array inside the library image (128 KiB per GPU
+ * that loads the library, held until the process exits), which bounds the input:
+ * count <= lordo_clip_coefficient_static_max_count() (2^29 elements); larger inputs are rejected
+ * with LORDO_ERR_UNSUPPORTED and nothing is launched.
+ *
+ *   G_dev         device pointer, `count` elements of g_dtype (lordo_dtype), 16-byte aligned,
+ *                 count a multiple of 8; read only
+ *   rho           clipping radius; <= 0 gives c = 1
+ *   coef_out_dev  device pointer to one float, written by the call (caller-owned)
+ *
+ * The call enqueues two kernels on `stream` and returns without synchronising. The first call on
+ * each device looks up the device address of the static array (with that device current); make
+ * that first call outside any stream capture. All calls on a device share the array: it holds
+ * whatever the previous call left (every slot a call reads it has written itself, so nothing needs
+ * clearing), and two calls whose kernels overlap on the GPU -- different streams, no ordering
+ * between them -- race on it. Calls on one stream are safe.
+ */
+LORDO_API int lordo_clip_coefficient_static(const void* G_dev, int g_dtype, int64_t count, float rho, float* coef_out_dev,
+                                            void* stream);
+LORDO_API int64_t lordo_clip_coefficient_static_max_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,8 @@ EXPORTS = [
     "lordo_query_workspace", "lordo_init", "lordo_inner_step", "lordo_inner_step_host", "lordo_outer_step",
     "lordo_refresh_subspace", "lordo_poll_status", "lordo_get_counters", "lordo_set_counters",
     "lordo_clip_coefficients", "lordo_launch_count", "lordo_last_error", "lordo_status_string", "lordo_destroy",
-    "lordo_fill_random", "lordo_profile_enable", "lordo_profile_read",
+    "lordo_fill_random", "lordo_profile_enable", "lordo_profile_read", "lordo_clip_coefficient_static",
+    "lordo_clip_coefficient_static_max_count",
 ]
 
 
@@ -85,6 +86,9 @@ def load_library() -> C.CDLL:
     lib.lordo_fill_random.argtypes = [C.c_uint64, i32, i32, i64, i32, i64, i64, vp, vp]
     lib.lordo_profile_enable.argtypes = [vp, i32]
     lib.lordo_profile_read.argtypes = [vp, vp, C.POINTER(f32)]
+    lib.lordo_clip_coefficient_static.argtypes = [vp, i32, i64, f32, vp, vp]
+    lib.lordo_clip_coefficient_static_max_count.argtypes = []
+    lib.lordo_clip_coefficient_static_max_count.restype = i64
     for name in EXPORTS:
         if getattr(lib, name).restype is C.c_int:
             getattr(lib, name).restype = C.c_int
@@ -142,6 +146,20 @@ def fill_random(seed: int, purpose: int, mat: int, index: int, replica: int, row
     if rc != 0:
         raise LordoError(rc, "lordo_fill_random", lib.lordo_status_string(rc).decode())
     return out
+
+
+def clip_coefficient_static(G: torch.Tensor, rho: float, out: torch.Tensor, stream=None) -> None:
+    """Clip coefficient of one gradient tensor through lordo_clip_coefficient_static, the entry
+    point that allocates no device memory. `out` is a one-element float32 CUDA tensor that the
+    caller provides; nothing is allocated here either."""
+    lib = load_library()
+    assert G.is_cuda and G.is_contiguous() and out.is_cuda and out.dtype == torch.float32 and out.numel() == 1
+    rc = lib.lordo_clip_coefficient_static(C.c_void_p(G.data_ptr()), _dtype_code(G.dtype), G.numel(), rho,
+                                           C.c_void_p(out.data_ptr()), _stream_handle(stream))
+    if rc != 0:
+        limit = lib.lordo_clip_coefficient_static_max_count()
+        raise LordoError(rc, "lordo_clip_coefficient_static",
+                         f"{lib.lordo_status_string(rc).decode()}; at most {limit} elements, a multiple of 8")
 
 
 class Lordo:
