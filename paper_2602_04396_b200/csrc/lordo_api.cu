@@ -5,6 +5,8 @@
 #include <string>
 #include <vector>
 
+#include <cuda.h>
+
 #include "lordo_kernels.h"
 
 using namespace lordo;
@@ -95,6 +97,12 @@ struct lordo_ctx {
   size_t tc_bf16_bytes = 0;
   long long tc_strips = 0, prep_blocks = 0;
   int tc_rn_max = 0, tc_rk_max = 0;
+  // TMA-fed kernels (bf16 storage): tensor maps per matrix, gradient maps re-encoded per pointer change
+  bool tma = false;
+  int sm_count = 0;
+  TmaMatMaps* d_maps = nullptr;
+  TmaGradMaps* d_gmaps = nullptr;
+  TmaGradMaps* h_gmaps = nullptr;  // pinned
   std::vector<TcProblem> h_tc;
   std::vector<TcPrep> h_prep;
   std::vector<long long> h_prep_start;
@@ -126,6 +134,41 @@ struct lordo_ctx {
 };
 
 namespace {
+
+typedef CUresult (*tmap_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+tmap_encode_fn tmap_encoder() {
+  static tmap_encode_fn fn = []() -> tmap_encode_fn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return reinterpret_cast<tmap_encode_fn>(p);
+  }();
+  return fn;
+}
+
+// bf16 tensor [d2][d1][d0] (d0 contiguous), box b0 x b1 x 1, written into 128 bytes at `out`.
+bool encode_map3(unsigned char* out, const void* base, long long d0, long long d1, long long d2, int b0, int b1, bool swizzle) {
+  tmap_encode_fn fn = tmap_encoder();
+  if (!fn) return false;
+  alignas(64) CUtensorMap tm;
+  const cuuint64_t dims[3] = {(cuuint64_t)d0, (cuuint64_t)d1, (cuuint64_t)d2};
+  const cuuint64_t strides[2] = {(cuuint64_t)d0 * 2, (cuuint64_t)d0 * (cuuint64_t)d1 * 2};
+  const cuuint32_t box[3] = {(cuuint32_t)b0, (cuuint32_t)b1, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  std::memcpy(out, &tm, 128);
+  return true;
+}
 
 int fail(lordo_ctx* c, int code, const std::string& msg) {
   if (c) c->err = msg;
@@ -286,6 +329,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         }
         tp.G_ind = c->d_Gtab + i; tp.G_off = wo;
         tp.cptr = c->d_coef + (size_t)i * K + k;
+        tp.mat = i; tp.replica = k; tp.pcopy = pk;
         c->h_tc.push_back(tp);
         c->tc_strips += (md.n + 127) / 128;
       }
@@ -296,6 +340,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     c->d_tc_probs = cv.take<TcProblem>(c->h_tc.size());
     c->d_tc_prep = cv.take<TcPrep>(c->h_prep.size());
     c->d_prep_start = cv.take<long long>(c->h_prep_start.size());
+    c->tma = cfg.w_dtype == LORDO_BF16;
+    c->d_maps = cv.take<TmaMatMaps>(n_mats);
+    c->d_gmaps = cv.take<TmaGradMaps>(n_mats);
   }
 
   // ---------------- launch plans ----------------
@@ -592,6 +639,15 @@ int set_gradients(lordo_ctx* c, const void* const* G, cudaStream_t st) {
   CUDA_OK(c, cudaStreamSynchronize(st));
   for (int i = 0; i < c->n_mats; ++i) { c->h_Gtab[i] = G[i]; c->last_G[i] = G[i]; }
   CUDA_OK(c, cudaMemcpyAsync(c->d_Gtab, c->h_Gtab, sizeof(void*) * c->n_mats, cudaMemcpyHostToDevice, st));
+  if (c->tma) {
+    for (int i = 0; i < c->n_mats; ++i) {
+      const lordo_mat& a = c->mats[i];
+      if (!encode_map3(c->h_gmaps[i].g_sw, G[i], a.n, a.m, c->K, 64, 64, true) ||
+          !encode_map3(c->h_gmaps[i].g_ns, G[i], a.n, a.m, c->K, 64, 64, false))
+        return fail(c, LORDO_ERR_CUDA, "tensor map encoding failed for a gradient");
+    }
+    CUDA_OK(c, cudaMemcpyAsync(c->d_gmaps, c->h_gmaps, sizeof(TmaGradMaps) * c->n_mats, cudaMemcpyHostToDevice, st));
+  }
   return LORDO_OK;
 }
 
@@ -690,6 +746,35 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
     INIT_CUDA(cudaMemcpyAsync(c->d_tc_probs, c->h_tc.data(), sizeof(TcProblem) * c->h_tc.size(), cudaMemcpyHostToDevice, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_tc_prep, c->h_prep.data(), sizeof(TcPrep) * c->h_prep.size(), cudaMemcpyHostToDevice, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_prep_start, c->h_prep_start.data(), 8 * c->h_prep_start.size(), cudaMemcpyHostToDevice, st));
+    if (c->tma) {
+      int dev = 0;
+      INIT_CUDA(cudaGetDevice(&dev));
+      INIT_CUDA(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+      std::vector<TmaMatMaps> hm(nm);
+      bool good = tmap_encoder() != nullptr;
+      const bool loc = c->cfg.variant == LORDO_LOCAL;
+      for (int i = 0; i < nm && good; ++i) {
+        const MatDev& md = c->h_mats[i];
+        const TcProblem& tp = c->h_tc[(size_t)i * c->K];  // worker 0 of matrix i: base pointers of the copies
+        const int copies = loc ? c->K : 1;
+        std::memset(&hm[i], 0, sizeof(TmaMatMaps));
+        if (md.E) {
+          good = good && encode_map3(hm[i].e_sw, md.E, md.n, md.m, c->K, 64, 64, true);
+          good = good && encode_map3(hm[i].e_ns, md.E, md.n, md.m, c->K, 64, 64, false);
+        }
+        good = good && encode_map3(hm[i].w_ns, md.W, md.n, md.m, c->K, 64, 64, false);
+        good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n, true);
+        good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
+      }
+      if (good) {
+        INIT_CUDA(cudaMemcpyAsync(c->d_maps, hm.data(), sizeof(TmaMatMaps) * nm, cudaMemcpyHostToDevice, st));
+        INIT_CUDA(cudaStreamSynchronize(st));
+        INIT_CUDA(tma_configure());
+        if (cudaHostAlloc((void**)&c->h_gmaps, sizeof(TmaGradMaps) * nm, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
+      } else {
+        c->tma = false;  // no tensor-map encoder in this driver: the register-staged kernels run instead
+      }
+    }
   }
   INIT_CUDA(cudaMemsetAsync(c->d_Gtab, 0, sizeof(void*) * nm, st));
   INIT_CUDA(cudaStreamSynchronize(st));  // the host vectors above may now be reused
@@ -753,6 +838,16 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
 
   if (c->tc) {
     ss.lr = lr;
+    if (c->tma) {
+      {
+        ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
+        launch_project_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, c->d_status, st);
+      }
+      {
+        ProfScope ps(c, st, PC_APPLY);
+        launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, c->d_status, st);
+      }
+    } else {
     {
       ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
       launch_project_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rn_max, ss, c->cfg.w_dtype == LORDO_BF16,
@@ -762,6 +857,7 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
       ProfScope ps(c, st, PC_APPLY);
       launch_apply_tc(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->tc_rk_max, ss, c->cfg.w_dtype == LORDO_BF16,
                       c->d_status, st);
+    }
     }
     c->launches += 2;
     rc = check_launch(c, "tensor-core inner step");
@@ -937,6 +1033,7 @@ int lordo_destroy(lordo_ctx* c) {
   if (!c) return LORDO_ERR_INVALID_ARG;
   if (c->h_Gtab) cudaFreeHost(c->h_Gtab);
   if (c->h_status) cudaFreeHost(c->h_status);
+  if (c->h_gmaps) cudaFreeHost(c->h_gmaps);
   for (const lordo_ctx::Span& sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;

@@ -86,6 +86,17 @@ struct TcProblem {
   const void* const* G_ind;    // entry of the per-call gradient pointer table
   long long G_off;             // element offset of this worker inside it
   const float* cptr;           // clip coefficient
+  int mat, replica, pcopy, pad;  // matrix index, worker index, which copy of P (0 for Global)
+};
+
+// Tensor maps (opaque 128-byte objects encoded on the host) of one matrix for the TMA-fed kernels.
+// "sw": 64 x 64 boxes with the 128-byte swizzle (operands of the projection); "ns": 64 x 64 boxes
+// without swizzle (tiles the update epilogue reads and writes in place).
+struct alignas(128) TmaMatMaps {
+  unsigned char e_sw[128], pt[128], p16[128], e_ns[128], w_ns[128];
+};
+struct alignas(128) TmaGradMaps {  // re-encoded whenever the caller's gradient pointer changes
+  unsigned char g_sw[128], g_ns[128];
 };
 
 struct TcPrep {
@@ -103,6 +114,13 @@ void launch_project_tc(const TcProblem* probs, int nprobs, long long total_strip
                        unsigned* status, cudaStream_t st);
 void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips, int r_k_max, const StepScalars& sc, int bf16,
                      unsigned* status, cudaStream_t st);
+
+// TMA-fed persistent kernels for bf16 storage (lordo_tma.cu).
+cudaError_t tma_configure();
+void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
+                        const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
+void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
+                      const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
 
 // Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
 // gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the

@@ -1,0 +1,462 @@
+// TMA-fed, persistent tensor-core kernels of the inner step for bf16 storage of G, E and W.
+//
+//   project_tma_kernel  The streamed operand never passes through registers as single elements:
+//                       TMA brings 64-row tiles of G, E (and of P^T) into 128B-swizzled shared
+//                       memory, four warps turn the G tile into c*G + E in place (16-byte vector
+//                       operations, layout-agnostic), and the tile is consumed as an MN-major
+//                       operand by tcgen05.mma. Two accumulator buffers in tensor memory let the
+//                       moment-update epilogue of one strip run under the main loop of the next.
+//   apply_tma_kernel    The strip's two low-rank operands (g^T, U~^T) live in tensor memory as the
+//                       A operands; rows of P and the tiles of G, E, W arrive by TMA; the epilogue
+//                       works on the tiles in shared memory (one column per thread) and the
+//                       updated E and W tiles leave by TMA stores.
+//
+// One CTA per SM; a CTA walks the list of 128-column strips with stride gridDim.x. Every role walks
+// the same list, so stage and phase counters stay in step without further communication.
+#include "lordo_kernels.h"
+#include "lordo_umma.cuh"
+
+namespace lordo {
+
+using namespace umma;
+
+namespace {
+
+constexpr int kStrip = 128;
+
+__device__ __forceinline__ int find_problem(const TcProblem* __restrict__ probs, int nprobs, long long strip) {
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].strip_start <= strip) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
+__device__ __forceinline__ float bf16_to_f(unsigned short x) { return __uint_as_float(((uint32_t)x) << 16); }
+__device__ __forceinline__ unsigned short f_to_bf16(float v) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  return *reinterpret_cast<const unsigned short*>(&h);
+}
+
+// ---- projection ---------------------------------------------------------------------------------
+constexpr int kPStages = 3;
+constexpr uint32_t kPStageBytes = 65536;  // G 16 KB | E 16 KB | P^T tile up to 32 KB
+constexpr int kPXformWarps = 4, kPEpiWarps = 8;
+constexpr int kPThreads = (2 + kPXformWarps + kPEpiWarps) * 32;  // 448
+
+// ---- update -------------------------------------------------------------------------------------
+constexpr int kARows = 64;                // rows of W per step = MMA N
+constexpr int kAInStages = 3;             // G | E | W tiles, 16 KB each
+constexpr uint32_t kAInStageBytes = 49152;
+constexpr int kAPStages = 2;              // rows of P, up to 32 KB
+constexpr uint32_t kAPStageBytes = 32768;
+constexpr int kAEpiWarps = 16;
+constexpr int kAThreads = (2 + kAEpiWarps) * 32;  // 576
+
+}  // namespace
+
+// =================================================================================================
+__global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
+                                                                   const TmaMatMaps* __restrict__ maps,
+                                                                   const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
+                                                                   unsigned* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t full_bar[kPStages], xform_bar[kPStages], empty_bar[kPStages], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_slot;
+  __shared__ float dsum_s[kStrip];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool ef = sc.ef != 0;
+
+  if (tid == 0) {
+    for (int s = 0; s < kPStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], kPXformWarps * 32); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kPEpiWarps * 32); }
+    mbar_init_fence();
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ------------------------------------------------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+        const int n0 = (int)(strip - pr->strip_start) * kStrip;
+        const TmaMatMaps* mm = maps + pr->mat;
+        const TmaGradMaps* gm = gmaps + pr->mat;
+        const int nkb = pr->m_k / 64, rep = pr->replica, pc = pr->pcopy;
+        const uint32_t tx = 16384u + (ef ? 16384u : 0u) + (uint32_t)pr->r_n * 128u;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kPStages;
+          ok = mbar_wait(&empty_bar[s], ((it / kPStages) & 1u) ^ 1u, status);
+          if (!ok) break;
+          unsigned char* base = smem + s * kPStageBytes;
+          mbar_expect_tx(&full_bar[s], tx);
+          tma_load_3d(base, gm->g_sw, n0, kb * 64, rep, &full_bar[s]);
+          tma_load_3d(base + 8192, gm->g_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
+          if (ef) {
+            tma_load_3d(base + 16384, mm->e_sw, n0, kb * 64, rep, &full_bar[s]);
+            tma_load_3d(base + 24576, mm->e_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
+          }
+          tma_load_3d(base + 32768, mm->pt, kb * 64, 0, pc, &full_bar[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issue ---------------------------------------------------------------
+    if (lane == 0) {
+      uint32_t it = 0, si = 0;
+      bool ok = true;
+      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+        const int nkb = pr->m_k / 64;
+        const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)pr->r_n) | kIdescAMajorMN;
+        const uint32_t buf = si & 1u;
+        ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
+        if (!ok) break;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kPStages;
+          ok = mbar_wait(&xform_bar[s], (it / kPStages) & 1u, status);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t sA = smem_u32(smem + s * kPStageBytes), sB = sA + 32768;
+#pragma unroll
+          for (int k16 = 0; k16 < 4; ++k16)
+            mma_bf16(tmem + buf * 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          mma_commit(&empty_bar[s]);
+        }
+        if (ok) mma_commit(&acc_full[buf]);
+      }
+    }
+  } else if (warp < 2 + kPXformWarps) {
+    // ---------------- transform: G tile <- c*G + E, in place ------------------------------------
+    const int xt = tid - 64;
+    uint32_t it = 0;
+    bool ok = true;
+    for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+      const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+      const int nkb = pr->m_k / 64;
+      const float c = *pr->cptr;
+      for (int kb = 0; kb < nkb; ++kb, ++it) {
+        const int s = it % kPStages;
+        ok = mbar_wait(&full_bar[s], (it / kPStages) & 1u, status);
+        if (!ok) break;
+        uint4* G = reinterpret_cast<uint4*>(smem + s * kPStageBytes);
+        const uint4* E = G + 1024;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int idx = xt + i * 128;
+          const uint4 g = G[idx];
+          uint4 e = make_uint4(0u, 0u, 0u, 0u);
+          if (ef) e = E[idx];
+          uint4 a;
+          a.x = pack2_bf16(fmaf(c, bf_lo(g.x), bf_lo(e.x)), fmaf(c, bf_hi(g.x), bf_hi(e.x)));
+          a.y = pack2_bf16(fmaf(c, bf_lo(g.y), bf_lo(e.y)), fmaf(c, bf_hi(g.y), bf_hi(e.y)));
+          a.z = pack2_bf16(fmaf(c, bf_lo(g.z), bf_lo(e.z)), fmaf(c, bf_hi(g.z), bf_hi(e.z)));
+          a.w = pack2_bf16(fmaf(c, bf_lo(g.w), bf_lo(e.w)), fmaf(c, bf_hi(g.w), bf_hi(e.w)));
+          G[idx] = a;
+        }
+        fence_async_smem();
+        mbar_arrive(&xform_bar[s]);
+      }
+    }
+  } else {
+    // ---------------- epilogue: moments on this thread's column, out of tensor memory -----------
+    const int q = warp & 3, half = (warp - (2 + kPXformWarps)) >> 2;
+    const float b1 = sc.beta1, b2 = sc.beta2, w = sc.omega;
+    const bool low = sc.form == LORDO_QHM_LOW;
+    uint32_t si = 0;
+    bool ok = true;
+    for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+      const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+      const int n = pr->n, r = pr->r, r_n = pr->r_n, r_k = pr->r_k;
+      const long long n0 = (strip - pr->strip_start) * kStrip;
+      const long long ecol = n0 + q * 32 + lane;
+      const bool e_ok = ecol < n;
+      const long long ecolc = e_ok ? ecol : (long long)n - 1;
+      float* __restrict__ up_ = pr->u;
+      float* __restrict__ vp_ = pr->v;
+      __nv_bfloat16* __restrict__ gT = pr->gT16 + ecolc * r_k;
+      __nv_bfloat16* __restrict__ uT = pr->uT16 + ecolc * r_k;
+      const uint32_t buf = si & 1u;
+      ok = mbar_wait<64>(&acc_full[buf], (si >> 1) & 1u, status);
+      if (!ok) break;
+      tc_fence_after_sync();
+      float dsum = 0.f;
+      for (int ch = half; ch < r_n / 16; ch += 2) {
+        float u[16], v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const size_t idx = (size_t)(unsigned)min(ch * 16 + i, r - 1) * (size_t)n + (size_t)ecolc;
+          u[i] = up_[idx];
+          v[i] = vp_[idx];
+        }
+        float g[16];
+        tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + buf * 256 + (uint32_t)(ch * 16), g);
+        uint32_t gp[8], upk[8];
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+          float o[2];
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            const int row = ch * 16 + i + t;
+            const float gg = g[i + t];
+            const float un = b1 * u[i + t] + (1.f - b1) * gg;
+            const float vn = b2 * v[i + t] + (1.f - b2) * gg * gg;
+            const float uh = un * sc.inv_bc1;
+            const float D = sqrtf(vn * sc.inv_bc2) + sc.eps;
+            o[t] = low ? (w * uh + (1.f - w) * gg) / D : uh / D;
+            if (e_ok && row < r) {
+              const size_t idx = (size_t)(unsigned)row * (size_t)n + (size_t)ecol;
+              up_[idx] = un;
+              vp_[idx] = vn;
+              dsum += D;
+            } else {
+              o[t] = 0.f;
+            }
+          }
+          gp[i >> 1] = pack2_bf16(g[i], g[i + 1]);
+          upk[i >> 1] = pack2_bf16(o[0], o[1]);
+        }
+        if (e_ok) {
+          uint4* gd = reinterpret_cast<uint4*>(gT + ch * 16);
+          uint4* ud = reinterpret_cast<uint4*>(uT + ch * 16);
+          gd[0] = make_uint4(gp[0], gp[1], gp[2], gp[3]); gd[1] = make_uint4(gp[4], gp[5], gp[6], gp[7]);
+          ud[0] = make_uint4(upk[0], upk[1], upk[2], upk[3]); ud[1] = make_uint4(upk[4], upk[5], upk[6], upk[7]);
+        }
+      }
+      tc_fence_before_sync();
+      mbar_arrive(&acc_empty[buf]);
+      if (sc.form == LORDO_QHM_FULL) {  // mu(D): mean over the rank axis, one value per column
+        if (half == 1) dsum_s[q * 32 + lane] = dsum;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (half == 0 && e_ok) pr->dcol[ecol] = (dsum + dsum_s[q * 32 + lane]) / (float)r;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_free(tmem, 512);
+}
+
+// =================================================================================================
+__global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
+                                                                 const TmaMatMaps* __restrict__ maps,
+                                                                 const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
+                                                                 unsigned* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* sP = smem;                               // kAPStages x 32 KB
+  unsigned char* sIn = smem + kAPStages * kAPStageBytes;  // kAInStages x 48 KB
+  __shared__ uint64_t p_full[kAPStages], p_empty[kAPStages], in_full[kAInStages], in_free[kAInStages], acc_full[2], acc_empty[2], x_ready;
+  __shared__ uint32_t tmem_slot;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool ef = sc.ef != 0;
+
+  if (tid == 0) {
+    for (int s = 0; s < kAPStages; ++s) { mbar_init(&p_full[s], 1); mbar_init(&p_empty[s], 1); }
+    for (int s = 0; s < kAInStages; ++s) { mbar_init(&in_full[s], 1); mbar_init(&in_free[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kAEpiWarps * 32); }
+    mbar_init(&x_ready, kAEpiWarps * 32);
+    mbar_init_fence();
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+  // tensor memory: columns [0,128) g^T, [128,256) U~^T (two bf16 per column), [256,512) two buffers of two accumulators
+
+  if (warp == 0) {
+    // ---------------- TMA producer: rows of P, tiles of G, E, W --------------------------------
+    if (lane == 0) {
+      uint32_t jt = 0;
+      bool ok = true;
+      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+        const int n0 = (int)(strip - pr->strip_start) * kStrip;
+        const TmaMatMaps* mm = maps + pr->mat;
+        const TmaGradMaps* gm = gmaps + pr->mat;
+        const int nkb = pr->r_k / 64, rep = pr->replica, pc = pr->pcopy;
+        const int nsteps = (pr->m + kARows - 1) / kARows;
+        for (int t = 0; t < nsteps; ++t, ++jt) {
+          const int ps = jt % kAPStages, is = jt % kAInStages;
+          ok = mbar_wait(&p_empty[ps], ((jt / kAPStages) & 1u) ^ 1u, status);
+          if (!ok) break;
+          mbar_expect_tx(&p_full[ps], (uint32_t)nkb * 8192u);
+          for (int kb = 0; kb < nkb; ++kb) tma_load_3d(sP + ps * kAPStageBytes + kb * 8192, mm->p16, kb * 64, t * kARows, pc, &p_full[ps]);
+          ok = mbar_wait(&in_free[is], ((jt / kAInStages) & 1u) ^ 1u, status);
+          if (!ok) break;
+          unsigned char* base = sIn + is * kAInStageBytes;
+          mbar_expect_tx(&in_full[is], ef ? 49152u : 32768u);
+          tma_load_3d(base, gm->g_ns, n0, t * kARows, rep, &in_full[is]);
+          tma_load_3d(base + 8192, gm->g_ns, n0 + 64, t * kARows, rep, &in_full[is]);
+          if (ef) {
+            tma_load_3d(base + 16384, mm->e_ns, n0, t * kARows, rep, &in_full[is]);
+            tma_load_3d(base + 24576, mm->e_ns, n0 + 64, t * kARows, rep, &in_full[is]);
+          }
+          tma_load_3d(base + 32768, mm->w_ns, n0, t * kARows, rep, &in_full[is]);
+          tma_load_3d(base + 40960, mm->w_ns, n0 + 64, t * kARows, rep, &in_full[is]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issue: A operands from tensor memory ----------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_f32(128, kARows);
+      uint32_t jt = 0, si = 0;
+      bool ok = true;
+      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+        const int nkb = pr->r_k / 64;
+        const int nsteps = (pr->m + kARows - 1) / kARows;
+        ok = mbar_wait(&x_ready, si & 1u, status);
+        if (!ok) break;
+        for (int t = 0; t < nsteps; ++t, ++jt) {
+          const int ps = jt % kAPStages;
+          const uint32_t b = jt & 1u;
+          ok = mbar_wait(&p_full[ps], (jt / kAPStages) & 1u, status);
+          if (ok) ok = mbar_wait(&acc_empty[b], ((jt >> 1) & 1u) ^ 1u, status);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t pbase = smem_u32(sP + ps * kAPStageBytes);
+          const uint32_t d1 = tmem + 256 + b * 128, d2 = d1 + 64;
+          for (int kb = 0; kb < nkb; ++kb) {
+#pragma unroll
+            for (int k16 = 0; k16 < 4; ++k16) {
+              const uint32_t acc = (kb > 0 || k16 > 0) ? 1u : 0u;
+              const uint64_t bd = smem_desc_k128(pbase + kb * 8192 + k16 * 32);
+              const uint32_t acol = (uint32_t)(kb * 4 + k16) * 8;
+              mma_bf16_ts(d1, tmem + acol, bd, idesc, acc);
+              mma_bf16_ts(d2, tmem + 128 + acol, bd, idesc, acc);
+            }
+          }
+          mma_commit(&p_empty[ps]);
+          mma_commit(&acc_full[b]);
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue: one column per thread, 16 rows per step --------------------------
+    const int ew = warp - 2;
+    const int q = warp & 3, grp = ew >> 2;  // lane quarter (fixed by the hardware), row group 0..3
+    const int colq = q * 32 + lane;          // column within the strip
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    const int tile_off = (colq >> 6) * 8192 + (colq & 63) * 2;  // inside a 16 KB tile of two 64-column boxes
+    const float lr = sc.lr, om = sc.omega;
+    const bool full = sc.form == LORDO_QHM_FULL;
+    const float a2w = full ? om : 1.f;
+    uint32_t jt = 0, si = 0;
+    bool ok = true;
+    for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+      const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+      const int n = pr->n, r_k = pr->r_k;
+      const int n0 = (int)(strip - pr->strip_start) * kStrip;
+      const TmaMatMaps* mm = maps + pr->mat;
+      const int rep = pr->replica;
+      const int nsteps = (pr->m + kARows - 1) / kARows;
+      const long long col = (long long)n0 + colq;
+      const long long colc = col < n ? col : (long long)n - 1;
+      const float c = *pr->cptr;
+      const float cd = full ? (1.f - om) * c / pr->dcol[colc] : 0.f;
+      // this thread's quarter of its column's low-rank operands -> tensor memory (r_k/8 columns each)
+      {
+        const int per = r_k / 8;  // 32-bit columns of one operand handled by this row group
+        const __nv_bfloat16* __restrict__ g16 = pr->gT16 + colc * r_k + grp * (r_k / 4);
+        const __nv_bfloat16* __restrict__ u16 = pr->uT16 + colc * r_k + grp * (r_k / 4);
+        const bool live = col < n;
+        for (int c0 = 0; c0 < per; c0 += 8) {
+          uint4 glo = *reinterpret_cast<const uint4*>(g16 + c0 * 2), ghi = *reinterpret_cast<const uint4*>(g16 + c0 * 2 + 8);
+          uint4 ulo = *reinterpret_cast<const uint4*>(u16 + c0 * 2), uhi = *reinterpret_cast<const uint4*>(u16 + c0 * 2 + 8);
+          if (!live) { glo = ghi = ulo = uhi = make_uint4(0u, 0u, 0u, 0u); }
+          tmem_st8(tmem + lane_base + (uint32_t)(grp * per + c0), glo, ghi);
+          tmem_st8(tmem + lane_base + 128u + (uint32_t)(grp * per + c0), ulo, uhi);
+        }
+        tmem_st_wait();
+        tc_fence_before_sync();
+        mbar_arrive(&x_ready);
+      }
+      for (int t = 0; t < nsteps; ++t, ++jt) {
+        const int is = jt % kAInStages;
+        const uint32_t b = jt & 1u;
+        unsigned char* base = sIn + is * kAInStageBytes + tile_off + grp * 16 * 128;
+        ok = mbar_wait<32>(&in_full[is], (jt / kAInStages) & 1u, status);
+        if (ok) ok = mbar_wait<32>(&acc_full[b], (jt >> 1) & 1u, status);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
+        float g[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(base + j * 128));
+        float acc[16];
+        if (ef) {
+          tmem_ld16(taddr, acc);  // (P g)^T
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            unsigned short* ep = reinterpret_cast<unsigned short*>(base + 16384 + j * 128);
+            *ep = f_to_bf16((c * g[j] + bf16_to_f(*ep)) - acc[j]);
+          }
+        }
+        tmem_ld16(taddr + 64, acc);  // (P U~)^T
+        tc_fence_before_sync();
+        mbar_arrive(&acc_empty[b]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          unsigned short* wp = reinterpret_cast<unsigned short*>(base + 32768 + j * 128);
+          *wp = f_to_bf16(bf16_to_f(*wp) - lr * (cd * g[j] + a2w * acc[j]));
+        }
+        fence_async_smem();
+        asm volatile("bar.sync 2, 512;" ::: "memory");
+        if (ew == 0 && lane == 0) {
+          unsigned char* sb = sIn + is * kAInStageBytes;
+          if (ef) {
+            tma_store_3d(mm->e_ns, n0, t * kARows, rep, sb + 16384);
+            tma_store_3d(mm->e_ns, n0 + 64, t * kARows, rep, sb + 24576);
+          }
+          tma_store_3d(mm->w_ns, n0, t * kARows, rep, sb + 32768);
+          tma_store_3d(mm->w_ns, n0 + 64, t * kARows, rep, sb + 40960);
+          tma_store_commit();
+          tma_store_wait_read();
+          mbar_arrive(&in_free[is]);
+        }
+      }
+    }
+    if (ew == 0 && lane == 0) tma_store_wait_all();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_free(tmem, 512);
+}
+
+// =================================================================================================
+cudaError_t tma_configure() {
+  cudaError_t e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(apply_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)(kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024));
+}
+
+void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
+                        const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
+  const long long g = total_strips < grid ? total_strips : grid;
+  project_tma_kernel<<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+}
+void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
+                      const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
+  const long long g = total_strips < grid ? total_strips : grid;
+  apply_tma_kernel<<<(unsigned)g, kAThreads, kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, st>>>(probs, nprobs, total_strips,
+                                                                                                             maps, gmaps, sc, status);
+}
+
+}  // namespace lordo

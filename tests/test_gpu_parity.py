@@ -124,6 +124,22 @@ def test_fast_mode_inner_steps(shape, form, variant):
     assert st["W"] < FAST_TOL * 3 * 0.01 / 0.02, st
 
 
+@pytest.mark.parametrize("shape", [(200, 136, 24), (320, 264, 72), (200, 520, 136), (704, 256, 256), (2048, 384, 256)])
+@pytest.mark.parametrize("form,variant,ef", [(2, 0, True), (1, 1, True), (0, 0, False)])
+def test_fast_mode_inner_steps_bf16(shape, form, variant, ef):
+    """bf16 storage of W, G, E: the TMA-fed kernels. Stored bf16 values add their own 2^-9 rounding."""
+    m, n, r = shape
+    wl = _small(m=m, n=n, r=r, K=2, H=3, rounds=1, clip_rho=30.0, w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    spec = RunSpec(wl, variant=variant, form=form, error_feedback=ef, refresh=False, lr=0.01, omega=0.9, check_mode=0, eps=0.05)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert opt.poll_status() == 0
+    assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["E"] < 2 * FAST_TOL, st
+    assert _update_error(opt, orc, spec) < 0.05, _update_error(opt, orc, spec)
+    d = hz.bf16_ulp_distance(hz._np_state(opt.W[0]), orc.W[0])
+    assert (d <= 1).mean() > 0.99 and d.max() <= 8, ((d <= 1).mean(), d.max())
+
+
 def test_fast_mode_adam_eps():
     """With Adam's own eps = 1e-8 the first steps' update is sign-like, and an entry of the low-rank
     gradient that is smaller than the bf16 rounding of its terms can land on the other sign; that is
