@@ -77,19 +77,29 @@ def bytes_of(dt: str) -> int:
     return 2 if dt == "bf16" else 4
 
 
-def algorithmic_bytes(wl, variant: int, form: int, ef: bool = True) -> dict:
-    """Bytes each kernel class must move per launch if every tensor crossed HBM exactly once
-    (operands shared by the K replicas counted once)."""
+def algorithmic_bytes(wl, variant: int, form: int, ef: bool = True, fast: bool = True) -> dict:
+    """Bytes each kernel class must move per launch if every tensor it touches crossed HBM exactly
+    once (operands shared by the K replicas counted once). In fast mode the moment update is part of
+    the projection kernel (u, v read and written, bf16 transposed g^ and U~ written) and the update
+    kernel reads those two bf16 operands; in check mode g^ and U~ are fp32 and the moments have a
+    kernel of their own."""
     K = wl.K
     bw, bg, be = bytes_of(wl.w_dtype), bytes_of(wl.g_dtype), bytes_of(wl.e_dtype)
     out = dict(clip=0, project=0, moments=0, apply=0, outer_states=0, outer_weights=0)
     for m, n, r in wl.mats:
         mn, rn = m * n, r * n
         p_copies = K if variant == 1 else 1
+        dcol = K * n * 4 if form == 2 else 0
         out["clip"] += K * mn * bg
-        out["project"] += K * mn * (bg + (be if ef else 0)) + p_copies * m * r * 4 + K * rn * 4
-        out["moments"] += K * rn * 4 * 6 + (K * n * 4 if form == 2 else 0)  # read g,u,v; write u,v,U~
-        out["apply"] += K * mn * (bg + (2 * be if ef else 0) + 2 * bw) + p_copies * m * r * 4 + K * rn * 4 * 2
+        stream_in = K * mn * (bg + (be if ef else 0))
+        stream_rw = K * mn * (bg + (2 * be if ef else 0) + 2 * bw)
+        if fast:
+            out["project"] += stream_in + p_copies * m * r * 2 + K * rn * (16 + 4) + dcol
+            out["apply"] += stream_rw + p_copies * m * r * 2 + K * rn * 4 + dcol
+        else:
+            out["project"] += stream_in + p_copies * m * r * 4 + K * rn * 4
+            out["moments"] += K * rn * 4 * 6 + dcol  # read g,u,v; write u,v,U~
+            out["apply"] += stream_rw + p_copies * m * r * 4 + K * rn * 4 * 2 + dcol
         out["outer_states"] += 2 * (2 * K * rn * 4)
         out["outer_weights"] += 2 * K * mn * bw + mn * 4 * 5  # X0 r/w, B r/w, Delta w
     return out
@@ -317,7 +327,8 @@ def main():
     value = params / (ms_total * 1e-3)
 
     # ---- per-class figures and the roofline of the dominant kernel -----------------------------
-    abytes = algorithmic_bytes(wl, hp["variant"], hp["form"])
+    tc_active = (args.mode == "fast" and max(r for _, _, r in wl.mats) <= 256 and wl.w_dtype == wl.g_dtype == wl.e_dtype)
+    abytes = algorithmic_bytes(wl, hp["variant"], hp["form"], True, tc_active)
     per_launch = {"clip": n_inner, "project": n_inner, "moments": n_inner, "apply": n_inner, "outer_states": args.steps,
                   "outer_weights": args.steps, "refresh": args.steps * (H if wl.refresh_every_step else 1)}
     kernels = {}

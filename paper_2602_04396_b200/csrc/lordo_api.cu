@@ -761,8 +761,10 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         if (md.E) {
           good = good && encode_map3(hm[i].e_sw, md.E, md.n, md.m, c->K, 64, 64, true);
           good = good && encode_map3(hm[i].e_ns, md.E, md.n, md.m, c->K, 64, 64, false);
+          good = good && encode_map3(hm[i].e_st, md.E, md.n, md.m, c->K, 64, 16, false);
         }
         good = good && encode_map3(hm[i].w_ns, md.W, md.n, md.m, c->K, 64, 64, false);
+        good = good && encode_map3(hm[i].w_st, md.W, md.n, md.m, c->K, 64, 16, false);
         good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n, true);
         good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
       }

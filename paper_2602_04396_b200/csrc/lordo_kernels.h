@@ -94,6 +94,7 @@ struct TcProblem {
 // without swizzle (tiles the update epilogue reads and writes in place).
 struct alignas(128) TmaMatMaps {
   unsigned char e_sw[128], pt[128], p16[128], e_ns[128], w_ns[128];
+  unsigned char e_st[128], w_st[128];  // 64 x 16 boxes, no swizzle: stores of one row group of the update epilogue
 };
 struct alignas(128) TmaGradMaps {  // re-encoded whenever the caller's gradient pointer changes
   unsigned char g_sw[128], g_ns[128];

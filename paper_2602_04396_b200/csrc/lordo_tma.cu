@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
 
   if (tid == 0) {
     for (int s = 0; s < kAPStages; ++s) { mbar_init(&p_full[s], 1); mbar_init(&p_empty[s], 1); }
-    for (int s = 0; s < kAInStages; ++s) { mbar_init(&in_full[s], 1); mbar_init(&in_free[s], 1); }
+    for (int s = 0; s < kAInStages; ++s) { mbar_init(&in_full[s], 1); mbar_init(&in_free[s], 4); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kAEpiWarps * 32); }
     mbar_init(&x_ready, kAEpiWarps * 32);
     mbar_init_fence();
@@ -416,23 +416,25 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           unsigned short* wp = reinterpret_cast<unsigned short*>(base + 32768 + j * 128);
           *wp = f_to_bf16(bf16_to_f(*wp) - lr * (cd * g[j] + a2w * acc[j]));
         }
+        // the four warps of a row group hand their 16 rows to the TMA engine on their own
         fence_async_smem();
-        asm volatile("bar.sync 2, 512;" ::: "memory");
-        if (ew == 0 && lane == 0) {
-          unsigned char* sb = sIn + is * kAInStageBytes;
+        asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory");
+        if ((ew & 3) == 0 && lane == 0) {
+          unsigned char* sb = sIn + is * kAInStageBytes + grp * 16 * 128;
+          const int row = t * kARows + grp * 16;
           if (ef) {
-            tma_store_3d(mm->e_ns, n0, t * kARows, rep, sb + 16384);
-            tma_store_3d(mm->e_ns, n0 + 64, t * kARows, rep, sb + 24576);
+            tma_store_3d(mm->e_st, n0, row, rep, sb + 16384);
+            tma_store_3d(mm->e_st, n0 + 64, row, rep, sb + 24576);
           }
-          tma_store_3d(mm->w_ns, n0, t * kARows, rep, sb + 32768);
-          tma_store_3d(mm->w_ns, n0 + 64, t * kARows, rep, sb + 40960);
+          tma_store_3d(mm->w_st, n0, row, rep, sb + 32768);
+          tma_store_3d(mm->w_st, n0 + 64, row, rep, sb + 40960);
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(&in_free[is]);
         }
       }
     }
-    if (ew == 0 && lane == 0) tma_store_wait_all();
+    if ((ew & 3) == 0 && lane == 0) tma_store_wait_all();
   }
   tc_fence_before_sync();
   __syncthreads();
