@@ -90,11 +90,11 @@ struct TcProblem {
 };
 
 // Tensor maps (opaque 128-byte objects encoded on the host) of one matrix for the TMA-fed kernels.
-// "sw": 64 x 64 boxes with the 128-byte swizzle (operands of the projection); "ns": 64 x 64 boxes
-// without swizzle (tiles the update epilogue reads and writes in place).
+// "sw": 64 x 64 boxes with the 128-byte swizzle (operands of the projection); "ns": 128 x 64 boxes
+// without swizzle (tiles the update epilogue reads and writes in place); "st": 128 x 16 boxes.
 struct alignas(128) TmaMatMaps {
   unsigned char e_sw[128], pt[128], p16[128], e_ns[128], w_ns[128];
-  unsigned char e_st[128], w_st[128];  // 64 x 16 boxes, no swizzle: stores of one row group of the update epilogue
+  unsigned char e_st[128], w_st[128];  // stores of one row group of the update epilogue
 };
 struct alignas(128) TmaGradMaps {  // re-encoded whenever the caller's gradient pointer changes
   unsigned char g_sw[128], g_ns[128];

@@ -54,7 +54,7 @@ constexpr uint32_t kAInStageBytes = 49152;
 constexpr int kAPStages = 2;              // rows of P, up to 32 KB
 constexpr uint32_t kAPStageBytes = 32768;
 constexpr int kAEpiWarps = 16;
-constexpr int kAThreads = (2 + kAEpiWarps) * 32;  // 576
+constexpr int kAThreads = (3 + kAEpiWarps) * 32;  // 608: TMA inputs, MMA, 16 epilogue warps, TMA rows of P
 
 }  // namespace
 
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
   // tensor memory: columns [0,128) g^T, [128,256) U~^T (two bf16 per column), [256,512) two buffers of two accumulators
 
   if (warp == 0) {
-    // ---------------- TMA producer: rows of P, tiles of G, E, W --------------------------------
+    // ---------------- TMA producer: tiles of G, E, W ---------------------------------------------
     if (lane == 0) {
       uint32_t jt = 0;
       bool ok = true;
@@ -288,26 +288,36 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         const int n0 = (int)(strip - pr->strip_start) * kStrip;
         const TmaMatMaps* mm = maps + pr->mat;
         const TmaGradMaps* gm = gmaps + pr->mat;
-        const int nkb = pr->r_k / 64, rep = pr->replica, pc = pr->pcopy;
+        const int rep = pr->replica;
         const int nsteps = (pr->m + kARows - 1) / kARows;
         for (int t = 0; t < nsteps; ++t, ++jt) {
-          const int ps = jt % kAPStages, is = jt % kAInStages;
-          ok = mbar_wait(&p_empty[ps], ((jt / kAPStages) & 1u) ^ 1u, status);
-          if (!ok) break;
-          mbar_expect_tx(&p_full[ps], (uint32_t)nkb * 8192u);
-          for (int kb = 0; kb < nkb; ++kb) tma_load_3d(sP + ps * kAPStageBytes + kb * 8192, mm->p16, kb * 64, t * kARows, pc, &p_full[ps]);
+          const int is = jt % kAInStages;
           ok = mbar_wait(&in_free[is], ((jt / kAInStages) & 1u) ^ 1u, status);
           if (!ok) break;
           unsigned char* base = sIn + is * kAInStageBytes;
           mbar_expect_tx(&in_full[is], ef ? 49152u : 32768u);
           tma_load_3d(base, gm->g_ns, n0, t * kARows, rep, &in_full[is]);
-          tma_load_3d(base + 8192, gm->g_ns, n0 + 64, t * kARows, rep, &in_full[is]);
-          if (ef) {
-            tma_load_3d(base + 16384, mm->e_ns, n0, t * kARows, rep, &in_full[is]);
-            tma_load_3d(base + 24576, mm->e_ns, n0 + 64, t * kARows, rep, &in_full[is]);
-          }
+          if (ef) tma_load_3d(base + 16384, mm->e_ns, n0, t * kARows, rep, &in_full[is]);
           tma_load_3d(base + 32768, mm->w_ns, n0, t * kARows, rep, &in_full[is]);
-          tma_load_3d(base + 40960, mm->w_ns, n0 + 64, t * kARows, rep, &in_full[is]);
+        }
+      }
+    }
+  } else if (warp == 2 + kAEpiWarps) {
+    // ---------------- TMA producer: rows of P ---------------------------------------------------
+    if (lane == 0) {
+      uint32_t jt = 0;
+      bool ok = true;
+      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+        const TmaMatMaps* mm = maps + pr->mat;
+        const int nkb = pr->r_k / 64, pc = pr->pcopy;
+        const int nsteps = (pr->m + kARows - 1) / kARows;
+        for (int t = 0; t < nsteps; ++t, ++jt) {
+          const int ps = jt % kAPStages;
+          ok = mbar_wait(&p_empty[ps], ((jt / kAPStages) & 1u) ^ 1u, status);
+          if (!ok) break;
+          mbar_expect_tx(&p_full[ps], (uint32_t)nkb * 8192u);
+          for (int kb = 0; kb < nkb; ++kb) tma_load_3d(sP + ps * kAPStageBytes + kb * 8192, mm->p16, kb * 64, t * kARows, pc, &p_full[ps]);
         }
       }
     }
@@ -353,7 +363,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
     const int q = warp & 3, grp = ew >> 2;  // lane quarter (fixed by the hardware), row group 0..3
     const int colq = q * 32 + lane;          // column within the strip
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-    const int tile_off = (colq >> 6) * 8192 + (colq & 63) * 2;  // inside a 16 KB tile of two 64-column boxes
+    const int tile_off = colq * 2;  // inside a 16 KB tile of 64 rows x 128 columns
     const float lr = sc.lr, om = sc.omega;
     const bool full = sc.form == LORDO_QHM_FULL;
     const float a2w = full ? om : 1.f;
@@ -390,7 +400,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       for (int t = 0; t < nsteps; ++t, ++jt) {
         const int is = jt % kAInStages;
         const uint32_t b = jt & 1u;
-        unsigned char* base = sIn + is * kAInStageBytes + tile_off + grp * 16 * 128;
+        unsigned char* base = sIn + is * kAInStageBytes + tile_off + grp * 16 * 256;
         ok = mbar_wait<32>(&in_full[is], (jt / kAInStages) & 1u, status);
         if (ok) ok = mbar_wait<32>(&acc_full[b], (jt >> 1) & 1u, status);
         if (!ok) break;
@@ -398,13 +408,13 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
         float g[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(base + j * 128));
+        for (int j = 0; j < 16; ++j) g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(base + j * 256));
         float acc[16];
         if (ef) {
           tmem_ld16(taddr, acc);  // (P g)^T
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
-            unsigned short* ep = reinterpret_cast<unsigned short*>(base + 16384 + j * 128);
+            unsigned short* ep = reinterpret_cast<unsigned short*>(base + 16384 + j * 256);
             *ep = f_to_bf16((c * g[j] + bf16_to_f(*ep)) - acc[j]);
           }
         }
@@ -413,21 +423,17 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         mbar_arrive(&acc_empty[b]);
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          unsigned short* wp = reinterpret_cast<unsigned short*>(base + 32768 + j * 128);
+          unsigned short* wp = reinterpret_cast<unsigned short*>(base + 32768 + j * 256);
           *wp = f_to_bf16(bf16_to_f(*wp) - lr * (cd * g[j] + a2w * acc[j]));
         }
         // the four warps of a row group hand their 16 rows to the TMA engine on their own
         fence_async_smem();
         asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory");
         if ((ew & 3) == 0 && lane == 0) {
-          unsigned char* sb = sIn + is * kAInStageBytes + grp * 16 * 128;
+          unsigned char* sb = sIn + is * kAInStageBytes + grp * 16 * 256;
           const int row = t * kARows + grp * 16;
-          if (ef) {
-            tma_store_3d(mm->e_st, n0, row, rep, sb + 16384);
-            tma_store_3d(mm->e_st, n0 + 64, row, rep, sb + 24576);
-          }
+          if (ef) tma_store_3d(mm->e_st, n0, row, rep, sb + 16384);
           tma_store_3d(mm->w_st, n0, row, rep, sb + 32768);
-          tma_store_3d(mm->w_st, n0 + 64, row, rep, sb + 40960);
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(&in_free[is]);
