@@ -207,6 +207,23 @@ def run_oracle_sample(sample, variant_name: str, seed: int = 0):
     return dt, sample.weight_replicas * sample.H
 
 
+def max_over_ranks(value_ms: float, device=None) -> float:
+    """Slowest rank's time (every rank runs its own copy of the workload; there is no other
+    exchange on this path). Works on any initialised process group (NCCL on GPUs, gloo on CPU)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value_ms)
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank: int, world: int, ms_max: float) -> float:
+    """Whole-job throughput: the units all ranks processed divided by the slowest rank's time."""
+    return units_per_rank * world / (ms_max * 1e-3)
+
+
 def cpu_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -325,14 +342,9 @@ def main():
         sampler.stop()
     flags = opt.poll_status()
 
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-
+    ms_total = max_over_ranks(ms_total, dev)
     n_inner = H * args.steps
-    params = wl.weight_replicas * n_inner * world
-    value = params / (ms_total * 1e-3)
+    value = aggregate_value(wl.weight_replicas * n_inner, world, ms_total)
 
     # ---- per-class figures and the roofline of the dominant kernel -----------------------------
     tc_active = (args.mode == "fast" and max(r for _, _, r in wl.mats) <= 256 and wl.w_dtype == wl.g_dtype == wl.e_dtype)
@@ -384,11 +396,8 @@ def main():
         ev1.record()
         barrier()
         ms_e2e = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": wl.weight_replicas * n_done * world / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        ms_e2e = max_over_ranks(ms_e2e, dev)
+        e2e = {"value": aggregate_value(wl.weight_replicas * n_done, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": 4 * wl.K, "inner_steps_timed": n_done,
                "note": "inner steps through lordo_inner_step_host; the outer step and the refresh take no host input"}
         del G_host

@@ -467,3 +467,21 @@ def test_bf16_storage_rounds_once_per_step():
     for arr in (o.W[0], o.E[0]):
         assert np.array_equal(arr, lo.round_bf16(arr))
     assert np.array_equal(o.u[0], o.u[0].astype(np.float32).astype(np.float64))
+
+
+# ---------------------------------------------------------------------------------------------
+# stored outputs (tests/golden/, written by tests/golden/make_golden.py from the oracle alone)
+# ---------------------------------------------------------------------------------------------
+def test_golden_files_match_the_oracle():
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "make_golden.py"))
+    mg = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mg)
+    want = np.loadtxt(os.path.join(here, "generator_seed7_purpose2_mat5_index3_replica2_4x8.txt"))
+    assert np.array_equal(want, lo.random_matrix(7, 2, 5, 3, 2, 4, 8))
+    assert abs(want).max() <= 32 and want.std() > 2.0  # centred Binomial(64, 1/2): sd 4
+    for variant, form, name in ((0, 2, "global_fullqhm"), (1, 1, "local_lowqhm")):
+        stored = np.loadtxt(os.path.join(here, f"tiny_8x8_{name}_weights.txt"))
+        np.testing.assert_allclose(mg.tiny_run(variant, form), stored, rtol=1e-12, atol=1e-15)
