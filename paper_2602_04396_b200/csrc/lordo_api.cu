@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kMaxK = 64;
 
-enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3 };
+enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3, ST_SKETCH = 4, ST_CONVERT = 5 };
 enum Phase { PH_SUBSPACE = 0, PH_ROTATE = 1, PH_COMMIT = 2 };
 
 // One launch of the refresh / init / inner-step plans. The entries it works on are a contiguous
@@ -38,6 +38,8 @@ struct SlotBuilder {
     std::vector<CholProblem> ch;
     std::vector<RandProblem> rn;
     std::vector<CopyProblem> cp;
+    std::vector<SkProblem> sk;
+    std::vector<ConvProblem> cv;
   };
   std::vector<Slot> slots;
   size_t cur = 0;
@@ -85,6 +87,8 @@ struct lordo_ctx {
   CholProblem* d_chols = nullptr;
   RandProblem* d_rands = nullptr;
   CopyProblem* d_copies = nullptr;
+  SkProblem* d_sks = nullptr;
+  ConvProblem* d_convs = nullptr;
   float* d_scratch = nullptr;
   long long total_chunks = 0, total_mom_tiles = 0, total_wblks = 0, total_sblks = 0;
 
@@ -112,6 +116,10 @@ struct lordo_ctx {
   std::vector<CholProblem> h_chols;
   std::vector<RandProblem> h_rands;
   std::vector<CopyProblem> h_copies;
+  std::vector<SkProblem> h_sks;
+  std::vector<ConvProblem> h_convs;
+  struct SketchBufs { __nv_bfloat16 *om16 = nullptr, *pn16 = nullptr, *zq16 = nullptr; };
+  std::vector<SketchBufs> h_skbufs;  // per matrix: bf16 right-hand sides of the sketch products (refresh scratch)
   PlanStep inner_proj, inner_apply;
   std::vector<PlanStep> refresh_steps, init_steps;
 
@@ -252,8 +260,10 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       const lordo_mat& a = cfg.mats[i];
       const long long maxd = a.m > a.n ? a.m : a.n;
       const size_t nb = local ? K : 1;
-      const size_t per = (size_t)a.n * a.r + 2 * (size_t)a.m * a.r + (size_t)maxd * a.r + (q > 0 ? 2 * (size_t)a.n * a.r : 0) +
-                         4 * (size_t)a.r * a.r;
+      size_t per = (size_t)a.n * a.r + 2 * (size_t)a.m * a.r + (size_t)maxd * a.r + (q > 0 ? 2 * (size_t)a.n * a.r : 0) +
+                   4 * (size_t)a.r * a.r;
+      // bf16 right-hand sides of the tensor-core sketch products (Omega, P', Z), counted in floats
+      per += ((size_t)a.n * a.r + (q > 0 ? (size_t)a.m * a.r + (size_t)a.n * a.r : 0)) / 2 + 64;
       mat_scratch[i] = nb * per;
       if (acc > 0 && acc + mat_scratch[i] > kRefreshScratchFloats) { ++grp; acc = 0; }
       group_of[i] = grp;
@@ -271,7 +281,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   for (int i = 0; i < n_mats; ++i) {
     const lordo_mat& a = cfg.mats[i];
     MatDev& md = c->h_mats[i];
-    md.m = a.m; md.n = a.n; md.r = a.r; md.pad = 0;
+    md.m = a.m; md.n = a.n; md.r = a.r; md.pad = 0; md.Delta16 = nullptr;
     md.ghat = cv.take<float>((size_t)K * a.r * a.n);
     md.util = cv.take<float>((size_t)K * a.r * a.n);
     md.dcol = cv.take<float>((size_t)K * a.n);
@@ -343,11 +353,15 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     c->tma = cfg.w_dtype == LORDO_BF16;
     c->d_maps = cv.take<TmaMatMaps>(n_mats);
     c->d_gmaps = cv.take<TmaGradMaps>(n_mats);
+    if (c->tma && !local)
+      for (int i = 0; i < n_mats; ++i) c->h_mats[i].Delta16 = cv.take<__nv_bfloat16>((size_t)c->h_mats[i].m * c->h_mats[i].n);
   }
 
   // ---------------- launch plans ----------------
   std::vector<GemmProblem>& P = c->h_probs;
-  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear();
+  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear();
+  c->h_skbufs.assign(n_mats, lordo_ctx::SketchBufs());
+  const bool tc_sketch = c->tc && c->tma;  // sketch products of the refresh on tensor cores
   auto gemm_prob = [&](int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
     GemmProblem g;
     std::memset(&g, 0, sizeof(g));
@@ -381,6 +395,12 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       } else if (st.type == ST_RANDOM) {
         st.first = (long long)c->h_rands.size(); st.count = (int)sl.rn.size(); st.tiles = 0;
         for (RandProblem& x : sl.rn) { x.blk_start = st.tiles; st.tiles += (x.count + 255) / 256; c->h_rands.push_back(x); }
+      } else if (st.type == ST_SKETCH) {
+        st.first = (long long)c->h_sks.size(); st.count = (int)sl.sk.size(); st.tiles = 0;
+        for (SkProblem& x : sl.sk) { x.tile_start = st.tiles; st.tiles += (x.M + 127) / 128; c->h_sks.push_back(x); }
+      } else if (st.type == ST_CONVERT) {
+        st.first = (long long)c->h_convs.size(); st.count = (int)sl.cv.size(); st.tiles = 0;
+        for (ConvProblem& x : sl.cv) { x.blk_start = st.tiles; st.tiles += (x.count + 1023) / 1024; c->h_convs.push_back(x); }
       } else {
         st.first = (long long)c->h_copies.size(); st.count = (int)sl.cp.size(); st.tiles = 0;
         for (CopyProblem& x : sl.cp) { x.blk_start = st.tiles; st.tiles += (x.chunks + 1023) / 1024; c->h_copies.push_back(x); }
@@ -484,6 +504,39 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       float* lw = s; s += (size_t)nb * r * r;
       float* rinv = s; s += (size_t)nb * r * r;
       float* rot = s; s += (size_t)nb * r * r;
+      __nv_bfloat16* om16 = reinterpret_cast<__nv_bfloat16*>(s); s += ((size_t)nb * n * r) / 2 + 16;
+      __nv_bfloat16 *pn16 = nullptr, *zq16 = nullptr;
+      if (q > 0) {
+        pn16 = reinterpret_cast<__nv_bfloat16*>(s); s += ((size_t)nb * m * r) / 2 + 16;
+        zq16 = reinterpret_cast<__nv_bfloat16*>(s); s += ((size_t)nb * n * r) / 2 + 16;
+      }
+      c->h_skbufs[i].om16 = om16; c->h_skbufs[i].pn16 = pn16; c->h_skbufs[i].zq16 = zq16;
+      // S * B on tensor cores: a_mn = 0 -> S rows are the output rows (Y = S B), 1 -> S^T B
+      auto sketch = [&](SlotBuilder& sb, int a_mn, unsigned char* map_b, float* C, long long cstride, long long Mo, long long Kd) {
+        SlotBuilder::Slot& sl = sb.next(ST_SKETCH, PH_SUBSPACE);
+        for (int b = 0; b < nb; ++b) {
+          SkProblem sp;
+          std::memset(&sp, 0, sizeof(sp));
+          sp.M = (int)Mo; sp.Kd = (int)Kd; sp.r = r; sp.r_n = (r + 15) / 16 * 16;
+          sp.a_mn = a_mn; sp.a_c2 = local ? b : 0; sp.b_c2 = b;
+          TmaMatMaps* mm = c->d_maps + i;
+          TmaGradMaps* gm = c->d_gmaps + i;
+          if (local) {
+            sp.map_a = a_mn ? gm->g_sw : gm->g_kb;
+            if (cfg.error_feedback) { sp.map_e = a_mn ? mm->e_sw : mm->e_kb; sp.cptr = c->d_coef + (size_t)i * K + b; }
+          } else {
+            sp.map_a = a_mn ? mm->d_sw : mm->d_kb;
+          }
+          sp.map_b = map_b;
+          sp.C = C + (long long)b * cstride; sp.ldc = r;
+          sl.sk.push_back(sp);
+        }
+      };
+      auto convert = [&](SlotBuilder& sb, const float* src, __nv_bfloat16* dst, size_t count) {
+        ConvProblem cp;
+        cp.src = src; cp.dst = dst; cp.count = (long long)count; cp.blk_start = 0;
+        sb.next(ST_CONVERT, PH_SUBSPACE).cv.push_back(cp);
+      };
 
       auto signal = [&](int b) {  // S of problem b: Delta (Global) or c_k G_k + E_k (Local), stored [m][n]
         if (!local) return plain(md.Delta, n);
@@ -501,22 +554,33 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         SlotBuilder::Slot& f = R.next(ST_RANDOM, PH_SUBSPACE);
         for (int b = 0; b < nb; ++b) {
           RandProblem rp;
-          rp.out = Om + (long long)b * n * r; rp.count = n * r; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
+          rp.out = tc_sketch ? nullptr : Om + (long long)b * n * r;
+          rp.out16 = tc_sketch ? om16 + (long long)b * n * r : nullptr;
+          rp.count = n * r; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
           f.rn.push_back(rp);
         }
       }
-      {  // Y = S Omega
+      if (tc_sketch) {  // Y = S Omega
+        if (!local) convert(R, md.Delta, md.Delta16, (size_t)m * n);  // bf16 copy of the Global signal
+        sketch(R, 0, (c->d_maps + i)->om16, Ya, m * r, m, n);
+      } else {
         SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
         for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
       }
       cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
       for (int it = 0; it < q; ++it) {
-        {  // Z = S^T P'
+        if (tc_sketch) {  // Z = S^T P'
+          convert(R, Pn, pn16, (size_t)nb * m * r);
+          sketch(R, 1, (c->d_maps + i)->pn16, Za, n * r, n, m);
+        } else {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, r, (int)m, signal(b), plain(Pn + (long long)b * m * r, r), nullptr, store_epi(Za + (long long)b * n * r, r)));
         }
         cholqr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n, r, nb, gram, lw, rinv);
-        {  // Y = S Z
+        if (tc_sketch) {  // Y = S Z
+          convert(R, Zq, zq16, (size_t)nb * n * r);
+          sketch(R, 0, (c->d_maps + i)->zq16, Ya, m * r, m, n);
+        } else {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Zq + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
         }
@@ -544,7 +608,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       add_copy(R, PH_COMMIT, md.P, Pn, (size_t)nb * m * r * sizeof(float));
       if (!local) {  // P_0 = orthonormalised random m x r matrix
         RandProblem rp;
-        rp.out = Ya; rp.count = m * r; rp.blk_start = 0; rp.purpose = 1; rp.mat = i; rp.replica = 0; rp.pad = 0;
+        rp.out = Ya; rp.out16 = nullptr; rp.count = m * r; rp.blk_start = 0; rp.purpose = 1; rp.mat = i; rp.replica = 0; rp.pad = 0;
         I.next(ST_RANDOM, PH_SUBSPACE, 0, 0, 0, 1).rn.push_back(rp);
         cholqr2(I, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, md.P, m * r, m, r, 1, gram, lw, rinv);
       }
@@ -556,6 +620,8 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   c->d_chols = cv.take<CholProblem>(c->h_chols.size() + 1);
   c->d_rands = cv.take<RandProblem>(c->h_rands.size() + 1);
   c->d_copies = cv.take<CopyProblem>(c->h_copies.size() + 1);
+  c->d_sks = cv.take<SkProblem>(c->h_sks.size() + 1);
+  c->d_convs = cv.take<ConvProblem>(c->h_convs.size() + 1);
 
   c->last_G.assign(n_mats, nullptr);
   return (cv.off + 255) & ~size_t(255);
@@ -618,6 +684,14 @@ int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t 
       launch_fill_random_grouped(c->d_rands + s.first, s.count, s.tiles, c->cfg.seed, s.p0 ? 0 : c->refreshes, st);
       c->launches += 1;
       return check_launch(c, "fill_random");
+    case ST_SKETCH:
+      launch_sketch_tma(c->d_sks + s.first, s.count, s.tiles, c->sm_count, c->d_status, st);
+      c->launches += 1;
+      return check_launch(c, "sketch");
+    case ST_CONVERT:
+      launch_convert_grouped(c->d_convs + s.first, s.count, s.tiles, st);
+      c->launches += 1;
+      return check_launch(c, "convert");
     case ST_COPY:
       launch_copy_grouped(c->d_copies + s.first, s.count, s.tiles, st);
       c->launches += 1;
@@ -643,6 +717,7 @@ int set_gradients(lordo_ctx* c, const void* const* G, cudaStream_t st) {
     for (int i = 0; i < c->n_mats; ++i) {
       const lordo_mat& a = c->mats[i];
       if (!encode_map3(c->h_gmaps[i].g_sw, G[i], a.n, a.m, c->K, 64, 64, true) ||
+          !encode_map3(c->h_gmaps[i].g_kb, G[i], a.n, a.m, c->K, 64, 128, true) ||
           !encode_map3(c->h_gmaps[i].g_ns, G[i], a.n, a.m, c->K, 128, 64, false))
         return fail(c, LORDO_ERR_CUDA, "tensor map encoding failed for a gradient");
     }
@@ -739,6 +814,8 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   if (!c->h_chols.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_chols, c->h_chols.data(), sizeof(CholProblem) * c->h_chols.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_rands.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_rands, c->h_rands.data(), sizeof(RandProblem) * c->h_rands.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_copies.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_copies, c->h_copies.data(), sizeof(CopyProblem) * c->h_copies.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_sks.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_sks, c->h_sks.data(), sizeof(SkProblem) * c->h_sks.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_convs.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_convs, c->h_convs.data(), sizeof(ConvProblem) * c->h_convs.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
   if (c->tc) {
     INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));
@@ -767,6 +844,17 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         good = good && encode_map3(hm[i].w_st, md.W, md.n, md.m, c->K, 128, 16, false);
         good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n, true);
         good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
+        // refresh: signal as rows (64 k x 128 rows) and right-hand sides [batch][Kd][r]
+        const int nbatch = loc ? c->K : 1;
+        if (md.E) good = good && encode_map3(hm[i].e_kb, md.E, md.n, md.m, c->K, 64, 128, true);
+        if (md.Delta16) {
+          good = good && encode_map3(hm[i].d_kb, md.Delta16, md.n, md.m, 1, 64, 128, true);
+          good = good && encode_map3(hm[i].d_sw, md.Delta16, md.n, md.m, 1, 64, 64, true);
+        }
+        const lordo_ctx::SketchBufs& sb = c->h_skbufs[i];
+        good = good && encode_map3(hm[i].om16, sb.om16, md.r, md.n, nbatch, 64, 64, true);
+        if (sb.pn16) good = good && encode_map3(hm[i].pn16, sb.pn16, md.r, md.m, nbatch, 64, 64, true);
+        if (sb.zq16) good = good && encode_map3(hm[i].zq16, sb.zq16, md.r, md.n, nbatch, 64, 64, true);
       }
       if (good) {
         INIT_CUDA(cudaMemcpyAsync(c->d_maps, hm.data(), sizeof(TmaMatMaps) * nm, cudaMemcpyHostToDevice, st));
@@ -774,7 +862,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         INIT_CUDA(tma_configure());
         if (cudaHostAlloc((void**)&c->h_gmaps, sizeof(TmaGradMaps) * nm, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
       } else {
-        c->tma = false;  // no tensor-map encoder in this driver: the register-staged kernels run instead
+        return bail(LORDO_ERR_CUDA);  // tensor maps could not be encoded (driver without cuTensorMapEncodeTiled?)
       }
     }
   }

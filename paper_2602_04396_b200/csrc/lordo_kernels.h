@@ -94,10 +94,13 @@ struct TcProblem {
 // without swizzle (tiles the update epilogue reads and writes in place); "st": 128 x 16 boxes.
 struct alignas(128) TmaMatMaps {
   unsigned char e_sw[128], pt[128], p16[128], e_ns[128], w_ns[128];
+  // refresh: E and Delta16 as 64 x 128 swizzled boxes ("kb", rows of S as MMA rows), Delta16 as
+  // 64 x 64 swizzled boxes, and the three bf16 right-hand sides [batch][Kd][r]
+  unsigned char e_kb[128], d_kb[128], d_sw[128], om16[128], pn16[128], zq16[128];
   unsigned char e_st[128], w_st[128];  // stores of one row group of the update epilogue
 };
 struct alignas(128) TmaGradMaps {  // re-encoded whenever the caller's gradient pointer changes
-  unsigned char g_sw[128], g_ns[128];
+  unsigned char g_sw[128], g_ns[128], g_kb[128];
 };
 
 struct TcPrep {
@@ -137,7 +140,8 @@ void launch_chol_inverse(const CholProblem* probs, int nprobs, int r_max, unsign
 // Grouped helpers of the refresh: random sketches and device-to-device copies for many matrices
 // in one launch each. blk_start is the first 256-thread block of the entry within the launch.
 struct RandProblem {
-  float* out;
+  float* out;            // fp32 output, may be null
+  __nv_bfloat16* out16;  // bf16 output, may be null
   long long count, blk_start;
   int purpose, mat, replica, pad;
 };
@@ -149,6 +153,28 @@ struct CopyProblem {
 void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long total_blocks, unsigned long long seed, long long index,
                                 cudaStream_t st);
 void launch_copy_grouped(const CopyProblem* probs, int nprobs, long long total_blocks, cudaStream_t st);
+struct ConvProblem {
+  const float* src;
+  __nv_bfloat16* dst;
+  long long count, blk_start;  // 1024 elements per block
+};
+void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long total_blocks, cudaStream_t st);
+
+// Tensor-core sketch products of the refresh (lordo_tma.cu): C[M x r] (fp32) = S * B with the big
+// signal matrix S streamed by TMA as bf16 (optionally formed as c*G + E in shared memory) and
+// B [Kd][r] in bf16. a_mn = 1: S is stored [Kd][M] (the product S^T P'); 0: stored [M][Kd].
+struct SkProblem {
+  long long tile_start;      // first 128-row tile of this problem within the launch
+  int M, Kd, r, r_n;
+  int a_mn, a_c2, b_c2, pad;  // third TMA coordinate (worker / batch index) of A and of B
+  const void* map_a;         // 64 x 64 swizzled boxes (a_mn) or 64 x 128 swizzled boxes
+  const void* map_e;         // same shape over E, or null
+  const void* map_b;         // 64 x 64 swizzled boxes over B [batch][Kd][r]
+  const float* cptr;         // scale of A when map_e is set (clip coefficient), else null
+  float* C;
+  long long ldc;
+};
+void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, unsigned* status, cudaStream_t st);
 
 // streaming kernels
 void launch_sumsq_partial(const MatDev* mats, const void* const* G, const long long* chunk_start, int n_mats, int K, int g_dt,

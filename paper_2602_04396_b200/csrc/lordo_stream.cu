@@ -262,7 +262,24 @@ __global__ void __launch_bounds__(256) fill_random_grouped_kernel(const RandProb
   if (c >= pb.count) return;
   const unsigned long long key = stream_key(seed, pb.purpose, pb.mat, index, pb.replica);
   const unsigned long long w = mix64(key + kGolden * (unsigned long long)(c + 1));
-  pb.out[c] = (float)(__popcll(w) - 32);
+  const float val = (float)(__popcll(w) - 32);
+  if (pb.out) pb.out[c] = val;
+  if (pb.out16) pb.out16[c] = __float2bfloat16_rn(val);  // integers in [-32, 32]: exact in bf16
+}
+
+// fp32 -> bf16 copies of many buffers in one launch (operands of the tensor-core sketch products)
+__global__ void __launch_bounds__(256) convert_grouped_kernel(const ConvProblem* __restrict__ probs, int nprobs) {
+  const long long blk = blockIdx.x;
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].blk_start <= blk) lo = mid; else hi = mid - 1;
+  }
+  const ConvProblem pb = probs[lo];
+  const long long e = ((blk - pb.blk_start) * 256 + threadIdx.x) * 4;  // count is a multiple of 8
+  if (e >= pb.count) return;
+  const float4 v = *reinterpret_cast<const float4*>(pb.src + e);
+  store4(pb.dst, LORDO_BF16, e, v);
 }
 
 // Device-to-device copies of many buffers in one launch (16-byte chunks).
@@ -292,6 +309,9 @@ __global__ void __launch_bounds__(256) copy_grouped_kernel(const CopyProblem* __
 void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long total_blocks, unsigned long long seed, long long index,
                                 cudaStream_t st) {
   fill_random_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs, seed, index);
+}
+void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long total_blocks, cudaStream_t st) {
+  convert_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs);
 }
 void launch_copy_grouped(const CopyProblem* probs, int nprobs, long long total_blocks, cudaStream_t st) {
   copy_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs);

@@ -448,8 +448,12 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
 }
 
 // =================================================================================================
+cudaError_t sketch_configure();
+
 cudaError_t tma_configure() {
-  cudaError_t e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
+  cudaError_t e = sketch_configure();
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(apply_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)(kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024));
@@ -465,6 +469,182 @@ void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips
   const long long g = total_strips < grid ? total_strips : grid;
   apply_tma_kernel<<<(unsigned)g, kAThreads, kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, st>>>(probs, nprobs, total_strips,
                                                                                                              maps, gmaps, sc, status);
+}
+
+}  // namespace lordo
+
+// =================================================================================================
+// Sketch products of the refresh: C = S * B (fp32 out), S streamed by TMA. Same pipeline as the
+// projection: TMA -> (optional c*G + E in place) -> tcgen05.mma -> epilogue out of tensor memory,
+// two accumulator buffers, one CTA per SM walking the tile list.
+// =================================================================================================
+namespace lordo {
+using namespace umma;
+namespace {
+constexpr int kSStages = 3;
+constexpr uint32_t kSStageBytes = 65536;  // A 16 KB | E 16 KB | B up to 32 KB
+constexpr int kSThreads = (2 + 4 + 4) * 32;  // TMA, MMA, 4 transform warps, 4 epilogue warps
+constexpr uint32_t kIdescBMajorMN = 1u << 16;
+
+__device__ __forceinline__ int find_sk(const SkProblem* __restrict__ probs, int nprobs, long long tile) {
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].tile_start <= tile) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+}  // namespace
+
+__global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProblem* __restrict__ probs, int nprobs, long long total_tiles,
+                                                                  unsigned* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t full_bar[kSStages], xform_bar[kSStages], empty_bar[kSStages], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_slot;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    for (int s = 0; s < kSStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], 128); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    mbar_init_fence();
+  }
+  if (warp == 1) tmem_alloc(&tmem_slot, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
+        const int m0 = (int)(tile - pr->tile_start) * 128;
+        const int nkb = (pr->Kd + 63) / 64, nbox = (pr->r_n + 63) / 64;
+        const bool has_e = pr->map_e != nullptr;
+        const uint32_t tx = 16384u + (has_e ? 16384u : 0u) + (uint32_t)nbox * 8192u;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kSStages;
+          ok = mbar_wait(&empty_bar[s], ((it / kSStages) & 1u) ^ 1u, status);
+          if (!ok) break;
+          unsigned char* base = smem + s * kSStageBytes;
+          mbar_expect_tx(&full_bar[s], tx);
+          if (pr->a_mn) {  // S stored [Kd][M]: two boxes of 64 k-rows x 64 columns
+            tma_load_3d(base, pr->map_a, m0, kb * 64, pr->a_c2, &full_bar[s]);
+            tma_load_3d(base + 8192, pr->map_a, m0 + 64, kb * 64, pr->a_c2, &full_bar[s]);
+            if (has_e) {
+              tma_load_3d(base + 16384, pr->map_e, m0, kb * 64, pr->a_c2, &full_bar[s]);
+              tma_load_3d(base + 24576, pr->map_e, m0 + 64, kb * 64, pr->a_c2, &full_bar[s]);
+            }
+          } else {         // S stored [M][Kd]: one box of 128 rows x 64 k
+            tma_load_3d(base, pr->map_a, kb * 64, m0, pr->a_c2, &full_bar[s]);
+            if (has_e) tma_load_3d(base + 16384, pr->map_e, kb * 64, m0, pr->a_c2, &full_bar[s]);
+          }
+          for (int j = 0; j < nbox; ++j) tma_load_3d(base + 32768 + j * 8192, pr->map_b, j * 64, kb * 64, pr->b_c2, &full_bar[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, si = 0;
+      bool ok = true;
+      for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++si) {
+        const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
+        const int nkb = (pr->Kd + 63) / 64;
+        const bool a_mn = pr->a_mn != 0;
+        const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)pr->r_n) | kIdescBMajorMN | (a_mn ? kIdescAMajorMN : 0u);
+        const uint32_t buf = si & 1u;
+        ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
+        if (!ok) break;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % kSStages;
+          ok = mbar_wait(&xform_bar[s], (it / kSStages) & 1u, status);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t sA = smem_u32(smem + s * kSStageBytes), sB = sA + 32768;
+#pragma unroll
+          for (int k16 = 0; k16 < 4; ++k16) {
+            const uint64_t ad = a_mn ? smem_desc_mn128(sA + k16 * 2048) : smem_desc_k128(sA + k16 * 32);
+            mma_bf16(tmem + buf * 256, ad, smem_desc_mn128(sB + k16 * 2048), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          }
+          mma_commit(&empty_bar[s]);
+        }
+        if (ok) mma_commit(&acc_full[buf]);
+      }
+    }
+  } else if (warp < 6) {
+    const int xt = tid - 64;
+    uint32_t it = 0;
+    bool ok = true;
+    for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
+      const int nkb = (pr->Kd + 63) / 64;
+      const bool has_e = pr->map_e != nullptr;
+      const float c = pr->cptr ? *pr->cptr : 1.f;
+      for (int kb = 0; kb < nkb; ++kb, ++it) {
+        const int s = it % kSStages;
+        ok = mbar_wait(&full_bar[s], (it / kSStages) & 1u, status);
+        if (!ok) break;
+        if (has_e) {
+          uint4* G = reinterpret_cast<uint4*>(smem + s * kSStageBytes);
+          const uint4* E = G + 1024;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int idx = xt + i * 128;
+            const uint4 g = G[idx], e = E[idx];
+            uint4 a;
+            a.x = pack2_bf16(fmaf(c, bf_lo(g.x), bf_lo(e.x)), fmaf(c, bf_hi(g.x), bf_hi(e.x)));
+            a.y = pack2_bf16(fmaf(c, bf_lo(g.y), bf_lo(e.y)), fmaf(c, bf_hi(g.y), bf_hi(e.y)));
+            a.z = pack2_bf16(fmaf(c, bf_lo(g.z), bf_lo(e.z)), fmaf(c, bf_hi(g.z), bf_hi(e.z)));
+            a.w = pack2_bf16(fmaf(c, bf_lo(g.w), bf_lo(e.w)), fmaf(c, bf_hi(g.w), bf_hi(e.w)));
+            G[idx] = a;
+          }
+          fence_async_smem();
+        }
+        mbar_arrive(&xform_bar[s]);
+      }
+    }
+  } else {
+    // epilogue: lane = row of the tile, r_n fp32 columns out of tensor memory
+    const int q = warp & 3;
+    uint32_t si = 0;
+    bool ok = true;
+    for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++si) {
+      const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
+      const long long row = (tile - pr->tile_start) * 128 + q * 32 + lane;
+      const bool row_ok = row < pr->M;
+      float* __restrict__ crow = pr->C + (row_ok ? row : 0) * pr->ldc;
+      const int r = pr->r, r_n = pr->r_n;
+      const uint32_t buf = si & 1u;
+      ok = mbar_wait<64>(&acc_full[buf], (si >> 1) & 1u, status);
+      if (!ok) break;
+      tc_fence_after_sync();
+      for (int ch = 0; ch < r_n / 16; ++ch) {
+        float v[16];
+        tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + buf * 256 + (uint32_t)(ch * 16), v);
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            if (ch * 16 + j < r) *reinterpret_cast<float4*>(crow + ch * 16 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+      }
+      tc_fence_before_sync();
+      mbar_arrive(&acc_empty[buf]);
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_free(tmem, 512);
+}
+
+cudaError_t sketch_configure() {
+  return cudaFuncSetAttribute(sketch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSStages * kSStageBytes + 1024));
+}
+void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, unsigned* status, cudaStream_t st) {
+  const long long g = total_tiles < grid ? total_tiles : grid;
+  sketch_tma_kernel<<<(unsigned)g, kSThreads, kSStages * kSStageBytes + 1024, st>>>(probs, nprobs, total_tiles, status);
 }
 
 }  // namespace lordo

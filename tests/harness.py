@@ -130,11 +130,29 @@ def run_lockstep_refresh(spec: RunSpec):
     lr, b1, om = f32(spec.lr), f32(spec.beta1), f32(spec.omega)
     worst: Dict[str, float] = {}
 
-    def after_refresh():
+    def after_refresh(signals=None):
         torch.cuda.synchronize()
         st = compare_states(opt, orc)
         for k in ("P_angle", "P_orth", "u", "v"):
             worst[k] = max(worst.get(k, 0.0), st[k])
+        if signals is not None:
+            # share of the signal's energy that the CUDA path's subspace captures, relative to the
+            # oracle's subspace for the same signal and sketch
+            for i, per_rep in enumerate(signals):
+                Pg, Po = _np_state(opt.P[i]), orc.P[i]
+                if Pg.ndim == 2:
+                    Pg, Po = Pg[None], Po[None]
+                for k, S in enumerate(per_rep):
+                    ratio = float(np.sum((Pg[k].T @ S) ** 2) / max(np.sum((Po[k].T @ S) ** 2), 1e-300))
+                    worst["energy"] = min(worst.get("energy", 1e9), ratio)
+
+    def local_signals(G):
+        coef = lo.clip_coefficients(G, orc.cfg.clip_rho, orc.cfg.clip_scope)
+        out = []
+        for i in range(len(wl.mats)):
+            out.append([coef[i, k] * np.asarray(G[i][k], dtype=np.float64) + (orc.E[i][k] if spec.error_feedback else 0.0)
+                        for k in range(wl.K)])
+        return out
 
     for rnd in range(spec.n_rounds):
         for h in range(spec.n_H):
@@ -143,9 +161,10 @@ def run_lockstep_refresh(spec: RunSpec):
             if spec.variant == 1 and h == 0:
                 torch.cuda.synchronize()
                 sync_oracle_from_gpu(opt, orc)
+                sig = local_signals(G)
                 opt.refresh_subspace(Gd, spec.beta1)
                 orc.refresh_subspace(G, b1)
-                after_refresh()
+                after_refresh(sig)
             opt.inner_step(Gd, spec.lr, spec.beta1, spec.omega, spec.form)
             orc.inner_step(G, lr, b1, om, spec.form)
         opt.outer_step()
@@ -153,9 +172,10 @@ def run_lockstep_refresh(spec: RunSpec):
         if spec.variant == 0:
             torch.cuda.synchronize()
             sync_oracle_from_gpu(opt, orc)
+            sig = [[orc.Delta[i].copy()] for i in range(len(wl.mats))]
             opt.refresh_subspace(None, spec.beta1)
             orc.refresh_subspace(None, b1)
-            after_refresh()
+            after_refresh(sig)
     torch.cuda.synchronize()
     return opt, orc, worst
 

@@ -177,6 +177,24 @@ def test_fast_mode_full_loop_with_refresh():
             assert bool(torch.isfinite(w.float()).all())
 
 
+@pytest.mark.parametrize("variant,form,q", [(0, 2, 0), (0, 2, 2), (1, 1, 0), (1, 1, 2)])
+@pytest.mark.parametrize("shape", [(264, 200, 32), (520, 392, 136)])
+def test_fast_mode_refresh_on_tensor_cores(variant, form, q, shape):
+    """bf16 storage in fast mode: the sketch products S*Omega, S^T*P', S*Z run on tensor cores with
+    bf16 operands, so the basis is not the oracle's vector by vector. What a range finder is for is
+    checked instead, on the CUDA path's own state: the new basis is orthonormal and captures the same
+    share of the signal's energy as the oracle's basis (to 1 %), and the rotated moments are finite."""
+    m, n, r = shape
+    wl = _small(m=m, n=n, r=r, K=2, H=2, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0, power_iters=q,
+                w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0, eps=0.05)
+    opt, orc, worst = hz.run_lockstep_refresh(spec)
+    assert opt.poll_status() == 0
+    assert worst["P_orth"] < 1e-5 and abs(worst["energy"] - 1.0) < 1e-2, worst
+    for t in list(opt.u) + list(opt.v) + list(opt.P):
+        assert bool(torch.isfinite(t).all())
+
+
 # ------------------------------------------------------------------ outer step
 
 @pytest.mark.parametrize("outer", [0, 1])
