@@ -140,6 +140,18 @@ def test_fast_mode_inner_steps_bf16(shape, form, variant, ef):
     assert (d <= 1).mean() > 0.99 and d.max() <= 8, ((d <= 1).mean(), d.max())
 
 
+@pytest.mark.parametrize("shape", [(64, 64, 8), (24, 264, 16), (1024, 8, 8), (72, 136, 64), (130, 1032, 24)])
+def test_fast_mode_bf16_small_and_ragged_shapes(shape):
+    """Shapes below one tile in one or both directions, and strips / row blocks with ragged tails."""
+    m, n, r = shape
+    wl = _small(m=m, n=n, r=r, K=3, H=2, rounds=2, clip_rho=30.0, w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    spec = RunSpec(wl, variant=1, form=2, refresh=False, lr=0.01, omega=0.9, check_mode=0, eps=0.05, outer=1)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert opt.poll_status() == 0
+    assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["E"] < 2 * FAST_TOL and st["X0"] < 0.05, st
+
+
 def test_fast_mode_adam_eps():
     """With Adam's own eps = 1e-8 the first steps' update is sign-like, and an entry of the low-rank
     gradient that is smaller than the bf16 rounding of its terms can land on the other sign; that is
