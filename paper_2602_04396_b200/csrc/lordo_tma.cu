@@ -406,25 +406,28 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
-        float g[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(base + j * 256));
-        float acc[16];
-        if (ef) {
-          tmem_ld16(taddr, acc);  // (P g)^T
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            unsigned short* ep = reinterpret_cast<unsigned short*>(base + 16384 + j * 256);
-            *ep = f_to_bf16((c * g[j] + bf16_to_f(*ep)) - acc[j]);
-          }
-        }
-        tmem_ld16(taddr + 64, acc);  // (P U~)^T
+        // both accumulators come out of tensor memory together and the buffer goes back to the MMA
+        // warp before any arithmetic; the tiles are then updated in place, 8 rows at a time
+        float a1[16], a2[16];
+        tmem_ld16x2(taddr, taddr + 64, a1, a2);  // (P g)^T, (P U~)^T
         tc_fence_before_sync();
         mbar_arrive(&acc_empty[b]);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          unsigned short* wp = reinterpret_cast<unsigned short*>(base + 32768 + j * 256);
-          *wp = f_to_bf16(bf16_to_f(*wp) - lr * (cd * g[j] + a2w * acc[j]));
+        for (int h = 0; h < 2; ++h) {
+          float g[8], e[8], w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            unsigned char* rowp = base + (h * 8 + j) * 256;
+            g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp));
+            e[j] = ef ? bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 16384)) : 0.f;
+            w[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 32768));
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            unsigned char* rowp = base + (h * 8 + j) * 256;
+            if (ef) *reinterpret_cast<unsigned short*>(rowp + 16384) = f_to_bf16((c * g[j] + e[j]) - a1[h * 8 + j]);
+            *reinterpret_cast<unsigned short*>(rowp + 32768) = f_to_bf16(w[j] - lr * (cd * g[j] + a2w * a2[h * 8 + j]));
+          }
         }
         // the four warps of a row group hand their 16 rows to the TMA engine on their own
         fence_async_smem();
