@@ -731,7 +731,7 @@ int run_clip(lordo_ctx* c, cudaStream_t st) {
   launch_sumsq_partial(c->d_mats, c->d_Gtab, c->d_chunk_start, c->n_mats, c->K, c->cfg.g_dtype, c->d_partial, c->total_chunks, st);
   launch_clip_finalize(c->d_mats, c->d_chunk_start, c->n_mats, c->K, c->d_partial, c->cfg.clip_rho, c->cfg.clip_scope, c->d_coef,
                        c->d_sumsq, c->d_status, st);
-  c->launches += 2;
+  c->launches += 3;
   return check_launch(c, "clip");
 }
 

@@ -40,43 +40,45 @@ __global__ void __launch_bounds__(256) sumsq_partial_kernel(const MatDev* __rest
   }
 }
 
-// One block per replica. Sums the partials of every matrix in a fixed order.
-__global__ void __launch_bounds__(256) clip_finalize_kernel(const MatDev* __restrict__ mats, const long long* __restrict__ chunk_start,
-                                                            int n_mats, int K, const double* __restrict__ partial, float rho,
-                                                            int scope, float* __restrict__ coef, double* __restrict__ sumsq,
-                                                            unsigned* __restrict__ status) {
-  const int k = blockIdx.x;
+// Step 1: one block per (matrix, replica) sums that pair's partials in a fixed order.
+__global__ void __launch_bounds__(256) clip_matrix_sums_kernel(const MatDev* __restrict__ mats, const long long* __restrict__ chunk_start,
+                                                               int K, const double* __restrict__ partial, float rho, int scope,
+                                                               float* __restrict__ coef, double* __restrict__ sumsq) {
+  const int i = blockIdx.x, k = blockIdx.y;
   __shared__ double red[256];
-  __shared__ double total_s;
-  double total = 0.0;
-  for (int i = 0; i < n_mats; ++i) {
-    const long long elems = mats[i].m * mats[i].n;
-    const long long chunks = (elems + kSqChunk - 1) / kSqChunk;
-    const double* p = partial + chunk_start[i] + (long long)k * chunks;
-    double a = 0.0;
-    for (long long c = threadIdx.x; c < chunks; c += 256) a += p[c];
-    red[threadIdx.x] = a;
-    __syncthreads();
-    for (int s = 128; s > 0; s >>= 1) {
-      if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
-      __syncthreads();
-    }
-    const double s_i = red[0];
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      sumsq[(long long)i * K + k] = s_i;
-      if (scope == 1) coef[(long long)i * K + k] = fminf(1.f, rho / ((float)sqrt(s_i) + 1e-6f));
-    }
-    total += s_i;
-  }
-  if (threadIdx.x == 0) total_s = total;
+  const long long elems = mats[i].m * mats[i].n;
+  const long long chunks = (elems + kSqChunk - 1) / kSqChunk;
+  const double* p = partial + chunk_start[i] + (long long)k * chunks;
+  double a = 0.0;
+  for (long long c = threadIdx.x; c < chunks; c += 256) a += p[c];
+  red[threadIdx.x] = a;
   __syncthreads();
-  total = total_s;
-  if (threadIdx.x == 0 && !isfinite(total)) atomicOr(status, LORDO_FLAG_NONFINITE_GRAD);
-  if (scope == 0) {
-    const float c = fminf(1.f, rho / ((float)sqrt(total) + 1e-6f));
-    for (int i = threadIdx.x; i < n_mats; i += 256) coef[(long long)i * K + k] = c;
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
   }
+  if (threadIdx.x == 0) {
+    const double s_i = red[0];
+    sumsq[(long long)i * K + k] = s_i;
+    if (scope == 1) coef[(long long)i * K + k] = fminf(1.f, rho / ((float)sqrt(s_i) + 1e-6f));
+  }
+}
+
+// Step 2: one block per replica adds the matrices' sums in matrix order (thread 0, so the order
+// is fixed) and writes the coefficient of the per-worker norm.
+__global__ void __launch_bounds__(256) clip_finalize_kernel(int n_mats, int K, float rho, int scope, float* __restrict__ coef,
+                                                            const double* __restrict__ sumsq, unsigned* __restrict__ status) {
+  const int k = blockIdx.x;
+  __shared__ float c_s;
+  if (threadIdx.x == 0) {
+    double total = 0.0;
+    for (int i = 0; i < n_mats; ++i) total += sumsq[(long long)i * K + k];
+    if (!isfinite(total)) atomicOr(status, LORDO_FLAG_NONFINITE_GRAD);
+    c_s = fminf(1.f, rho / ((float)sqrt(total) + 1e-6f));
+  }
+  __syncthreads();
+  if (scope == 0)
+    for (int i = threadIdx.x; i < n_mats; i += 256) coef[(long long)i * K + k] = c_s;
 }
 
 __global__ void fill_float_kernel(float* __restrict__ p, long long count, float value) {
@@ -322,7 +324,8 @@ void launch_sumsq_partial(const MatDev* mats, const void* const* G, const long l
 }
 void launch_clip_finalize(const MatDev* mats, const long long* chunk_start, int n_mats, int K, const double* partial, float rho,
                           int scope, float* coef, double* sumsq, unsigned* status, cudaStream_t st) {
-  clip_finalize_kernel<<<K, 256, 0, st>>>(mats, chunk_start, n_mats, K, partial, rho, scope, coef, sumsq, status);
+  clip_matrix_sums_kernel<<<dim3(n_mats, K), 256, 0, st>>>(mats, chunk_start, K, partial, rho, scope, coef, sumsq);
+  clip_finalize_kernel<<<K, 256, 0, st>>>(n_mats, K, rho, scope, coef, sumsq, status);
 }
 void launch_fill_float(float* p, long long count, float value, cudaStream_t st) {
   fill_float_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(p, count, value);
