@@ -356,3 +356,70 @@ def test_config5_scaled():
     opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
     st = _bf16_check(opt, orc)
     assert st["P_angle"] < ANGLE_TOL and st["u"] < 2e-3 and st["v"] < 2e-3, st
+
+
+# ------------------------------------------------------------------ full size, the bench's launch configuration
+
+def test_config4_full_size_fast_mode_sampled_columns():
+    """The whole 1B-shaped stack (168 matrices, K = 8, r = 256, bf16) in fast mode, exactly the launch
+    configuration bench.py times. The inner step is separable by column (column j of W, E, u, v depends
+    on column j of G only, given P and the clip coefficient), so the oracle recomputes sampled columns
+    of one matrix per shape class one by one; the clip coefficients are checked against a plain
+    torch reduction over all gradients."""
+    from paper_2602_04396_b200 import lordo
+    free, _total = torch.cuda.mem_get_info()
+    if free < 125 * 2 ** 30:
+        pytest.skip("needs about 120 GB of free device memory")
+    wl = synth.scaled(synth.config(4), H=2)
+    seed, lr, beta1, omega, form = 11, 0.004, 0.999, 0.97, 2
+    W0 = synth.init_weights_device(wl, seed)
+    sampled = {0: None, 4: None, 6: None}  # one attention, one gate/up, one down projection
+    rng = np.random.default_rng(5)
+    for i in sampled:
+        m, n, r = wl.mats[i]
+        cols = np.unique(np.concatenate([rng.integers(0, n, 6), [0, n - 1]]))
+        sampled[i] = (cols, W0[i][:, torch.from_numpy(cols).cuda()].float().cpu().numpy().astype(np.float64))
+    opt = lordo.Lordo(wl.mats, wl.K, wl.H, W0, g_dtype=torch.bfloat16, e_dtype=torch.bfloat16, variant=0, error_feedback=True,
+                      beta2=0.999, eps=0.05, clip_rho=wl.clip_rho, outer=lordo.OUTER_NESTEROV, outer_lr=0.8, outer_momentum=0.9,
+                      seed=seed, check_mode=0)
+    del W0
+    oracles = {}
+    for i, (cols, w0) in sampled.items():
+        m, n, r = wl.mats[i]
+        cfg = lo.OracleConfig(mats=((m, len(cols), r),), K=wl.K, H=wl.H, variant=0, beta2=hz.f32(0.999), eps=hz.f32(0.05), clip_rho=0.0,
+                              w_dtype="bf16", e_dtype="bf16", state_dtype="f32")
+        P0 = lo.store(lo.householder_qr_q(lo.random_matrix(seed, lo.PURPOSE_P0, i, 0, 0, m, r)), "f32")
+        oracles[i] = lo.LordoOracle(cfg, [w0], P0=[P0])
+    G = None
+    for h in range(2):
+        G = synth.gradients_device(wl, seed, 0, h, out=G)
+        sq = torch.zeros(wl.K, dtype=torch.float64, device="cuda")
+        for g in G:
+            sq += g.float().pow(2).sum(dim=(1, 2), dtype=torch.float64)
+        c_want = np.minimum(1.0, wl.clip_rho / (np.sqrt(sq.cpu().numpy()) + 1e-6))
+        opt.inner_step(G, lr, beta1, omega, form)
+        c_got = opt.clip_coefficients().cpu().numpy()
+        assert np.abs(c_got - c_want[None, :]).max() <= 2e-6 * c_want.max()
+        for i, (cols, _w0) in sampled.items():
+            gj = G[i][:, :, torch.from_numpy(cols).cuda()].float().cpu().numpy().astype(np.float64)
+            oracles[i].inner_step([gj * c_want[:, None, None]], hz.f32(lr), hz.f32(beta1), hz.f32(omega), form)
+    assert opt.poll_status() == 0
+    for i, (cols, _w0) in sampled.items():
+        orc = oracles[i]
+        jj = torch.from_numpy(cols).cuda()
+        got = {name: getattr(opt, name)[i][:, :, jj].float().cpu().numpy().astype(np.float64) for name in ("W", "E", "u", "v")}
+        assert hz.scaled_error(got["u"], orc.u[0]) < FAST_TOL and hz.scaled_error(got["v"], orc.v[0]) < 2 * FAST_TOL, i
+        assert hz.scaled_error(got["E"], orc.E[0]) < 2 * FAST_TOL, i
+        d = hz.bf16_ulp_distance(got["W"], orc.W[0])
+        assert (d <= 1).mean() > 0.99 and d.max() <= 8, (i, (d <= 1).mean(), d.max())
+    # outer step and Global refresh at full size: properties that hold at any size
+    opt.outer_step()
+    opt.refresh_subspace(None, beta1)
+    assert opt.poll_status() == 0
+    for i in sampled:
+        W = opt.W[i]
+        assert bool((W == W[0:1]).all())  # every worker holds the broadcast model
+        assert float((opt.X0[i] - W[0].float()).abs().max()) <= 2.0 ** -8 * float(opt.X0[i].abs().max())
+        P = opt.P[i].double()
+        assert float((P.T @ P - torch.eye(P.shape[1], device="cuda", dtype=torch.float64)).abs().max()) < 1e-5
+    opt.close()
