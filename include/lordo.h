@@ -165,7 +165,11 @@ LORDO_API int lordo_refresh_subspace(lordo_ctx* ctx, const void* const* G_or_nul
  * LORDO_ERR_NUMERIC if it is non-zero, else LORDO_OK. */
 LORDO_API int lordo_poll_status(lordo_ctx* ctx, void* stream, uint32_t* flags);
 
-/* Counters for checkpoint / resume: {inner steps done, refreshes done, outer steps done, 0}. */
+/* Counters for checkpoint / resume: {inner steps done, refreshes done, outer steps done, inner steps
+ * done in the current round}. A checkpoint is the caller's tensors (W, E, P, u, v, X0, B, Delta) plus
+ * these four numbers: restore the tensors into the buffers of a context made with the same
+ * configuration, then call lordo_set_counters (which also makes the library rebuild its internal
+ * copies of P before the next step). */
 LORDO_API int lordo_get_counters(const lordo_ctx* ctx, int64_t out[4]);
 LORDO_API int lordo_set_counters(lordo_ctx* ctx, const int64_t in[4]);
 

@@ -132,6 +132,7 @@ struct lordo_ctx {
   int64_t steps = 0, refreshes = 0, outers = 0, launches = 0;
   int steps_in_round = 0;
   bool after_outer = false;
+  bool p_copies_stale = false;  // the caller may have restored P: the bf16 operand copies are remade before the next use
   std::string err;
 
   // optional per-kernel-class timing (lordo_profile_enable)
@@ -928,6 +929,11 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
 
   if (c->tc) {
     ss.lr = lr;
+    if (c->p_copies_stale) {
+      launch_prep_projection(c->d_tc_prep, c->d_prep_start, (int)c->h_prep.size(), c->prep_blocks, st);
+      c->launches += 1;
+      c->p_copies_stale = false;
+    }
     if (c->tma) {
       {
         ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
@@ -1085,6 +1091,7 @@ int lordo_set_counters(lordo_ctx* c, const int64_t in[4]) {
   if (in[0] < 0 || in[1] < 0 || in[2] < 0 || in[3] < 0 || in[3] > c->cfg.H) return fail(c, LORDO_ERR_INVALID_ARG, "counter out of range");
   c->steps = in[0]; c->refreshes = in[1]; c->outers = in[2]; c->steps_in_round = (int)in[3];
   c->after_outer = false;
+  c->p_copies_stale = true;  // a restored checkpoint brings its own P
   return LORDO_OK;
 }
 

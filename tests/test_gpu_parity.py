@@ -423,3 +423,51 @@ def test_config4_full_size_fast_mode_sampled_columns():
         P = opt.P[i].double()
         assert float((P.T @ P - torch.eye(P.shape[1], device="cuda", dtype=torch.float64)).abs().max()) < 1e-5
     opt.close()
+
+
+# ------------------------------------------------------------------ determinism and checkpoint / resume
+
+def _run_rounds_gpu(opt, wl, seed, rounds, first_round, variant, form, lr=0.01, beta1=0.9, omega=0.9):
+    for rnd in range(first_round, first_round + rounds):
+        for h in range(wl.H):
+            G = hz.device_grads(wl, synth.gradients(wl, seed, rnd, h))
+            if variant == 1 and h == 0:
+                opt.refresh_subspace(G, beta1)
+            opt.inner_step(G, lr, beta1, omega, form)
+        opt.outer_step()
+        if variant == 0:
+            opt.refresh_subspace(None, beta1)
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dt,mode", [("f32", 1), ("bf16", 0)])
+@pytest.mark.parametrize("variant", [0, 1])
+def test_rerun_is_bitwise_identical_and_checkpoint_resumes(dt, mode, variant):
+    """Two runs of the same schedule give the same bits (no atomics, fixed summation orders), and a
+    run restored from the caller's tensors plus lordo_get_counters continues bit for bit."""
+    wl = _small(m=264, n=200, r=32, K=2, H=2, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0, w_dtype=dt, g_dtype=dt,
+                e_dtype=dt)
+    spec = RunSpec(wl, variant=variant, form=2, outer=1, check_mode=mode)
+    names = ("W", "E", "P", "u", "v", "X0", "B", "Delta")
+    a = hz.make_gpu(spec)
+    _run_rounds_gpu(a, wl, 0, 2, 0, variant, 2)
+    b = hz.make_gpu(spec)
+    _run_rounds_gpu(b, wl, 0, 1, 0, variant, 2)
+    saved = {n: [t.clone() for t in getattr(b, n)] for n in names}
+    counters = b.counters()
+    b.close()
+    c = hz.make_gpu(spec)
+    for n in names:
+        for dst, src in zip(getattr(c, n), saved[n]):
+            dst.copy_(src)
+    c.set_counters(counters)
+    _run_rounds_gpu(c, wl, 0, 1, 1, variant, 2)
+    for n in names:
+        for x, y in zip(getattr(a, n), getattr(c, n)):
+            assert torch.equal(x, y), n
+    d = hz.make_gpu(spec)
+    _run_rounds_gpu(d, wl, 0, 2, 0, variant, 2)
+    for n in names:
+        for x, y in zip(getattr(a, n), getattr(d, n)):
+            assert torch.equal(x, y), n
+    assert a.poll_status() == 0
