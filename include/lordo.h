@@ -165,6 +165,18 @@ LORDO_API int lordo_refresh_subspace(lordo_ctx* ctx, const void* const* G_or_nul
  * LORDO_ERR_NUMERIC if it is non-zero, else LORDO_OK. */
 LORDO_API int lordo_poll_status(lordo_ctx* ctx, void* stream, uint32_t* flags);
 
+/* Clears the sticky device flag word (after the caller has dealt with what lordo_poll_status reported). */
+LORDO_API int lordo_clear_status(lordo_ctx* ctx, void* stream);
+
+/*
+ * Self-test of the failure path of the tensor-core kernels: every wait inside them (on a TMA
+ * transfer, a tensor-core commit, another warp) is bounded; a wait that runs out sets
+ * LORDO_FLAG_DEVICE_TIMEOUT and the kernel runs to its normal end, so the context stays usable.
+ * This call enqueues a one-thread kernel that waits on a barrier nothing completes: about two
+ * seconds later lordo_poll_status reports the flag. It touches no optimizer state.
+ */
+LORDO_API int lordo_selftest_wait_timeout(lordo_ctx* ctx, void* stream);
+
 /* Counters for checkpoint / resume: {inner steps done, refreshes done, outer steps done, inner steps
  * done in the current round}. A checkpoint is the caller's tensors (W, E, P, u, v, X0, B, Delta) plus
  * these four numbers: restore the tensors into the buffers of a context made with the same

@@ -1080,6 +1080,19 @@ int lordo_poll_status(lordo_ctx* c, void* stream, uint32_t* flags) {
   return LORDO_OK;
 }
 
+int lordo_selftest_wait_timeout(lordo_ctx* c, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  launch_selftest_wait(c->d_status, reinterpret_cast<cudaStream_t>(stream));
+  c->launches += 1;
+  return check_launch(c, "selftest_wait");
+}
+
+int lordo_clear_status(lordo_ctx* c, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  CUDA_OK(c, cudaMemsetAsync(c->d_status, 0, sizeof(unsigned), reinterpret_cast<cudaStream_t>(stream)));
+  return LORDO_OK;
+}
+
 int lordo_get_counters(const lordo_ctx* c, int64_t out[4]) {
   if (!c || !out) return LORDO_ERR_INVALID_ARG;
   out[0] = c->steps; out[1] = c->refreshes; out[2] = c->outers; out[3] = c->steps_in_round;

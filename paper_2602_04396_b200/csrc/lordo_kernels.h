@@ -126,6 +126,8 @@ void launch_project_tma(const TcProblem* probs, int nprobs, long long total_stri
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
                       const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
 
+void launch_selftest_wait(unsigned* status, cudaStream_t st);
+
 // Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
 // gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the
 // diagonal. lwork: r*r floats per problem. Strides in floats between batch entries.

@@ -651,3 +651,19 @@ void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles
 }
 
 }  // namespace lordo
+
+// =================================================================================================
+// Self-test of the bounded wait: one thread waits on an mbarrier phase that nothing completes. The
+// wait must give up after its limit, set LORDO_FLAG_DEVICE_TIMEOUT in *status and let the kernel end.
+// =================================================================================================
+namespace lordo {
+__global__ void selftest_wait_kernel(unsigned* __restrict__ status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    umma::mbar_init(&bar, 1);
+    umma::mbar_init_fence();
+    (void)umma::mbar_wait(&bar, 0u, status);
+  }
+}
+void launch_selftest_wait(unsigned* status, cudaStream_t st) { selftest_wait_kernel<<<1, 32, 0, st>>>(status); }
+}  // namespace lordo

@@ -25,7 +25,7 @@ EXPORTS = [
     "lordo_refresh_subspace", "lordo_poll_status", "lordo_get_counters", "lordo_set_counters",
     "lordo_clip_coefficients", "lordo_launch_count", "lordo_last_error", "lordo_status_string", "lordo_destroy",
     "lordo_fill_random", "lordo_profile_enable", "lordo_profile_read", "lordo_clip_coefficient_static",
-    "lordo_clip_coefficient_static_max_count",
+    "lordo_clip_coefficient_static_max_count", "lordo_clear_status", "lordo_selftest_wait_timeout",
 ]
 
 
@@ -86,6 +86,8 @@ def load_library() -> C.CDLL:
     lib.lordo_fill_random.argtypes = [C.c_uint64, i32, i32, i64, i32, i64, i64, vp, vp]
     lib.lordo_profile_enable.argtypes = [vp, i32]
     lib.lordo_profile_read.argtypes = [vp, vp, C.POINTER(f32)]
+    lib.lordo_clear_status.argtypes = [vp, vp]
+    lib.lordo_selftest_wait_timeout.argtypes = [vp, vp]
     lib.lordo_clip_coefficient_static.argtypes = [vp, i32, i64, f32, vp, vp]
     lib.lordo_clip_coefficient_static_max_count.argtypes = []
     lib.lordo_clip_coefficient_static_max_count.restype = i64
@@ -256,6 +258,12 @@ class Lordo:
         if rc not in (0, 7):
             self._check(rc, "lordo_poll_status")
         return flags.value
+
+    def clear_status(self, stream=None):
+        self._check(self.lib.lordo_clear_status(self._ctx, _stream_handle(stream)), "lordo_clear_status")
+
+    def selftest_wait_timeout(self, stream=None):
+        self._check(self.lib.lordo_selftest_wait_timeout(self._ctx, _stream_handle(stream)), "lordo_selftest_wait_timeout")
 
     def counters(self) -> List[int]:
         out = (C.c_int64 * 4)()

@@ -249,6 +249,25 @@ def test_rank_deficient_sketch_raises_flag_and_stays_finite():
     assert bool(torch.isfinite(opt.P[0]).all())
 
 
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    """A device-side wait that nothing completes gives up after its limit, raises the timeout flag and
+    lets the kernel end; the same context then runs a correct step."""
+    wl = _small(m=200, n=136, r=24, K=2, H=2, rounds=1, clip_rho=30.0)
+    spec = RunSpec(wl, refresh=False, lr=0.01)
+    opt = hz.make_gpu(spec)
+    opt.selftest_wait_timeout()
+    assert opt.poll_status() & 4
+    opt.clear_status()
+    assert opt.poll_status() == 0
+    orc = hz.make_oracle(spec)
+    for h in range(2):
+        G = synth.gradients(wl, 0, 0, h)
+        opt.inner_step(hz.device_grads(wl, G), 0.01, 0.9, 0.97, 0)
+        orc.inner_step(G, hz.f32(0.01), hz.f32(0.9), hz.f32(0.97), 0)
+    st = hz.compare_states(opt, orc)
+    assert st["W"] < W_TOL and st["u"] < 1e-4 and opt.poll_status() == 0, st
+
+
 def test_call_order_is_checked():
     from paper_2602_04396_b200 import lordo
     wl = _small(m=64, n=64, r=8, K=2, H=2, rounds=1)
