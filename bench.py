@@ -347,7 +347,8 @@ def main():
     value = aggregate_value(wl.weight_replicas * n_inner, world, ms_total)
 
     # ---- per-class figures and the roofline of the dominant kernel -----------------------------
-    tc_active = (args.mode == "fast" and max(r for _, _, r in wl.mats) <= 256 and wl.w_dtype == wl.g_dtype == wl.e_dtype)
+    tc_active = (args.mode == "fast" and wl.w_dtype == wl.g_dtype == wl.e_dtype and
+                 max(r for _, _, r in wl.mats) <= (512 if wl.w_dtype == "bf16" else 256))
     abytes = algorithmic_bytes(wl, hp["variant"], hp["form"], True, tc_active)
     per_launch = {"clip": n_inner, "project": n_inner, "moments": n_inner, "apply": n_inner, "outer_states": args.steps,
                   "outer_weights": args.steps, "refresh": args.steps * (H if wl.refresh_every_step else 1)}

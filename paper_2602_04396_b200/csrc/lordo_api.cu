@@ -296,8 +296,8 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
 
   // ---------------- tensor-core operand copies and problem table ----------------
   c->tc = cfg.check_mode == 0 && cfg.g_dtype == cfg.w_dtype && (!cfg.error_feedback || cfg.e_dtype == cfg.w_dtype);
-  for (int i = 0; i < n_mats; ++i)
-    if (cfg.mats[i].r > 256) c->tc = false;  // larger ranks run on the fp32 path
+  for (int i = 0; i < n_mats; ++i)  // ranks above 512 (above 256 with fp32 storage) run on the fp32 path
+    if (cfg.mats[i].r > (cfg.w_dtype == LORDO_BF16 ? 512 : 256)) c->tc = false;
   c->h_tc.clear(); c->h_prep.clear(); c->h_prep_start.assign(1, 0);
   c->tc_strips = 0; c->tc_rn_max = 0; c->tc_rk_max = 0;
   if (c->tc) {
@@ -686,7 +686,7 @@ int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t 
       c->launches += 1;
       return check_launch(c, "fill_random");
     case ST_SKETCH:
-      launch_sketch_tma(c->d_sks + s.first, s.count, s.tiles, c->sm_count, c->d_status, st);
+      launch_sketch_tma(c->d_sks + s.first, s.count, s.tiles, c->sm_count, c->tc_rn_max > 256, c->d_status, st);
       c->launches += 1;
       return check_launch(c, "sketch");
     case ST_CONVERT:
@@ -819,7 +819,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   if (!c->h_convs.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_convs, c->h_convs.data(), sizeof(ConvProblem) * c->h_convs.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
   if (c->tc) {
-    INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));
+    if (!c->tma) INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));  // register-staged kernels (fp32 storage)
     INIT_CUDA(cudaMemsetAsync(c->d_tc_bf16, 0, c->tc_bf16_bytes, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_tc_probs, c->h_tc.data(), sizeof(TcProblem) * c->h_tc.size(), cudaMemcpyHostToDevice, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_tc_prep, c->h_prep.data(), sizeof(TcPrep) * c->h_prep.size(), cudaMemcpyHostToDevice, st));
@@ -843,7 +843,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         }
         good = good && encode_map3(hm[i].w_ns, md.W, md.n, md.m, c->K, 128, 64, false);
         good = good && encode_map3(hm[i].w_st, md.W, md.n, md.m, c->K, 128, 16, false);
-        good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n, true);
+        good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n < 256 ? tp.r_n : 256, true);
         good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
         // refresh: signal as rows (64 k x 128 rows) and right-hand sides [batch][Kd][r]
         const int nbatch = loc ? c->K : 1;
@@ -935,13 +935,22 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
       c->p_copies_stale = false;
     }
     if (c->tma) {
+      const int big = c->tc_rn_max > 256;
       {
         ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
-        launch_project_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, c->d_status, st);
+        launch_project_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, big, c->d_status, st);
       }
       {
         ProfScope ps(c, st, PC_APPLY);
-        launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, c->d_status, st);
+        if (!big) {
+          launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, 0, c->d_status, st);
+        } else {  // 256 < r <= 512: the error-feedback sweep, then the model-update sweep
+          if (c->cfg.error_feedback) {
+            launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, 1, c->d_status, st);
+            c->launches += 1;
+          }
+          launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, 2, c->d_status, st);
+        }
       }
     } else {
     {

@@ -122,9 +122,10 @@ void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips,
 // TMA-fed persistent kernels for bf16 storage (lordo_tma.cu).
 cudaError_t tma_configure();
 void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                        const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
+                        const StepScalars& sc, int grid, int big, unsigned* status, cudaStream_t st);
+// mode 0: r <= 256, one sweep; modes 1 and 2: the two sweeps for 256 < r <= 512
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                      const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
+                      const StepScalars& sc, int grid, int mode, unsigned* status, cudaStream_t st);
 
 void launch_selftest_wait(unsigned* status, cudaStream_t st);
 
@@ -176,7 +177,7 @@ struct SkProblem {
   float* C;
   long long ldc;
 };
-void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, unsigned* status, cudaStream_t st);
+void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, int big, unsigned* status, cudaStream_t st);
 
 // streaming kernels
 void launch_sumsq_partial(const MatDev* mats, const void* const* G, const long long* chunk_start, int n_mats, int K, int g_dt,

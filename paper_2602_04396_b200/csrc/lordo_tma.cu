@@ -59,13 +59,18 @@ constexpr int kAThreads = (3 + kAEpiWarps) * 32;  // 608: TMA inputs, MMA, 16 ep
 }  // namespace
 
 // =================================================================================================
+// BIG: 256 < r <= 512. The accumulator then fills all 512 columns of tensor memory (one buffer, no
+// overlap of the epilogue with the next strip) and a stage holds a 64 KB P^T tile (two stages).
+template <bool BIG>
 __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
                                                                    const TmaMatMaps* __restrict__ maps,
                                                                    const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
                                                                    unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ uint64_t full_bar[kPStages], xform_bar[kPStages], empty_bar[kPStages], acc_full[2], acc_empty[2];
+  constexpr int ST = BIG ? 2 : 3;
+  constexpr uint32_t SB = BIG ? 98304u : kPStageBytes;
+  __shared__ uint64_t full_bar[3], xform_bar[3], empty_bar[3], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ float dsum_s[kStrip];
 
@@ -73,7 +78,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
   const bool ef = sc.ef != 0;
 
   if (tid == 0) {
-    for (int s = 0; s < kPStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], kPXformWarps * 32); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < ST; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], kPXformWarps * 32); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kPEpiWarps * 32); }
     mbar_init_fence();
   }
@@ -94,12 +99,13 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
         const TmaMatMaps* mm = maps + pr->mat;
         const TmaGradMaps* gm = gmaps + pr->mat;
         const int nkb = pr->m_k / 64, rep = pr->replica, pc = pr->pcopy;
-        const uint32_t tx = 16384u + (ef ? 16384u : 0u) + (uint32_t)pr->r_n * 128u;
+        const int pt_rows = pr->r_n < 256 ? pr->r_n : 256;  // rows of one P^T box
+        const uint32_t tx = 16384u + (ef ? 16384u : 0u) + (uint32_t)pt_rows * 128u * (BIG ? 2u : 1u);
         for (int kb = 0; kb < nkb; ++kb, ++it) {
-          const int s = it % kPStages;
-          ok = mbar_wait(&empty_bar[s], ((it / kPStages) & 1u) ^ 1u, status);
+          const int s = it % ST;
+          ok = mbar_wait(&empty_bar[s], ((it / ST) & 1u) ^ 1u, status);
           if (!ok) break;
-          unsigned char* base = smem + s * kPStageBytes;
+          unsigned char* base = smem + s * SB;
           mbar_expect_tx(&full_bar[s], tx);
           tma_load_3d(base, gm->g_sw, n0, kb * 64, rep, &full_bar[s]);
           tma_load_3d(base + 8192, gm->g_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
@@ -108,6 +114,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
             tma_load_3d(base + 24576, mm->e_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
           }
           tma_load_3d(base + 32768, mm->pt, kb * 64, 0, pc, &full_bar[s]);
+          if (BIG) tma_load_3d(base + 32768 + pt_rows * 128, mm->pt, kb * 64, 256, pc, &full_bar[s]);
         }
       }
     }
@@ -119,19 +126,24 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
         const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
         const int nkb = pr->m_k / 64;
-        const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)pr->r_n) | kIdescAMajorMN;
-        const uint32_t buf = si & 1u;
-        ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
+        const uint32_t n_lo = pr->r_n < 256 ? (uint32_t)pr->r_n : 256u, n_hi = (uint32_t)pr->r_n - n_lo;
+        const uint32_t idesc = idesc_bf16_f32(128, n_lo) | kIdescAMajorMN;
+        const uint32_t idesc_hi = idesc_bf16_f32(128, n_hi ? n_hi : 16u) | kIdescAMajorMN;
+        const uint32_t buf = BIG ? 0u : (si & 1u);
+        ok = mbar_wait(&acc_empty[buf], ((BIG ? si : (si >> 1)) & 1u) ^ 1u, status);
         if (!ok) break;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
-          const int s = it % kPStages;
-          ok = mbar_wait(&xform_bar[s], (it / kPStages) & 1u, status);
+          const int s = it % ST;
+          ok = mbar_wait(&xform_bar[s], (it / ST) & 1u, status);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t sA = smem_u32(smem + s * kPStageBytes), sB = sA + 32768;
+          const uint32_t sA = smem_u32(smem + s * SB), sB = sA + 32768;
 #pragma unroll
-          for (int k16 = 0; k16 < 4; ++k16)
-            mma_bf16(tmem + buf * 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          for (int k16 = 0; k16 < 4; ++k16) {
+            const uint32_t acc = (kb > 0 || k16 > 0) ? 1u : 0u;
+            mma_bf16(tmem + buf * 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc, acc);
+            if (BIG && n_hi) mma_bf16(tmem + 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + 256 * 128 + k16 * 32), idesc_hi, acc);
+          }
           mma_commit(&empty_bar[s]);
         }
         if (ok) mma_commit(&acc_full[buf]);
@@ -147,10 +159,10 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       const int nkb = pr->m_k / 64;
       const float c = *pr->cptr;
       for (int kb = 0; kb < nkb; ++kb, ++it) {
-        const int s = it % kPStages;
-        ok = mbar_wait(&full_bar[s], (it / kPStages) & 1u, status);
+        const int s = it % ST;
+        ok = mbar_wait(&full_bar[s], (it / ST) & 1u, status);
         if (!ok) break;
-        uint4* G = reinterpret_cast<uint4*>(smem + s * kPStageBytes);
+        uint4* G = reinterpret_cast<uint4*>(smem + s * SB);
         const uint4* E = G + 1024;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -187,8 +199,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       float* __restrict__ vp_ = pr->v;
       __nv_bfloat16* __restrict__ gT = pr->gT16 + ecolc * r_k;
       __nv_bfloat16* __restrict__ uT = pr->uT16 + ecolc * r_k;
-      const uint32_t buf = si & 1u;
-      ok = mbar_wait<64>(&acc_full[buf], (si >> 1) & 1u, status);
+      const uint32_t buf = BIG ? 0u : (si & 1u);
+      ok = mbar_wait<64>(&acc_full[buf], (BIG ? si : (si >> 1)) & 1u, status);
       if (!ok) break;
       tc_fence_after_sync();
       float dsum = 0.f;
@@ -250,14 +262,22 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
 }
 
 // =================================================================================================
+// MODE 0: r <= 256, both products in one sweep. For 256 < r <= 512 one low-rank operand alone fills
+// 256 columns of tensor memory, so the update is two sweeps of the same kernel: MODE 1 does the
+// error-feedback line (operand g^T, tiles G and E), MODE 2 the model update (operand U~^T, tiles G, W).
+template <int MODE>
 __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
                                                                  const TmaMatMaps* __restrict__ maps,
                                                                  const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
                                                                  unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* sP = smem;                               // kAPStages x 32 KB
-  unsigned char* sIn = smem + kAPStages * kAPStageBytes;  // kAInStages x 48 KB
+  constexpr uint32_t PSB = MODE ? 65536u : kAPStageBytes;  // one stage of rows of P
+  constexpr int INST = MODE ? 2 : kAInStages;
+  constexpr bool DO_E = MODE != 2, DO_W = MODE != 1;
+  constexpr uint32_t A2COL = MODE ? 0u : 128u;             // first column of the U~^T operand
+  unsigned char* sP = smem;                      // kAPStages stages of rows of P
+  unsigned char* sIn = smem + kAPStages * PSB;   // INST stages of G | E | W tiles (48 KB each)
   __shared__ uint64_t p_full[kAPStages], p_empty[kAPStages], in_full[kAInStages], in_free[kAInStages], acc_full[2], acc_empty[2], x_ready;
   __shared__ uint32_t tmem_slot;
 
@@ -266,7 +286,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
 
   if (tid == 0) {
     for (int s = 0; s < kAPStages; ++s) { mbar_init(&p_full[s], 1); mbar_init(&p_empty[s], 1); }
-    for (int s = 0; s < kAInStages; ++s) { mbar_init(&in_full[s], 1); mbar_init(&in_free[s], 4); }
+    for (int s = 0; s < INST; ++s) { mbar_init(&in_full[s], 1); mbar_init(&in_free[s], 4); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kAEpiWarps * 32); }
     mbar_init(&x_ready, kAEpiWarps * 32);
     mbar_init_fence();
@@ -276,7 +296,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
-  // tensor memory: columns [0,128) g^T, [128,256) U~^T (two bf16 per column), [256,512) two buffers of two accumulators
+  // tensor memory: columns [0,256) the low-rank operands, two bf16 per column (MODE 0: g^T then U~^T,
+  // 128 columns each); [256,512) two buffers of two accumulators
 
   if (warp == 0) {
     // ---------------- TMA producer: tiles of G, E, W ---------------------------------------------
@@ -291,14 +312,15 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         const int rep = pr->replica;
         const int nsteps = (pr->m + kARows - 1) / kARows;
         for (int t = 0; t < nsteps; ++t, ++jt) {
-          const int is = jt % kAInStages;
-          ok = mbar_wait(&in_free[is], ((jt / kAInStages) & 1u) ^ 1u, status);
+          const int is = jt % INST;
+          ok = mbar_wait(&in_free[is], ((jt / INST) & 1u) ^ 1u, status);
           if (!ok) break;
           unsigned char* base = sIn + is * kAInStageBytes;
-          mbar_expect_tx(&in_full[is], ef ? 49152u : 32768u);
+          const bool ld_e = DO_E && ef;
+          mbar_expect_tx(&in_full[is], 16384u + (ld_e ? 16384u : 0u) + (DO_W ? 16384u : 0u));
           tma_load_3d(base, gm->g_ns, n0, t * kARows, rep, &in_full[is]);
-          if (ef) tma_load_3d(base + 16384, mm->e_ns, n0, t * kARows, rep, &in_full[is]);
-          tma_load_3d(base + 32768, mm->w_ns, n0, t * kARows, rep, &in_full[is]);
+          if (ld_e) tma_load_3d(base + 16384, mm->e_ns, n0, t * kARows, rep, &in_full[is]);
+          if (DO_W) tma_load_3d(base + 32768, mm->w_ns, n0, t * kARows, rep, &in_full[is]);
         }
       }
     }
@@ -317,7 +339,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           ok = mbar_wait(&p_empty[ps], ((jt / kAPStages) & 1u) ^ 1u, status);
           if (!ok) break;
           mbar_expect_tx(&p_full[ps], (uint32_t)nkb * 8192u);
-          for (int kb = 0; kb < nkb; ++kb) tma_load_3d(sP + ps * kAPStageBytes + kb * 8192, mm->p16, kb * 64, t * kARows, pc, &p_full[ps]);
+          for (int kb = 0; kb < nkb; ++kb) tma_load_3d(sP + ps * PSB + kb * 8192, mm->p16, kb * 64, t * kARows, pc, &p_full[ps]);
         }
       }
     }
@@ -340,7 +362,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           if (ok) ok = mbar_wait(&acc_empty[b], ((jt >> 1) & 1u) ^ 1u, status);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t pbase = smem_u32(sP + ps * kAPStageBytes);
+          const uint32_t pbase = smem_u32(sP + ps * PSB);
           const uint32_t d1 = tmem + 256 + b * 128, d2 = d1 + 64;
           for (int kb = 0; kb < nkb; ++kb) {
 #pragma unroll
@@ -348,8 +370,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
               const uint32_t acc = (kb > 0 || k16 > 0) ? 1u : 0u;
               const uint64_t bd = smem_desc_k128(pbase + kb * 8192 + k16 * 32);
               const uint32_t acol = (uint32_t)(kb * 4 + k16) * 8;
-              mma_bf16_ts(d1, tmem + acol, bd, idesc, acc);
-              mma_bf16_ts(d2, tmem + 128 + acol, bd, idesc, acc);
+              if (DO_E) mma_bf16_ts(d1, tmem + acol, bd, idesc, acc);
+              if (DO_W) mma_bf16_ts(d2, tmem + A2COL + acol, bd, idesc, acc);
             }
           }
           mma_commit(&p_empty[ps]);
@@ -387,21 +409,26 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         const __nv_bfloat16* __restrict__ u16 = pr->uT16 + colc * r_k + grp * (r_k / 4);
         const bool live = col < n;
         for (int c0 = 0; c0 < per; c0 += 8) {
-          uint4 glo = *reinterpret_cast<const uint4*>(g16 + c0 * 2), ghi = *reinterpret_cast<const uint4*>(g16 + c0 * 2 + 8);
-          uint4 ulo = *reinterpret_cast<const uint4*>(u16 + c0 * 2), uhi = *reinterpret_cast<const uint4*>(u16 + c0 * 2 + 8);
-          if (!live) { glo = ghi = ulo = uhi = make_uint4(0u, 0u, 0u, 0u); }
-          tmem_st8(tmem + lane_base + (uint32_t)(grp * per + c0), glo, ghi);
-          tmem_st8(tmem + lane_base + 128u + (uint32_t)(grp * per + c0), ulo, uhi);
+          if (DO_E) {
+            uint4 glo = *reinterpret_cast<const uint4*>(g16 + c0 * 2), ghi = *reinterpret_cast<const uint4*>(g16 + c0 * 2 + 8);
+            if (!live) glo = ghi = make_uint4(0u, 0u, 0u, 0u);
+            tmem_st8(tmem + lane_base + (uint32_t)(grp * per + c0), glo, ghi);
+          }
+          if (DO_W) {
+            uint4 ulo = *reinterpret_cast<const uint4*>(u16 + c0 * 2), uhi = *reinterpret_cast<const uint4*>(u16 + c0 * 2 + 8);
+            if (!live) ulo = uhi = make_uint4(0u, 0u, 0u, 0u);
+            tmem_st8(tmem + lane_base + A2COL + (uint32_t)(grp * per + c0), ulo, uhi);
+          }
         }
         tmem_st_wait();
         tc_fence_before_sync();
         mbar_arrive(&x_ready);
       }
       for (int t = 0; t < nsteps; ++t, ++jt) {
-        const int is = jt % kAInStages;
+        const int is = jt % INST;
         const uint32_t b = jt & 1u;
         unsigned char* base = sIn + is * kAInStageBytes + tile_off + grp * 16 * 256;
-        ok = mbar_wait<32>(&in_full[is], (jt / kAInStages) & 1u, status);
+        ok = mbar_wait<32>(&in_full[is], (jt / INST) & 1u, status);
         if (ok) ok = mbar_wait<32>(&acc_full[b], (jt >> 1) & 1u, status);
         if (!ok) break;
         tc_fence_after_sync();
@@ -409,7 +436,13 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         // both accumulators come out of tensor memory together and the buffer goes back to the MMA
         // warp before any arithmetic; the tiles are then updated in place, 8 rows at a time
         float a1[16], a2[16];
-        tmem_ld16x2(taddr, taddr + 64, a1, a2);  // (P g)^T, (P U~)^T
+        if (MODE == 0) {
+          tmem_ld16x2(taddr, taddr + 64, a1, a2);  // (P g)^T, (P U~)^T
+        } else if (MODE == 1) {
+          tmem_ld16(taddr, a1);
+        } else {
+          tmem_ld16(taddr + 64, a2);
+        }
         tc_fence_before_sync();
         mbar_arrive(&acc_empty[b]);
 #pragma unroll
@@ -419,14 +452,14 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           for (int j = 0; j < 8; ++j) {
             unsigned char* rowp = base + (h * 8 + j) * 256;
             g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp));
-            e[j] = ef ? bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 16384)) : 0.f;
-            w[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 32768));
+            e[j] = (DO_E && ef) ? bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 16384)) : 0.f;
+            w[j] = DO_W ? bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 32768)) : 0.f;
           }
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             unsigned char* rowp = base + (h * 8 + j) * 256;
-            if (ef) *reinterpret_cast<unsigned short*>(rowp + 16384) = f_to_bf16((c * g[j] + e[j]) - a1[h * 8 + j]);
-            *reinterpret_cast<unsigned short*>(rowp + 32768) = f_to_bf16(w[j] - lr * (cd * g[j] + a2w * a2[h * 8 + j]));
+            if (DO_E && ef) *reinterpret_cast<unsigned short*>(rowp + 16384) = f_to_bf16((c * g[j] + e[j]) - a1[h * 8 + j]);
+            if (DO_W) *reinterpret_cast<unsigned short*>(rowp + 32768) = f_to_bf16(w[j] - lr * (cd * g[j] + a2w * a2[h * 8 + j]));
           }
         }
         // the four warps of a row group hand their 16 rows to the TMA engine on their own
@@ -435,8 +468,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         if ((ew & 3) == 0 && lane == 0) {
           unsigned char* sb = sIn + is * kAInStageBytes + grp * 16 * 256;
           const int row = t * kARows + grp * 16;
-          if (ef) tma_store_3d(mm->e_st, n0, row, rep, sb + 16384);
-          tma_store_3d(mm->w_st, n0, row, rep, sb + 32768);
+          if (DO_E && ef) tma_store_3d(mm->e_st, n0, row, rep, sb + 16384);
+          if (DO_W) tma_store_3d(mm->w_st, n0, row, rep, sb + 32768);
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(&in_free[is]);
@@ -456,22 +489,31 @@ cudaError_t sketch_configure();
 cudaError_t tma_configure() {
   cudaError_t e = sketch_configure();
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
+  e = cudaFuncSetAttribute(project_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(apply_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)(kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024));
+  e = cudaFuncSetAttribute(project_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
+  if (e != cudaSuccess) return e;
+  const int smem = (int)(kAPStages * 65536 + 2 * kAInStageBytes + 1024);  // the largest of the three modes
+  e = cudaFuncSetAttribute(apply_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(apply_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(apply_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
 void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                        const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
+                        const StepScalars& sc, int grid, int big, unsigned* status, cudaStream_t st) {
   const long long g = total_strips < grid ? total_strips : grid;
-  project_tma_kernel<<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+  if (big) project_tma_kernel<true><<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+  else project_tma_kernel<false><<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
 }
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                      const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
-  const long long g = total_strips < grid ? total_strips : grid;
-  apply_tma_kernel<<<(unsigned)g, kAThreads, kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, st>>>(probs, nprobs, total_strips,
-                                                                                                             maps, gmaps, sc, status);
+                      const StepScalars& sc, int grid, int mode, unsigned* status, cudaStream_t st) {
+  const unsigned g = (unsigned)(total_strips < grid ? total_strips : grid);
+  const size_t small = kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, large = kAPStages * 65536 + 2 * kAInStageBytes + 1024;
+  if (mode == 0) apply_tma_kernel<0><<<g, kAThreads, small, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+  else if (mode == 1) apply_tma_kernel<1><<<g, kAThreads, large, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+  else apply_tma_kernel<2><<<g, kAThreads, large, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
 }
 
 }  // namespace lordo
@@ -499,16 +541,19 @@ __device__ __forceinline__ int find_sk(const SkProblem* __restrict__ probs, int 
 }
 }  // namespace
 
+template <bool BIG>
 __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProblem* __restrict__ probs, int nprobs, long long total_tiles,
                                                                   unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ uint64_t full_bar[kSStages], xform_bar[kSStages], empty_bar[kSStages], acc_full[2], acc_empty[2];
+  constexpr int ST = BIG ? 2 : 3;
+  constexpr uint32_t SB = BIG ? 98304u : kSStageBytes;
+  __shared__ uint64_t full_bar[3], xform_bar[3], empty_bar[3], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    for (int s = 0; s < kSStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], 128); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < ST; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], 128); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
     mbar_init_fence();
   }
@@ -529,10 +574,10 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
         const bool has_e = pr->map_e != nullptr;
         const uint32_t tx = 16384u + (has_e ? 16384u : 0u) + (uint32_t)nbox * 8192u;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
-          const int s = it % kSStages;
-          ok = mbar_wait(&empty_bar[s], ((it / kSStages) & 1u) ^ 1u, status);
+          const int s = it % ST;
+          ok = mbar_wait(&empty_bar[s], ((it / ST) & 1u) ^ 1u, status);
           if (!ok) break;
-          unsigned char* base = smem + s * kSStageBytes;
+          unsigned char* base = smem + s * SB;
           mbar_expect_tx(&full_bar[s], tx);
           if (pr->a_mn) {  // S stored [Kd][M]: two boxes of 64 k-rows x 64 columns
             tma_load_3d(base, pr->map_a, m0, kb * 64, pr->a_c2, &full_bar[s]);
@@ -557,20 +602,23 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
         const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
         const int nkb = (pr->Kd + 63) / 64;
         const bool a_mn = pr->a_mn != 0;
-        const uint32_t idesc = idesc_bf16_f32(128, (uint32_t)pr->r_n) | kIdescBMajorMN | (a_mn ? kIdescAMajorMN : 0u);
-        const uint32_t buf = si & 1u;
-        ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
+        const uint32_t n_lo = pr->r_n < 256 ? (uint32_t)pr->r_n : 256u, n_hi = (uint32_t)pr->r_n - n_lo;
+        const uint32_t majors = kIdescBMajorMN | (a_mn ? kIdescAMajorMN : 0u);
+        const uint32_t idesc = idesc_bf16_f32(128, n_lo) | majors, idesc_hi = idesc_bf16_f32(128, n_hi ? n_hi : 16u) | majors;
+        const uint32_t buf = BIG ? 0u : (si & 1u);
+        ok = mbar_wait(&acc_empty[buf], ((BIG ? si : (si >> 1)) & 1u) ^ 1u, status);
         if (!ok) break;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
-          const int s = it % kSStages;
-          ok = mbar_wait(&xform_bar[s], (it / kSStages) & 1u, status);
+          const int s = it % ST;
+          ok = mbar_wait(&xform_bar[s], (it / ST) & 1u, status);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t sA = smem_u32(smem + s * kSStageBytes), sB = sA + 32768;
+          const uint32_t sA = smem_u32(smem + s * SB), sB = sA + 32768;
 #pragma unroll
           for (int k16 = 0; k16 < 4; ++k16) {
             const uint64_t ad = a_mn ? smem_desc_mn128(sA + k16 * 2048) : smem_desc_k128(sA + k16 * 32);
             mma_bf16(tmem + buf * 256, ad, smem_desc_mn128(sB + k16 * 2048), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            if (BIG && n_hi) mma_bf16(tmem + 256, ad, smem_desc_mn128(sB + 4 * 8192 + k16 * 2048), idesc_hi, (kb > 0 || k16 > 0) ? 1u : 0u);
           }
           mma_commit(&empty_bar[s]);
         }
@@ -587,11 +635,11 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
       const bool has_e = pr->map_e != nullptr;
       const float c = pr->cptr ? *pr->cptr : 1.f;
       for (int kb = 0; kb < nkb; ++kb, ++it) {
-        const int s = it % kSStages;
-        ok = mbar_wait(&full_bar[s], (it / kSStages) & 1u, status);
+        const int s = it % ST;
+        ok = mbar_wait(&full_bar[s], (it / ST) & 1u, status);
         if (!ok) break;
         if (has_e) {
-          uint4* G = reinterpret_cast<uint4*>(smem + s * kSStageBytes);
+          uint4* G = reinterpret_cast<uint4*>(smem + s * SB);
           const uint4* E = G + 1024;
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
@@ -620,8 +668,8 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
       const bool row_ok = row < pr->M;
       float* __restrict__ crow = pr->C + (row_ok ? row : 0) * pr->ldc;
       const int r = pr->r, r_n = pr->r_n;
-      const uint32_t buf = si & 1u;
-      ok = mbar_wait<64>(&acc_full[buf], (si >> 1) & 1u, status);
+      const uint32_t buf = BIG ? 0u : (si & 1u);
+      ok = mbar_wait<64>(&acc_full[buf], (BIG ? si : (si >> 1)) & 1u, status);
       if (!ok) break;
       tc_fence_after_sync();
       for (int ch = 0; ch < r_n / 16; ++ch) {
@@ -643,11 +691,14 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
 }
 
 cudaError_t sketch_configure() {
-  return cudaFuncSetAttribute(sketch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSStages * kSStageBytes + 1024));
+  cudaError_t e = cudaFuncSetAttribute(sketch_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSStages * kSStageBytes + 1024));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(sketch_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSStages * kSStageBytes + 1024));
 }
-void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, unsigned* status, cudaStream_t st) {
+void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, int big, unsigned* status, cudaStream_t st) {
   const long long g = total_tiles < grid ? total_tiles : grid;
-  sketch_tma_kernel<<<(unsigned)g, kSThreads, kSStages * kSStageBytes + 1024, st>>>(probs, nprobs, total_tiles, status);
+  if (big) sketch_tma_kernel<true><<<(unsigned)g, kSThreads, kSStages * kSStageBytes + 1024, st>>>(probs, nprobs, total_tiles, status);
+  else sketch_tma_kernel<false><<<(unsigned)g, kSThreads, kSStages * kSStageBytes + 1024, st>>>(probs, nprobs, total_tiles, status);
 }
 
 }  // namespace lordo

@@ -124,7 +124,8 @@ def test_fast_mode_inner_steps(shape, form, variant):
     assert st["W"] < FAST_TOL * 3 * 0.01 / 0.02, st
 
 
-@pytest.mark.parametrize("shape", [(200, 136, 24), (320, 264, 72), (200, 520, 136), (704, 256, 256), (2048, 384, 256)])
+@pytest.mark.parametrize("shape", [(200, 136, 24), (320, 264, 72), (200, 520, 136), (704, 256, 256), (2048, 384, 256), (600, 520, 320),
+                                   (704, 640, 512)])
 @pytest.mark.parametrize("form,variant,ef", [(2, 0, True), (1, 1, True), (0, 0, False)])
 def test_fast_mode_inner_steps_bf16(shape, form, variant, ef):
     """bf16 storage of W, G, E: the TMA-fed kernels. Stored bf16 values add their own 2^-9 rounding."""
@@ -190,7 +191,7 @@ def test_fast_mode_full_loop_with_refresh():
 
 
 @pytest.mark.parametrize("variant,form,q", [(0, 2, 0), (0, 2, 2), (1, 1, 0), (1, 1, 2)])
-@pytest.mark.parametrize("shape", [(264, 200, 32), (520, 392, 136)])
+@pytest.mark.parametrize("shape", [(264, 200, 32), (520, 392, 136), (704, 520, 320)])
 def test_fast_mode_refresh_on_tensor_cores(variant, form, q, shape):
     """bf16 storage in fast mode: the sketch products S*Omega, S^T*P', S*Z run on tensor cores with
     bf16 operands, so the basis is not the oracle's vector by vector. What a range finder is for is
