@@ -65,19 +65,22 @@ def parse_args():
     ap.add_argument("--mode", default="fast", choices=["fast", "check"])
     ap.add_argument("--inner-steps", type=int, default=0, help="override H (non-standard; recorded in config)")
     ap.add_argument("--layers", type=int, default=0, help="keep only the first N decoder layers (profiling; recorded in config)")
+    ap.add_argument("--matrices", type=int, default=0, help="keep only the first N matrices (profiling / memory; recorded in config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
 
 
-def workload(name: str, H: int = 0, layers: int = 0):
+def workload(name: str, H: int = 0, layers: int = 0, matrices: int = 0):
     from paper_2602_04396_b200 import synth
     wl = synth.config(int(name[3:]))
     if H > 0:
         wl = synth.scaled(wl, H=H)
     if layers > 0 and len(wl.mats) >= 7 * layers:
         wl = synth.scaled(wl, mats=wl.mats[:7 * layers], name=f"{wl.name}_first{layers}layers")
+    if 0 < matrices < len(wl.mats):
+        wl = synth.scaled(wl, mats=wl.mats[:matrices], name=f"{wl.name}_first{matrices}matrices")
     return wl
 
 
@@ -239,7 +242,7 @@ def reference_main(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    wl = workload(args.workload, args.inner_steps, args.layers)
+    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
     sample, desc = oracle_sample(wl, args.variant)
     for _ in range(min(args.warmup, 1)):
         run_oracle_sample(sample, args.variant)
@@ -283,7 +286,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = workload(args.workload, args.inner_steps, args.layers)
+    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
     hp = HYPER[args.variant]
     H = wl.H
     seed = 1000 + rank  # every rank runs its own copy of the workload on its own inputs
