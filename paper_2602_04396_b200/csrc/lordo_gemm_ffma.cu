@@ -222,17 +222,19 @@ void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, in
 
 // ---------------------------------------------------------------------------------------------
 // Cholesky of the Gram matrix + inverse of the triangular factor, one block per problem.
-// Left-looking column Cholesky, fp64 accumulation, L kept in global memory (L2-resident).
+// Left-looking column Cholesky with fp64 accumulation. The factor is kept TRANSPOSED in global
+// memory (Lt[k][i] = L[i][k], L2-resident) so that thread i's sweep over its own row of L reads
+// consecutive addresses across the block; the row of the pivot column is staged in shared memory.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __restrict__ probs, unsigned* __restrict__ status) {
-  extern __shared__ float row_j[];  // r floats: row j of L (columns < j)
+  extern __shared__ float row_s[];  // r floats: row j of L (columns < j), later row i of L
   __shared__ float pivot_s;
   __shared__ float maxdiag_s;
   const CholProblem pb = probs[blockIdx.x];
   const int r = pb.r;
-  const float* A = pb.gram;
-  float* L = pb.lwork;
-  float* X = pb.rinv;
+  const float* __restrict__ A = pb.gram;
+  float* __restrict__ Lt = pb.lwork;
+  float* __restrict__ X = pb.rinv;
   const int t = threadIdx.x, nt = blockDim.x;
 
   if (t == 0) {
@@ -249,13 +251,23 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
   const float abs_floor = maxdiag_s > 0.f ? maxdiag_s * 1e-12f : 1.f;
 
   for (int j = 0; j < r; ++j) {
-    for (int k = t; k < j; k += nt) row_j[k] = L[(long long)j * r + k];
+    for (int k = t; k < j; k += nt) row_s[k] = Lt[(long long)k * r + j];  // L[j][k]
     __syncthreads();
-    // s_i = A[i][j] - sum_{k<j} L[i][k] L[j][k] for i >= j
+    // s_i = A[i][j] - sum_{k<j} L[i][k] L[j][k] for i >= j   (A is symmetric: row j is read)
     for (int i = j + t; i < r; i += nt) {
-      const float* Li = L + (long long)i * r;
-      double s = (double)A[(long long)i * r + j];
-      for (int k = 0; k < j; ++k) s -= (double)Li[k] * (double)row_j[k];
+      const float* __restrict__ col = Lt + i;
+      double s0 = (double)A[(long long)j * r + i], s1 = 0.0, s2 = 0.0, s3 = 0.0;
+      int k = 0;
+      for (; k + 4 <= j; k += 4) {
+        const float l0 = col[(long long)k * r], l1 = col[(long long)(k + 1) * r], l2 = col[(long long)(k + 2) * r],
+                    l3 = col[(long long)(k + 3) * r];
+        s0 -= (double)l0 * (double)row_s[k];
+        s1 -= (double)l1 * (double)row_s[k + 1];
+        s2 -= (double)l2 * (double)row_s[k + 2];
+        s3 -= (double)l3 * (double)row_s[k + 3];
+      }
+      for (; k < j; ++k) s0 -= (double)col[(long long)k * r] * (double)row_s[k];
+      const double s = (s0 + s1) + (s2 + s3);
       if (i == j) {
         float d = (float)s;
         const float floor_pivot = fmaxf(kBreakdown * A[(long long)j * r + j], abs_floor);
@@ -265,36 +277,47 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
         }
         pivot_s = sqrtf(d);
       }
-      L[(long long)i * r + j] = (float)s;  // unscaled for now
+      Lt[(long long)j * r + i] = (float)s;  // unscaled for now; written and re-read by the same thread
     }
     __syncthreads();
     const float piv = pivot_s;
     for (int i = j + t; i < r; i += nt) {
-      float* Lij = L + (long long)i * r + j;
-      *Lij = (i == j) ? piv : (*Lij / piv);
+      float* Lji = Lt + (long long)j * r + i;
+      *Lji = (i == j) ? piv : (*Lji / piv);
     }
     __syncthreads();
   }
 
-  // Linv: column c solved by thread c (forward substitution), kept transposed-free in X as
-  // X[i][c] = Linv[i][c]; afterwards rinv = Linv^T is produced in place through lwork.
-  for (int c = t; c < r; c += nt) {
-    for (int i = 0; i < c; ++i) X[(long long)i * r + c] = 0.f;
-    X[(long long)c * r + c] = 1.f / L[(long long)c * r + c];
-    for (int i = c + 1; i < r; ++i) {
-      const float* Li = L + (long long)i * r;
-      double s = 0.0;
-      for (int k = c; k < i; ++k) s += (double)Li[k] * (double)X[(long long)k * r + c];
-      X[(long long)i * r + c] = (float)(-s / (double)Li[i]);
+  // X = L^-1 (lower triangular), column c by thread c: X[i][c] = -(sum_{k=c}^{i-1} L[i][k] X[k][c]) / L[i][i].
+  // Row i of L is staged in shared memory for everybody; X[k][c] is read along rows (consecutive c).
+  for (int c = t; c < r; c += nt)
+    for (int i = 0; i < r; ++i)
+      if (i < c) X[(long long)i * r + c] = 0.f;
+  for (int i = 0; i < r; ++i) {
+    for (int k = t; k <= i; k += nt) row_s[k] = Lt[(long long)k * r + i];  // L[i][k]
+    __syncthreads();
+    for (int c = t; c <= i; c += nt) {
+      if (c == i) {
+        X[(long long)i * r + c] = 1.f / row_s[i];
+      } else {
+        double s0 = 0.0, s1 = 0.0;
+        int k = c;
+        for (; k + 2 <= i; k += 2) {
+          s0 += (double)row_s[k] * (double)X[(long long)k * r + c];
+          s1 += (double)row_s[k + 1] * (double)X[(long long)(k + 1) * r + c];
+        }
+        for (; k < i; ++k) s0 += (double)row_s[k] * (double)X[(long long)k * r + c];
+        X[(long long)i * r + c] = (float)(-(s0 + s1) / (double)row_s[i]);
+      }
     }
+    __syncthreads();
   }
-  __syncthreads();
-  // R^-1 = (L^-1)^T : transpose X through L's storage
-  for (long long e = t; e < (long long)r * r; e += nt) L[e] = X[e];
+  // R^-1 = (L^-1)^T : transpose X through Lt's storage (the factor is no longer needed)
+  for (long long e = t; e < (long long)r * r; e += nt) Lt[e] = X[e];
   __syncthreads();
   for (long long e = t; e < (long long)r * r; e += nt) {
     const int i = (int)(e / r), c = (int)(e - (long long)i * r);
-    X[e] = L[(long long)c * r + i];
+    X[e] = Lt[(long long)c * r + i];
   }
 }
 
