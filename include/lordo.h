@@ -165,6 +165,16 @@ LORDO_API int lordo_refresh_subspace(lordo_ctx* ctx, const void* const* G_or_nul
  * LORDO_ERR_NUMERIC if it is non-zero, else LORDO_OK. */
 LORDO_API int lordo_poll_status(lordo_ctx* ctx, void* stream, uint32_t* flags);
 
+/*
+ * Diagnostics (Sec. "Experimental Framework", Metrics). mssv_dev: one float per projection matrix
+ * (n_mats for Global, n_mats * K for Local, matrix-major), the mean squared singular value
+ * (1/r) sum_i sigma_i^2 of Rot = P_new^T P_old of the LAST lordo_refresh_subspace (1 = the subspace
+ * did not move, 0 = it moved to an orthogonal one); valid until the next refresh overwrites the
+ * rotation matrices; LORDO_ERR_STATE before the first refresh. e_norm_dev: [n_mats][K] floats,
+ * ||E||_F of every error buffer. Either pointer may be NULL. Device pointers, caller-owned.
+ */
+LORDO_API int lordo_diagnostics(lordo_ctx* ctx, float* mssv_dev, float* e_norm_dev, void* stream);
+
 /* Clears the sticky device flag word (after the caller has dealt with what lordo_poll_status reported). */
 LORDO_API int lordo_clear_status(lordo_ctx* ctx, void* stream);
 

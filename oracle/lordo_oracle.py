@@ -194,6 +194,13 @@ def rotate_moments(u: np.ndarray, v: np.ndarray, P_new: np.ndarray, P_old: np.nd
     return u_new, v_new
 
 
+def mssv(P_new: np.ndarray, P_old: np.ndarray) -> float:
+    """Sec. "Experimental Framework", Metrics: mean squared singular value of the rotated basis
+    matrix R = Q_t^T Q_{t-1}, MSSV = (1/r) sum_i sigma_i^2, written out from the singular values."""
+    sigma = np.linalg.svd(np.asarray(P_new, dtype=np.float64).T @ np.asarray(P_old, dtype=np.float64), compute_uv=False)
+    return float(np.sum(sigma ** 2) / len(sigma))
+
+
 def clip_coefficients(G: Sequence[np.ndarray], rho: float, scope: int = 0) -> np.ndarray:
     """R8 / Algorithm 1 line "clip": coefficient per worker (scope 0: one norm over all matrices of
     the worker; scope 1: one per matrix). G[i] has shape [K, m_i, n_i]. Returns [n_mats, K]."""
@@ -245,6 +252,7 @@ class LordoOracle:
         self.refreshes = 0
         self.W, self.E, self.P, self.u, self.v, self.X0, self.B, self.Delta = [], [], [], [], [], [], [], []
         self.last_clip = None
+        self.last_mssv = None  # [n_mats][1 or K] MSSV of the last refresh that rotated (diagnostic)
         for i, (m, n, r) in enumerate(c.mats):
             w0 = store(W0[i], c.w_dtype)
             self.W.append(np.repeat(w0[None], c.K, axis=0))  # all workers start equal (Alg. 1 Require)
@@ -328,10 +336,12 @@ class LordoOracle:
         if c.variant == LOCAL:
             assert G is not None
             coef = clip_coefficients(G, c.clip_rho, c.clip_scope)
+        diag = [[] for _ in c.mats]
         for i, (m, n, r) in enumerate(c.mats):
             if c.variant == GLOBAL:
                 Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, 0, n, r)
                 P_new = store(compute_projection(self.Delta[i], Om, c.power_iters), c.state_dtype)
+                diag[i].append(mssv(P_new, self.P[i]))
                 if self.s > 0:
                     for k in range(c.K):
                         un, vn = rotate_moments(self.u[i][k], self.v[i][k], P_new, self.P[i], beta1, c.beta2, self.s)
@@ -345,11 +355,13 @@ class LordoOracle:
                         S = S + self.E[i][k]
                     Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, n, r)
                     P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
+                    diag[i].append(mssv(P_new, self.P[i][k]))
                     if self.s > 0:
                         un, vn = rotate_moments(self.u[i][k], self.v[i][k], P_new, self.P[i][k], beta1, c.beta2, self.s)
                         self.u[i][k] = store(un, c.state_dtype)
                         self.v[i][k] = store(vn, c.state_dtype)
                     self.P[i][k] = P_new
+        self.last_mssv = diag
         self.refreshes += 1
 
 

@@ -117,6 +117,8 @@ struct lordo_ctx {
   std::vector<RandProblem> h_rands;
   std::vector<CopyProblem> h_copies;
   std::vector<SkProblem> h_sks;
+  std::vector<DiagProblem> h_diag;  // one per rotation matrix, ordered by matrix then batch entry
+  DiagProblem* d_diag = nullptr;
   std::vector<ConvProblem> h_convs;
   struct SketchBufs { __nv_bfloat16 *om16 = nullptr, *pn16 = nullptr, *zq16 = nullptr; };
   std::vector<SketchBufs> h_skbufs;  // per matrix: bf16 right-hand sides of the sketch products (refresh scratch)
@@ -360,7 +362,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
 
   // ---------------- launch plans ----------------
   std::vector<GemmProblem>& P = c->h_probs;
-  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear();
+  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear(); c->h_diag.clear();
   c->h_skbufs.assign(n_mats, lordo_ctx::SketchBufs());
   const bool tc_sketch = c->tc && c->tma;  // sketch products of the refresh on tensor cores
   auto gemm_prob = [&](int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
@@ -587,8 +589,13 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         }
         cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
       }
-      {  // Rot = P'^T P
-        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_ROTATE, 1, 0, 0);
+      for (int b = 0; b < nb; ++b) {
+        DiagProblem dp;
+        dp.rot = rot + (long long)b * r * r; dp.r = r; dp.pad = 0;
+        c->h_diag.push_back(dp);
+      }
+      {  // Rot = P'^T P (always formed: it also carries the MSSV diagnostic)
+        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
         for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob(r, r, (int)m, plain(Pn + (long long)b * m * r, r), plain(md.P ? md.P + b * md.p_stride : nullptr, r), nullptr, store_epi(rot + (long long)b * r * r, r)));
       }
       {  // u', v' (into the transient g^ / U~ areas), then back
@@ -623,6 +630,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   c->d_copies = cv.take<CopyProblem>(c->h_copies.size() + 1);
   c->d_sks = cv.take<SkProblem>(c->h_sks.size() + 1);
   c->d_convs = cv.take<ConvProblem>(c->h_convs.size() + 1);
+  c->d_diag = cv.take<DiagProblem>(c->h_diag.size() + 1);
 
   c->last_G.assign(n_mats, nullptr);
   return (cv.off + 255) & ~size_t(255);
@@ -816,6 +824,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   if (!c->h_rands.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_rands, c->h_rands.data(), sizeof(RandProblem) * c->h_rands.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_copies.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_copies, c->h_copies.data(), sizeof(CopyProblem) * c->h_copies.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_sks.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_sks, c->h_sks.data(), sizeof(SkProblem) * c->h_sks.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_diag.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_diag, c->h_diag.data(), sizeof(DiagProblem) * c->h_diag.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_convs.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_convs, c->h_convs.data(), sizeof(ConvProblem) * c->h_convs.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
   if (c->tc) {
@@ -1087,6 +1096,23 @@ int lordo_poll_status(lordo_ctx* c, void* stream, uint32_t* flags) {
   if (flags) *flags = *c->h_status;
   if (*c->h_status) return fail(c, LORDO_ERR_NUMERIC, "device flag word is non-zero");
   return LORDO_OK;
+}
+
+int lordo_diagnostics(lordo_ctx* c, float* mssv_dev, float* e_norm_dev, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  if (!mssv_dev && !e_norm_dev) return fail(c, LORDO_ERR_INVALID_ARG, "nothing requested");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (mssv_dev) {
+    if (c->refreshes == 0) return fail(c, LORDO_ERR_STATE, "no refresh has run yet: there is no rotation matrix");
+    launch_mssv(c->d_diag, (int)c->h_diag.size(), mssv_dev, st);
+    c->launches += 1;
+  }
+  if (e_norm_dev) {
+    if (!c->cfg.error_feedback) return fail(c, LORDO_ERR_STATE, "error feedback is off: there is no error buffer");
+    launch_error_norms(c->d_mats, c->n_mats, c->K, c->cfg.e_dtype, e_norm_dev, st);
+    c->launches += 1;
+  }
+  return check_launch(c, "diagnostics");
 }
 
 int lordo_selftest_wait_timeout(lordo_ctx* c, void* stream) {

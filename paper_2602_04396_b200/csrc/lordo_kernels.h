@@ -129,6 +129,15 @@ void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips
 
 void launch_selftest_wait(unsigned* status, cudaStream_t st);
 
+// Diagnostics: MSSV = ||Rot||_F^2 / r of every rotation matrix of the last refresh, and ||E||_F per
+// (matrix, worker).
+struct DiagProblem {
+  const float* rot;  // r x r
+  int r, pad;
+};
+void launch_mssv(const DiagProblem* probs, int nprobs, float* out, cudaStream_t st);
+void launch_error_norms(const MatDev* mats, int n_mats, int K, int e_dt, float* out, cudaStream_t st);
+
 // Cholesky factor of a batch of r x r Gram matrices and the inverse of its transpose:
 // gram = R^T R (R upper triangular, positive diagonal); rinv = R^-1, row-major, zeros below the
 // diagonal. lwork: r*r floats per problem. Strides in floats between batch entries.

@@ -305,9 +305,50 @@ __global__ void __launch_bounds__(256) copy_grouped_kernel(const CopyProblem* __
     if (c + i < pb.chunks) dst[c + i] = v[i];
 }
 
+// Mean squared singular value of Rot = P'^T P (the paper's MSSV metric): the sum of the squared
+// singular values of a matrix is its squared Frobenius norm. One block per rotation matrix.
+__global__ void __launch_bounds__(256) mssv_kernel(const DiagProblem* __restrict__ probs, float* __restrict__ out) {
+  const DiagProblem pb = probs[blockIdx.x];
+  const long long count = (long long)pb.r * pb.r;
+  double a = 0.0;
+  for (long long e = threadIdx.x; e < count; e += 256) { const double x = (double)pb.rot[e]; a += x * x; }
+  __shared__ double red[256];
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[blockIdx.x] = (float)(red[0] / (double)pb.r);
+}
+
+// ||E||_F of one (matrix, worker) per block.
+__global__ void __launch_bounds__(256) error_norms_kernel(const MatDev* __restrict__ mats, int K, int e_dt, float* __restrict__ out) {
+  const int i = blockIdx.x, k = blockIdx.y;
+  const long long elems = mats[i].m * mats[i].n;
+  const void* E = mats[i].E;
+  double a = 0.0;
+  for (long long e = 4ll * threadIdx.x; e < elems; e += 4ll * 256) {  // elems is a multiple of 8
+    const float4 x = load4(E, e_dt, (long long)k * elems + e);
+    a += (double)(x.x * x.x + x.y * x.y) + (double)(x.z * x.z + x.w * x.w);
+  }
+  __shared__ double red[256];
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[(long long)i * K + k] = (float)sqrt(red[0]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // host launchers
 // ---------------------------------------------------------------------------------------------
+void launch_mssv(const DiagProblem* probs, int nprobs, float* out, cudaStream_t st) { mssv_kernel<<<nprobs, 256, 0, st>>>(probs, out); }
+void launch_error_norms(const MatDev* mats, int n_mats, int K, int e_dt, float* out, cudaStream_t st) {
+  error_norms_kernel<<<dim3(n_mats, K), 256, 0, st>>>(mats, K, e_dt, out);
+}
 void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long total_blocks, unsigned long long seed, long long index,
                                 cudaStream_t st) {
   fill_random_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs, seed, index);

@@ -250,6 +250,23 @@ def test_rank_deficient_sketch_raises_flag_and_stays_finite():
     assert bool(torch.isfinite(opt.P[0]).all())
 
 
+@pytest.mark.parametrize("variant", [0, 1])
+def test_diagnostics_mssv_and_error_norms(variant):
+    """MSSV of the last refresh's rotation matrices and ||E||_F, against the oracle's definitions."""
+    wl = synth.Workload("diag", ((264, 200, 32), (136, 312, 16)), K=2, H=2, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0)
+    spec = RunSpec(wl, variant=variant, form=2 if variant == 0 else 1, lr=0.01)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    mssv, en = opt.diagnostics()
+    want = np.array([x for per in orc.last_mssv for x in per])
+    assert np.abs(mssv.cpu().numpy() - want).max() < 1e-4, (mssv, want)
+    assert 0.0 <= want.min() and want.max() <= 1.0 + 1e-9
+    want_e = np.array([[np.linalg.norm(orc.E[i][k]) for k in range(wl.K)] for i in range(len(wl.mats))])
+    assert np.abs(en.cpu().numpy() - want_e).max() < 1e-4 * want_e.max()
+    fresh = hz.make_gpu(spec)
+    with pytest.raises(Exception):
+        fresh.diagnostics()  # no refresh yet
+
+
 def test_bounded_wait_reports_timeout_and_context_stays_usable():
     """A device-side wait that nothing completes gives up after its limit, raises the timeout flag and
     lets the kernel end; the same context then runs a correct step."""

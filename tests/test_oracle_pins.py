@@ -485,3 +485,21 @@ def test_golden_files_match_the_oracle():
     for variant, form, name in ((0, 2, "global_fullqhm"), (1, 1, "local_lowqhm")):
         stored = np.loadtxt(os.path.join(here, f"tiny_8x8_{name}_weights.txt"))
         np.testing.assert_allclose(mg.tiny_run(variant, form), stored, rtol=1e-12, atol=1e-15)
+
+
+# ---------------------------------------------------------------------------------------------
+# diagnostics: MSSV of the rotated basis matrix (Sec. "Experimental Framework", Metrics)
+# ---------------------------------------------------------------------------------------------
+def test_mssv_closed_forms():
+    rng = np.random.default_rng(3)
+    m, r = 40, 6
+    Q, _ = np.linalg.qr(rng.standard_normal((m, 2 * r)))
+    A, B = Q[:, :r], Q[:, r:]
+    assert abs(lo.mssv(A, A) - 1.0) < 1e-12                      # same subspace: every singular value is 1
+    assert abs(lo.mssv(A @ np.linalg.qr(rng.standard_normal((r, r)))[0], A) - 1.0) < 1e-12  # any basis of it
+    assert lo.mssv(B, A) < 1e-24                                  # orthogonal subspaces: all zero
+    C = np.concatenate([A[:, :3], B[:, :3]], axis=1)              # shares 3 of 6 directions
+    assert abs(lo.mssv(C, A) - 0.5) < 1e-12
+    # equals ||R||_F^2 / r, the form a kernel would use
+    R = C.T @ A
+    assert abs(lo.mssv(C, A) - np.sum(R * R) / r) < 1e-12
