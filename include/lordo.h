@@ -100,7 +100,9 @@ typedef struct {
   uint64_t seed;           /* seed of the counter-based generator for P_0 and the sketches */
   int32_t check_mode;      /* 1: every contraction in fp32 FMA arithmetic (parity mode);
                               0: bf16 tensor-core contractions where operands are bf16 */
-  int32_t reserved;
+  int32_t warm_start;      /* 0: every refresh starts from a fresh random sketch; 1: block power iteration
+                              started from the current P (max(power_iters, 1) iterations, no sketch), the
+                              cheaper estimator the paper names as an alternative ComputeProjection */
 } lordo_config;
 
 /* Host tables of device pointers, one entry per matrix. fp32 unless stated. */

@@ -180,6 +180,18 @@ def compute_projection(S: np.ndarray, Omega: np.ndarray, power_iters: int) -> np
     return Pn
 
 
+def compute_projection_warm(S: np.ndarray, P_old: np.ndarray, iters: int) -> np.ndarray:
+    """Block power iteration started from the previous basis (the cheaper ComputeProjection the paper
+    names, Sec. 2 "PowerSGD / block power iteration" and App. "Limitations"): `iters` >= 1 times
+    Z = qr(S^T P'), P' = qr(S Z), beginning with P' = P_old. No random sketch is drawn."""
+    S = np.asarray(S, dtype=np.float64)
+    Pn = np.asarray(P_old, dtype=np.float64)
+    for _ in range(max(int(iters), 1)):
+        Z = householder_qr_q(S.T @ Pn)
+        Pn = householder_qr_q(S @ Z)
+    return Pn
+
+
 def rotate_moments(u: np.ndarray, v: np.ndarray, P_new: np.ndarray, P_old: np.ndarray, beta1: float,
                    beta2: float, s: int) -> Tuple[np.ndarray, np.ndarray]:
     """Algorithm 1, moment-rotation lines (same in Algorithm 2). Rot = P_new^T P_old (r x r);
@@ -240,6 +252,7 @@ class OracleConfig:
     w_dtype: str = "f32"
     e_dtype: str = "f32"
     state_dtype: str = "f32"  # u, v, P, X0, B, Delta
+    warm_start: bool = False   # refresh by block power iteration from the current P (no sketch)
 
 
 class LordoOracle:
@@ -339,8 +352,11 @@ class LordoOracle:
         diag = [[] for _ in c.mats]
         for i, (m, n, r) in enumerate(c.mats):
             if c.variant == GLOBAL:
-                Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, 0, n, r)
-                P_new = store(compute_projection(self.Delta[i], Om, c.power_iters), c.state_dtype)
+                if c.warm_start:
+                    P_new = store(compute_projection_warm(self.Delta[i], self.P[i], c.power_iters), c.state_dtype)
+                else:
+                    Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, 0, n, r)
+                    P_new = store(compute_projection(self.Delta[i], Om, c.power_iters), c.state_dtype)
                 diag[i].append(mssv(P_new, self.P[i]))
                 if self.s > 0:
                     for k in range(c.K):
@@ -353,8 +369,11 @@ class LordoOracle:
                     S = coef[i, k] * np.asarray(G[i][k], dtype=np.float64)
                     if c.error_feedback:
                         S = S + self.E[i][k]
-                    Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, n, r)
-                    P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
+                    if c.warm_start:
+                        P_new = store(compute_projection_warm(S, self.P[i][k], c.power_iters), c.state_dtype)
+                    else:
+                        Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, n, r)
+                        P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
                     diag[i].append(mssv(P_new, self.P[i][k]))
                     if self.s > 0:
                         un, vn = rotate_moments(self.u[i][k], self.v[i][k], P_new, self.P[i][k], beta1, c.beta2, self.s)

@@ -235,7 +235,8 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   const int n_mats = cfg.n_mats, K = cfg.K;
   const bool real = ws != nullptr && buf != nullptr;
   const bool local = cfg.variant == LORDO_LOCAL;
-  const int q = cfg.power_iters;
+  const bool warm = cfg.warm_start != 0;  // start the subspace iteration from the previous P instead of a random sketch
+  const int q = (warm && cfg.power_iters < 1) ? 1 : cfg.power_iters;
   Carver cv(ws);
 
   c->d_mats = cv.take<MatDev>(n_mats);
@@ -553,24 +554,29 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         }
         return A;
       };
-      {
-        SlotBuilder::Slot& f = R.next(ST_RANDOM, PH_SUBSPACE);
-        for (int b = 0; b < nb; ++b) {
-          RandProblem rp;
-          rp.out = tc_sketch ? nullptr : Om + (long long)b * n * r;
-          rp.out16 = tc_sketch ? om16 + (long long)b * n * r : nullptr;
-          rp.count = n * r; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
-          f.rn.push_back(rp);
-        }
-      }
-      if (tc_sketch) {  // Y = S Omega
-        if (!local) convert(R, md.Delta, md.Delta16, (size_t)m * n);  // bf16 copy of the Global signal
-        sketch(R, 0, (c->d_maps + i)->om16, Ya, m * r, m, n);
+      if (warm) {  // block power iteration warm-started from the current basis
+        if (tc_sketch && !local) convert(R, md.Delta, md.Delta16, (size_t)m * n);
+        add_copy(R, PH_SUBSPACE, Pn, md.P, (size_t)nb * m * r * sizeof(float));
       } else {
-        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
-        for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
+        {
+          SlotBuilder::Slot& f = R.next(ST_RANDOM, PH_SUBSPACE);
+          for (int b = 0; b < nb; ++b) {
+            RandProblem rp;
+            rp.out = tc_sketch ? nullptr : Om + (long long)b * n * r;
+            rp.out16 = tc_sketch ? om16 + (long long)b * n * r : nullptr;
+            rp.count = n * r; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
+            f.rn.push_back(rp);
+          }
+        }
+        if (tc_sketch) {  // Y = S Omega
+          if (!local) convert(R, md.Delta, md.Delta16, (size_t)m * n);  // bf16 copy of the Global signal
+          sketch(R, 0, (c->d_maps + i)->om16, Ya, m * r, m, n);
+        } else {
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
+        }
+        cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
       }
-      cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
       for (int it = 0; it < q; ++it) {
         if (tc_sketch) {  // Z = S^T P'
           convert(R, Pn, pn16, (size_t)nb * m * r);

@@ -240,6 +240,27 @@ def test_refresh_and_rotation(variant, q):
     assert opt.poll_status() == 0
 
 
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("q", [0, 2])
+def test_refresh_warm_started_power_iteration(variant, q):
+    """The alternative ComputeProjection: block power iteration started from the current basis."""
+    wl = _small(m=264, n=200, r=32, K=2, H=2, rounds=3, grad="lowrank", power_iters=q, signal_rank=8, clip_rho=30.0)
+    spec = RunSpec(wl, variant=variant, form=2, lr=0.01, warm_start=True)
+    opt, orc, worst = hz.run_lockstep_refresh(spec)
+    assert worst["P_orth"] < 1e-5 and worst["P_angle"] < ANGLE_TOL and worst["u"] < 1e-3 and worst["v"] < 1e-3, worst
+    assert abs(worst["energy"] - 1.0) < 1e-4, worst
+
+
+def test_refresh_warm_started_fast_mode_bf16():
+    wl = _small(m=520, n=392, r=136, K=2, H=2, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0, power_iters=1,
+                w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    for variant, form in ((0, 2), (1, 1)):
+        spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0, eps=0.05, warm_start=True)
+        opt, orc, worst = hz.run_lockstep_refresh(spec)
+        assert opt.poll_status() == 0
+        assert worst["P_orth"] < 1e-5 and abs(worst["energy"] - 1.0) < 1e-2, worst
+
+
 def test_rank_deficient_sketch_raises_flag_and_stays_finite():
     wl = _small(m=128, n=96, r=16, K=1, H=1, rounds=1)
     opt = hz.make_gpu(RunSpec(wl, variant=1))

@@ -503,3 +503,34 @@ def test_mssv_closed_forms():
     # equals ||R||_F^2 / r, the form a kernel would use
     R = C.T @ A
     assert abs(lo.mssv(C, A) - np.sum(R * R) / r) < 1e-12
+
+
+# ---------------------------------------------------------------------------------------------
+# warm-started block power iteration (the alternative ComputeProjection)
+# ---------------------------------------------------------------------------------------------
+def test_warm_started_power_iteration_pins():
+    rng = np.random.default_rng(9)
+    m, n, r = 60, 48, 6
+    # exact rank r: one iteration from a generic orthonormal start lands on the column space of S
+    S = rng.standard_normal((m, r)) @ rng.standard_normal((r, n))
+    P0 = np.linalg.qr(rng.standard_normal((m, r)))[0]
+    P1 = lo.compute_projection_warm(S, P0, 1)
+    assert np.abs(P1.T @ P1 - np.eye(r)).max() < 1e-12
+    assert np.linalg.norm(S - P1 @ (P1.T @ S)) / np.linalg.norm(S) < 1e-10
+    # a start that already spans the dominant subspace stays there (fixed point up to the basis)
+    U, sv, Vt = np.linalg.svd(rng.standard_normal((m, n)), full_matrices=False)
+    sv = np.concatenate([np.linspace(10, 5, r), 0.05 * np.ones(len(sv) - r)])
+    S = (U * sv) @ Vt
+    P2 = lo.compute_projection_warm(S, U[:, :r], 1)
+    assert np.linalg.norm(P2 - U[:, :r] @ (U[:, :r].T @ P2), 2) < 1e-10
+    # from a generic start the angle to the SVD subspace shrinks like (sigma_{r+1}/sigma_r)^2 per iteration
+    angle = lambda P: np.arcsin(min(1.0, np.linalg.norm(P - U[:, :r] @ (U[:, :r].T @ P), 2)))
+    a1, a2, a3 = (angle(lo.compute_projection_warm(S, P0, it)) for it in (1, 2, 3))
+    assert a2 < a1 * 1e-3 and a3 <= a2 and a1 < 0.2
+    # the oracle's refresh uses it when asked to, and draws no sketch
+    cfg = lo.OracleConfig(mats=((m, n, r),), K=1, H=1, variant=lo.GLOBAL, warm_start=True, state_dtype="f64", w_dtype="f64", e_dtype="f64")
+    orc = lo.LordoOracle(cfg, [np.zeros((m, n))])
+    orc.Delta[0] = S
+    P_before = orc.P[0].copy()
+    orc.refresh_subspace(None)
+    assert np.allclose(orc.P[0], lo.compute_projection_warm(S, P_before, 0))
