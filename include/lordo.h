@@ -154,6 +154,14 @@ LORDO_API int lordo_inner_step_host(lordo_ctx* ctx, const void* const* G_host, v
 LORDO_API int lordo_outer_step(lordo_ctx* ctx, void* stream);
 
 /*
+ * Algorithm 1, lines "if t mod K_u = 0: u <- E_m[u]" and "if t mod K_v = 0: v <- E_m[v]" on their
+ * own, for schedules whose state-synchronisation intervals K_u, K_v differ from the model interval
+ * K_x = H (set sync_u = sync_v = 0 in the configuration and call this at the steps of your choice).
+ * May be called between any two inner steps.
+ */
+LORDO_API int lordo_sync_states(lordo_ctx* ctx, int sync_u, int sync_v, void* stream);
+
+/*
  * ComputeProjection and the moment-rotation lines of Algorithm 1 (Global: signal = Delta, G must
  * be NULL) or Algorithm 2 (Local: signal = c_k G_k + E_k per worker, G as for lordo_inner_step).
  * Range finder: Y = S Omega with an n x r integer sketch from `seed`, thin QR, `power_iters`

@@ -324,6 +324,15 @@ class LordoOracle:
                     raise ValueError(form)
                 self.W[i][k] = store(self.W[i][k] - lr * upd, c.w_dtype)
 
+    # -- Algorithm 1, the two state-synchronisation lines on their own (K_u, K_v != K_x) ------------
+    def sync_states(self, sync_u: bool, sync_v: bool) -> None:
+        c = self.cfg
+        for i in range(len(c.mats)):
+            if sync_u:
+                self.u[i][:] = store(self.u[i].mean(axis=0), c.state_dtype)[None]
+            if sync_v:
+                self.v[i][:] = store(self.v[i].mean(axis=0), c.state_dtype)[None]
+
     # -- Algorithm 1, the synchronisation block ---------------------------------------------------
     def outer_step(self) -> None:
         c = self.cfg

@@ -1052,6 +1052,19 @@ int lordo_outer_step(lordo_ctx* c, void* stream) {
   return LORDO_OK;
 }
 
+int lordo_sync_states(lordo_ctx* c, int sync_u, int sync_v, void* stream) {
+  if (!c) return LORDO_ERR_INVALID_ARG;
+  const int which = (sync_u ? 1 : 0) | (sync_v ? 2 : 0);
+  if (!which) return LORDO_OK;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  {
+    ProfScope ps(c, st, PC_OUTER_STATES);
+    launch_outer_states(c->d_mats, c->d_sblk_start, c->n_mats, c->total_sblks, c->K, which, st);
+  }
+  c->launches += 1;
+  return check_launch(c, "sync_states");
+}
+
 int lordo_refresh_subspace(lordo_ctx* c, const void* const* G, float beta1, void* stream) {
   if (!c) return LORDO_ERR_INVALID_ARG;
   const bool local = c->cfg.variant == LORDO_LOCAL;

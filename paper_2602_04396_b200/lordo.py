@@ -25,7 +25,7 @@ EXPORTS = [
     "lordo_refresh_subspace", "lordo_poll_status", "lordo_get_counters", "lordo_set_counters",
     "lordo_clip_coefficients", "lordo_launch_count", "lordo_last_error", "lordo_status_string", "lordo_destroy",
     "lordo_fill_random", "lordo_profile_enable", "lordo_profile_read", "lordo_clip_coefficient_static",
-    "lordo_clip_coefficient_static_max_count", "lordo_clear_status", "lordo_selftest_wait_timeout", "lordo_diagnostics",
+    "lordo_clip_coefficient_static_max_count", "lordo_clear_status", "lordo_selftest_wait_timeout", "lordo_diagnostics", "lordo_sync_states",
 ]
 
 
@@ -87,6 +87,7 @@ def load_library() -> C.CDLL:
     lib.lordo_profile_enable.argtypes = [vp, i32]
     lib.lordo_profile_read.argtypes = [vp, vp, C.POINTER(f32)]
     lib.lordo_clear_status.argtypes = [vp, vp]
+    lib.lordo_sync_states.argtypes = [vp, i32, i32, vp]
     lib.lordo_diagnostics.argtypes = [vp, vp, vp, vp]
     lib.lordo_selftest_wait_timeout.argtypes = [vp, vp]
     lib.lordo_clip_coefficient_static.argtypes = [vp, i32, i64, f32, vp, vp]
@@ -268,6 +269,9 @@ class Lordo:
         self._check(self.lib.lordo_diagnostics(self._ctx, C.c_void_p(mssv.data_ptr()), C.c_void_p(en.data_ptr()) if en is not None else None,
                                                _stream_handle(stream)), "lordo_diagnostics")
         return mssv, en
+
+    def sync_states(self, sync_u: bool, sync_v: bool, stream=None):
+        self._check(self.lib.lordo_sync_states(self._ctx, int(sync_u), int(sync_v), _stream_handle(stream)), "lordo_sync_states")
 
     def clear_status(self, stream=None):
         self._check(self.lib.lordo_clear_status(self._ctx, _stream_handle(stream)), "lordo_clear_status")

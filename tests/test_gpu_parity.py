@@ -226,6 +226,29 @@ def test_outer_step(outer, wdt):
     assert float((W - W[0:1]).abs().max()) == 0.0  # all replicas hold the broadcast model
 
 
+def test_decoupled_state_sync_intervals():
+    """K_u = 1, K_v = 2, K_x = H = 4: the state averages run on their own schedule between inner steps."""
+    wl = _small(m=136, n=200, r=16, K=3, H=4, rounds=2, clip_rho=30.0)
+    spec = RunSpec(wl, refresh=False, sync_u=False, sync_v=False, lr=0.01, outer=1)
+    opt, orc = hz.make_gpu(spec), hz.make_oracle(spec)
+    t = 0
+    for rnd in range(2):
+        for h in range(4):
+            G = synth.gradients(wl, 0, rnd, h)
+            opt.inner_step(hz.device_grads(wl, G), 0.01, 0.9, 0.9, 1)
+            orc.inner_step(G, hz.f32(0.01), hz.f32(0.9), hz.f32(0.9), 1)
+            t += 1
+            opt.sync_states(True, t % 2 == 0)
+            orc.sync_states(True, t % 2 == 0)
+        opt.outer_step()
+        orc.outer_step()
+    torch.cuda.synchronize()
+    st = hz.compare_states(opt, orc)
+    assert st["W"] < W_TOL and st["u"] < 1e-4 and st["v"] < 1e-4 and st["X0"] < W_TOL, st
+    u = opt.u[0]
+    assert float((u - u[0:1]).abs().max()) == 0.0  # u was averaged after the last step
+
+
 # ------------------------------------------------------------------ refresh
 
 @pytest.mark.parametrize("variant", [0, 1])

@@ -534,3 +534,15 @@ def test_warm_started_power_iteration_pins():
     P_before = orc.P[0].copy()
     orc.refresh_subspace(None)
     assert np.allclose(orc.P[0], lo.compute_projection_warm(S, P_before, 0))
+
+
+def test_sync_states_is_the_mean_over_workers():
+    cfg = lo.OracleConfig(mats=((8, 8, 4),), K=3, H=2, state_dtype="f64", w_dtype="f64", e_dtype="f64")
+    orc = lo.LordoOracle(cfg, [np.zeros((8, 8))])
+    rng = np.random.default_rng(1)
+    orc.u[0] = rng.standard_normal((3, 4, 8)); orc.v[0] = rng.random((3, 4, 8))
+    mu, v_before = orc.u[0].mean(axis=0), orc.v[0].copy()
+    orc.sync_states(True, False)
+    assert np.allclose(orc.u[0], mu[None]) and np.array_equal(orc.v[0], v_before)
+    orc.sync_states(False, True)
+    assert np.allclose(orc.v[0], v_before.mean(axis=0)[None])
