@@ -688,7 +688,7 @@ int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t 
   switch (s.type) {
     case ST_GEMM:
       sc.a_square = s.a_square;
-      launch_gemm(c->d_probs + s.first, s.count, s.tiles, s.atrans, s.dual, sc, st);
+      launch_gemm(c->d_probs + s.first, s.count, s.tiles, s.atrans, s.dual, c->cfg.check_mode != 0, sc, st);
       c->launches += 1;
       return check_launch(c, "gemm");
     case ST_CHOL:

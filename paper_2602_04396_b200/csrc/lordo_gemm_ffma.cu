@@ -53,7 +53,9 @@ __device__ __forceinline__ float4 operand_load4(const Operand& op, const void* b
   return make_float4(t[0], t[1], t[2], t[3]);
 }
 
-template <int ATRANS, int DUAL>
+// CARRY = 1: slice sums carried across k-slices in fp64 (parity mode). CARRY = 0: plain fp32
+// accumulation, half the registers (the fp32 work of the fast mode: QR and moment rotation).
+template <int ATRANS, int DUAL, int CARRY>
 __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __restrict__ probs, int nprobs, GemmScalars sc) {
   __shared__ __align__(16) float sA[BK][BM + PADS];
   __shared__ __align__(16) float sB[BK][BN + PADS];
@@ -88,14 +90,17 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
   const int ar = ATRANS ? (t >> 4) : (t >> 2), ac = ATRANS ? (t & 15) * 4 : (t & 3) * 4;
 
   float acc[4][4], acc2[DUAL ? 4 : 1][4];
-  double tot[4][4], tot2[DUAL ? 4 : 1][4];
+  double tot[CARRY ? 4 : 1][4], tot2[(CARRY && DUAL) ? 4 : 1][4];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       acc[i][j] = 0.f;
-      tot[i][j] = 0.0;
-      if constexpr (DUAL) { acc2[i][j] = 0.f; tot2[i][j] = 0.0; }
+      if constexpr (CARRY) tot[i][j] = 0.0;
+      if constexpr (DUAL) {
+        acc2[i][j] = 0.f;
+        if constexpr (CARRY) tot2[i][j] = 0.0;
+      }
     }
 
   float4 ra, rb, rb2 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -141,23 +146,27 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
         }
       }
     }
+    if constexpr (CARRY) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          tot[i][j] += (double)acc[i][j];
+          acc[i][j] = 0.f;
+          if constexpr (DUAL) { tot2[i][j] += (double)acc2[i][j]; acc2[i][j] = 0.f; }
+        }
+    }
+    __syncthreads();
+  }
+  if constexpr (CARRY) {
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        tot[i][j] += (double)acc[i][j];
-        acc[i][j] = 0.f;
-        if constexpr (DUAL) { tot2[i][j] += (double)acc2[i][j]; acc2[i][j] = 0.f; }
+        acc[i][j] = (float)tot[i][j];
+        if constexpr (DUAL) acc2[i][j] = (float)tot2[i][j];
       }
-    __syncthreads();
   }
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      acc[i][j] = (float)tot[i][j];
-      if constexpr (DUAL) acc2[i][j] = (float)tot2[i][j];
-    }
 
   // ---- epilogue: each thread owns rows m0+ty*4.., columns n0+tx*4..+3 (N is a multiple of 4)
   const Epilogue& ep = pr.epi;
@@ -211,13 +220,20 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
   }
 }
 
-void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, const GemmScalars& sc,
+void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, int carry, const GemmScalars& sc,
                  cudaStream_t st) {
   const unsigned grid = (unsigned)total_tiles;
-  if (atrans && !dual) gemm_ffma_kernel<1, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
-  else if (!atrans && !dual) gemm_ffma_kernel<0, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
-  else if (!atrans && dual) gemm_ffma_kernel<0, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
-  else gemm_ffma_kernel<1, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+  if (carry) {
+    if (atrans && !dual) gemm_ffma_kernel<1, 0, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+    else if (!atrans && !dual) gemm_ffma_kernel<0, 0, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+    else if (!atrans && dual) gemm_ffma_kernel<0, 1, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+    else gemm_ffma_kernel<1, 1, 1><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+  } else {
+    if (atrans && !dual) gemm_ffma_kernel<1, 0, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+    else if (!atrans && !dual) gemm_ffma_kernel<0, 0, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+    else if (!atrans && dual) gemm_ffma_kernel<0, 1, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+    else gemm_ffma_kernel<1, 1, 0><<<grid, 256, 0, st>>>(probs, nprobs, sc);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -61,7 +61,7 @@ struct GemmScalars {
   int form, ef, w_dt, e_dt, g_dt, a_square;
 };
 
-void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, const GemmScalars& sc,
+void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, int atrans, int dual, int carry, const GemmScalars& sc,
                  cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
