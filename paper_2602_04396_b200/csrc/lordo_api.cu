@@ -732,8 +732,7 @@ int set_gradients(lordo_ctx* c, const void* const* G, cudaStream_t st) {
     for (int i = 0; i < c->n_mats; ++i) {
       const lordo_mat& a = c->mats[i];
       if (!encode_map3(c->h_gmaps[i].g_sw, G[i], a.n, a.m, c->K, 64, 64, true) ||
-          !encode_map3(c->h_gmaps[i].g_kb, G[i], a.n, a.m, c->K, 64, 128, true) ||
-          !encode_map3(c->h_gmaps[i].g_ns, G[i], a.n, a.m, c->K, 128, 64, false))
+          !encode_map3(c->h_gmaps[i].g_kb, G[i], a.n, a.m, c->K, 64, 128, true))
         return fail(c, LORDO_ERR_CUDA, "tensor map encoding failed for a gradient");
     }
     CUDA_OK(c, cudaMemcpyAsync(c->d_gmaps, c->h_gmaps, sizeof(TmaGradMaps) * c->n_mats, cudaMemcpyHostToDevice, st));
@@ -853,11 +852,10 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         std::memset(&hm[i], 0, sizeof(TmaMatMaps));
         if (md.E) {
           good = good && encode_map3(hm[i].e_sw, md.E, md.n, md.m, c->K, 64, 64, true);
-          good = good && encode_map3(hm[i].e_ns, md.E, md.n, md.m, c->K, 128, 64, false);
-          good = good && encode_map3(hm[i].e_st, md.E, md.n, md.m, c->K, 128, 16, false);
+          good = good && encode_map3(hm[i].e_st, md.E, md.n, md.m, c->K, 64, 16, true);
         }
-        good = good && encode_map3(hm[i].w_ns, md.W, md.n, md.m, c->K, 128, 64, false);
-        good = good && encode_map3(hm[i].w_st, md.W, md.n, md.m, c->K, 128, 16, false);
+        good = good && encode_map3(hm[i].w_sw, md.W, md.n, md.m, c->K, 64, 64, true);
+        good = good && encode_map3(hm[i].w_st, md.W, md.n, md.m, c->K, 64, 16, true);
         good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n < 256 ? tp.r_n : 256, true);
         good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
         // refresh: signal as rows (64 k x 128 rows) and right-hand sides [batch][Kd][r]

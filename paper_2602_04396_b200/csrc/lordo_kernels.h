@@ -90,17 +90,17 @@ struct TcProblem {
 };
 
 // Tensor maps (opaque 128-byte objects encoded on the host) of one matrix for the TMA-fed kernels.
-// "sw": 64 x 64 boxes with the 128-byte swizzle (operands of the projection); "ns": 128 x 64 boxes
-// without swizzle (tiles the update epilogue reads and writes in place); "st": 128 x 16 boxes.
+// "sw": 64 x 64 boxes with the 128-byte swizzle (operands of the projection, and the tiles the update
+// epilogue reads and writes in place); "st": 64 x 16 boxes with the same swizzle.
 struct alignas(128) TmaMatMaps {
-  unsigned char e_sw[128], pt[128], p16[128], e_ns[128], w_ns[128];
+  unsigned char e_sw[128], pt[128], p16[128], w_sw[128];
   // refresh: E and Delta16 as 64 x 128 swizzled boxes ("kb", rows of S as MMA rows), Delta16 as
   // 64 x 64 swizzled boxes, and the three bf16 right-hand sides [batch][Kd][r]
   unsigned char e_kb[128], d_kb[128], d_sw[128], om16[128], pn16[128], zq16[128];
   unsigned char e_st[128], w_st[128];  // stores of one row group of the update epilogue
 };
 struct alignas(128) TmaGradMaps {  // re-encoded whenever the caller's gradient pointer changes
-  unsigned char g_sw[128], g_ns[128], g_kb[128];
+  unsigned char g_sw[128], g_kb[128];
 };
 
 struct TcPrep {

@@ -8,8 +8,8 @@
 //                       moment-update epilogue of one strip run under the main loop of the next.
 //   apply_tma_kernel    The strip's two low-rank operands (g^T, U~^T) live in tensor memory as the
 //                       A operands; rows of P and the tiles of G, E, W arrive by TMA; the epilogue
-//                       works on the tiles in shared memory (one column per thread) and the
-//                       updated E and W tiles leave by TMA stores.
+//                       works on the swizzled tiles in shared memory (four neighbouring columns per
+//                       thread, 8-byte accesses) and the updated E and W tiles leave by TMA stores.
 //
 // One CTA per SM; a CTA walks the list of 128-column strips with stride gridDim.x. Every role walks
 // the same list, so stage and phase counters stay in step without further communication.
@@ -318,9 +318,11 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           unsigned char* base = sIn + is * kAInStageBytes;
           const bool ld_e = DO_E && ef;
           mbar_expect_tx(&in_full[is], 16384u + (ld_e ? 16384u : 0u) + (DO_W ? 16384u : 0u));
-          tma_load_3d(base, gm->g_ns, n0, t * kARows, rep, &in_full[is]);
-          if (ld_e) tma_load_3d(base + 16384, mm->e_ns, n0, t * kARows, rep, &in_full[is]);
-          if (DO_W) tma_load_3d(base + 32768, mm->w_ns, n0, t * kARows, rep, &in_full[is]);
+          for (int hh = 0; hh < 2; ++hh) {  // two 64-column halves per tile, 8 KB each
+            tma_load_3d(base + hh * 8192, gm->g_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+            if (ld_e) tma_load_3d(base + 16384 + hh * 8192, mm->e_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+            if (DO_W) tma_load_3d(base + 32768 + hh * 8192, mm->w_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+          }
         }
       }
     }
@@ -380,12 +382,24 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       }
     }
   } else {
-    // ---------------- epilogue: one column per thread, 16 rows per step --------------------------
+    // ---------------- epilogue: 4 columns x 4 rows per thread and step ---------------------------
+    // Lane l = 8a + b of a warp's lane quarter holds strip column 32q + 4b + a, so that the two
+    // 16-lane accumulator loads hand thread t the four neighbouring columns 4(t/4)..+3 of rows
+    // 2(t%4), +1, +8, +9 of its row group: 8-byte accesses to the swizzled tiles, free of conflicts.
     const int ew = warp - 2;
     const int q = warp & 3, grp = ew >> 2;  // lane quarter (fixed by the hardware), row group 0..3
-    const int colq = q * 32 + lane;          // column within the strip
+    const int colq = q * 32 + 4 * (lane & 7) + (lane >> 3);  // column this lane's operands belong to
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-    const int tile_off = colq * 2;  // inside a 16 KB tile of 64 rows x 128 columns
+    const int tb = lane >> 2, tr = lane & 3;
+    const int ecol0 = q * 32 + 4 * tb;  // first of this thread's four epilogue columns
+    // byte offsets inside a 16 KB tile (two halves of 64 rows x 128 bytes, 128-byte swizzle)
+    uint32_t toff[4];
+#pragma unroll
+    for (int ri = 0; ri < 4; ++ri) {
+      const int rho = grp * 16 + (ri >> 1) * 8 + 2 * tr + (ri & 1);
+      const int chunk = 4 * (q & 1) + (tb >> 1);
+      toff[ri] = (uint32_t)((q >> 1) * 8192 + rho * 128 + ((chunk ^ (rho & 7)) << 4) + 8 * (tb & 1));
+    }
     const float lr = sc.lr, om = sc.omega;
     const bool full = sc.form == LORDO_QHM_FULL;
     const float a2w = full ? om : 1.f;
@@ -401,7 +415,12 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       const long long col = (long long)n0 + colq;
       const long long colc = col < n ? col : (long long)n - 1;
       const float c = *pr->cptr;
-      const float cd = full ? (1.f - om) * c / pr->dcol[colc] : 0.f;
+      float cd[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const long long ec = (long long)n0 + ecol0 + j;
+        cd[j] = full ? (1.f - om) * c / pr->dcol[ec < n ? ec : (long long)n - 1] : 0.f;
+      }
       // this thread's quarter of its column's low-rank operands -> tensor memory (r_k/8 columns each)
       {
         const int per = r_k / 8;  // 32-bit columns of one operand handled by this row group
@@ -427,49 +446,65 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       for (int t = 0; t < nsteps; ++t, ++jt) {
         const int is = jt % INST;
         const uint32_t b = jt & 1u;
-        unsigned char* base = sIn + is * kAInStageBytes + tile_off + grp * 16 * 256;
+        unsigned char* base = sIn + is * kAInStageBytes;
         ok = mbar_wait<32>(&in_full[is], (jt / INST) & 1u, status);
         if (ok) ok = mbar_wait<32>(&acc_full[b], (jt >> 1) & 1u, status);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
         // both accumulators come out of tensor memory together and the buffer goes back to the MMA
-        // warp before any arithmetic; the tiles are then updated in place, 8 rows at a time
-        float a1[16], a2[16];
-        if (MODE == 0) {
-          tmem_ld16x2(taddr, taddr + 64, a1, a2);  // (P g)^T, (P U~)^T
-        } else if (MODE == 1) {
-          tmem_ld16(taddr, a1);
-        } else {
-          tmem_ld16(taddr + 64, a2);
+        // warp before any arithmetic. a?[h][4k + 2jj + p]: column 2h + jj, row 8k + 2(t%4) + p.
+        float a1[2][8], a2[2][8];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (DO_E) tmem_ld_16x256b_x2(taddr + ((uint32_t)(h * 16) << 16), a1[h]);       // (P g)^T
+          if (DO_W) tmem_ld_16x256b_x2(taddr + 64 + ((uint32_t)(h * 16) << 16), a2[h]);  // (P U~)^T
+        }
+        tmem_ld_wait();
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (DO_E) tmem_ld_pin8(a1[h]);
+          if (DO_W) tmem_ld_pin8(a2[h]);
         }
         tc_fence_before_sync();
         mbar_arrive(&acc_empty[b]);
+        uint2 gv[4], ev[4], wv[4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          float g[8], e[8], w[8];
+        for (int ri = 0; ri < 4; ++ri) {
+          gv[ri] = *reinterpret_cast<const uint2*>(base + toff[ri]);
+          if (DO_E && ef) ev[ri] = *reinterpret_cast<const uint2*>(base + 16384 + toff[ri]);
+          if (DO_W) wv[ri] = *reinterpret_cast<const uint2*>(base + 32768 + toff[ri]);
+        }
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            unsigned char* rowp = base + (h * 8 + j) * 256;
-            g[j] = bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp));
-            e[j] = (DO_E && ef) ? bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 16384)) : 0.f;
-            w[j] = DO_W ? bf16_to_f(*reinterpret_cast<const unsigned short*>(rowp + 32768)) : 0.f;
+        for (int ri = 0; ri < 4; ++ri) {
+          const int k = ri >> 1, p = ri & 1;
+          const float g0 = bf_lo(gv[ri].x), g1 = bf_hi(gv[ri].x), g2 = bf_lo(gv[ri].y), g3 = bf_hi(gv[ri].y);
+          if (DO_E && ef) {
+            const float e0 = (c * g0 + bf_lo(ev[ri].x)) - a1[0][4 * k + p];
+            const float e1 = (c * g1 + bf_hi(ev[ri].x)) - a1[0][4 * k + 2 + p];
+            const float e2 = (c * g2 + bf_lo(ev[ri].y)) - a1[1][4 * k + p];
+            const float e3 = (c * g3 + bf_hi(ev[ri].y)) - a1[1][4 * k + 2 + p];
+            *reinterpret_cast<uint2*>(base + 16384 + toff[ri]) = make_uint2(pack2_bf16(e0, e1), pack2_bf16(e2, e3));
           }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            unsigned char* rowp = base + (h * 8 + j) * 256;
-            if (DO_E && ef) *reinterpret_cast<unsigned short*>(rowp + 16384) = f_to_bf16((c * g[j] + e[j]) - a1[h * 8 + j]);
-            if (DO_W) *reinterpret_cast<unsigned short*>(rowp + 32768) = f_to_bf16(w[j] - lr * (cd * g[j] + a2w * a2[h * 8 + j]));
+          if (DO_W) {
+            const float w0 = bf_lo(wv[ri].x) - lr * (cd[0] * g0 + a2w * a2[0][4 * k + p]);
+            const float w1 = bf_hi(wv[ri].x) - lr * (cd[1] * g1 + a2w * a2[0][4 * k + 2 + p]);
+            const float w2 = bf_lo(wv[ri].y) - lr * (cd[2] * g2 + a2w * a2[1][4 * k + p]);
+            const float w3 = bf_hi(wv[ri].y) - lr * (cd[3] * g3 + a2w * a2[1][4 * k + 2 + p]);
+            *reinterpret_cast<uint2*>(base + 32768 + toff[ri]) = make_uint2(pack2_bf16(w0, w1), pack2_bf16(w2, w3));
           }
         }
         // the four warps of a row group hand their 16 rows to the TMA engine on their own
         fence_async_smem();
         asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory");
         if ((ew & 3) == 0 && lane == 0) {
-          unsigned char* sb = sIn + is * kAInStageBytes + grp * 16 * 256;
+          unsigned char* sb = base + grp * 2048;
           const int row = t * kARows + grp * 16;
-          if (DO_E && ef) tma_store_3d(mm->e_st, n0, row, rep, sb + 16384);
-          if (DO_W) tma_store_3d(mm->w_st, n0, row, rep, sb + 32768);
+          for (int hh = 0; hh < 2; ++hh) {
+            if (n0 + hh * 64 >= n) break;
+            if (DO_E && ef) tma_store_3d(mm->e_st, n0 + hh * 64, row, rep, sb + 16384 + hh * 8192);
+            if (DO_W) tma_store_3d(mm->w_st, n0 + hh * 64, row, rep, sb + 32768 + hh * 8192);
+          }
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(&in_free[is]);

@@ -186,6 +186,23 @@ __device__ __forceinline__ void tmem_ld16x2(uint32_t taddr_a, uint32_t taddr_b, 
   for (int i = 0; i < 16; ++i) { va[i] = __uint_as_float(a[i]); vb[i] = __uint_as_float(b[i]); }
 }
 
+// 16 lanes x 16 columns starting at `taddr` (its lane field a multiple of 16), no wait. Thread t of the
+// warp receives, for column block k = 0, 1: v[4k+0], v[4k+1] = lane t/4, columns 8k + 2(t%4), +1;
+// v[4k+2], v[4k+3] = lane t/4 + 8, same columns.
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, float* v) {
+  uint32_t r[8];
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Keeps the compiler from using the eight loaded values before the wait that precedes this call.
+__device__ __forceinline__ void tmem_ld_pin8(float* v) {
+  asm volatile("" : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]));
+}
+
 // Byte offset of the 16-byte chunk `ch` (0..7) of row `i` inside a swizzled tile.
 __device__ __forceinline__ uint32_t swz_chunk(int i, int ch) {
   return (uint32_t)((i >> 3) * 1024 + (i & 7) * 128 + ((ch ^ (i & 7)) << 4));
