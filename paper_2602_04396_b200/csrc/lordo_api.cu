@@ -313,8 +313,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       const int copies = local ? K : 1;
       __nv_bfloat16* P16 = cv.take<__nv_bfloat16>((size_t)copies * m_k * r_k);
       __nv_bfloat16* PT16 = cv.take<__nv_bfloat16>((size_t)copies * r_n * m_k);
-      __nv_bfloat16* gT16 = cv.take<__nv_bfloat16>((size_t)K * md.n * r_k);
-      __nv_bfloat16* uT16 = cv.take<__nv_bfloat16>((size_t)K * md.n * r_k);
+      const size_t n_pad = (size_t)up(md.n, 128);  // whole strips: the TMA-fed kernels store these per strip
+      __nv_bfloat16* gT16 = cv.take<__nv_bfloat16>((size_t)K * n_pad * r_k);
+      __nv_bfloat16* uT16 = cv.take<__nv_bfloat16>((size_t)K * n_pad * r_k);
       if (r_n > c->tc_rn_max) c->tc_rn_max = r_n;
       if (r_k > c->tc_rk_max) c->tc_rk_max = r_k;
       for (int k = 0; k < copies; ++k) {
@@ -334,7 +335,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         tp.strip_start = c->tc_strips;
         tp.m = (int)md.m; tp.n = (int)md.n; tp.r = md.r; tp.r_k = r_k; tp.r_n = r_n; tp.m_k = m_k;
         tp.PT16 = PT16 + (size_t)pk * r_n * m_k; tp.P16 = P16 + (size_t)pk * m_k * r_k;
-        tp.gT16 = gT16 + (size_t)k * md.n * r_k; tp.uT16 = uT16 + (size_t)k * md.n * r_k;
+        tp.gT16 = gT16 + (size_t)k * n_pad * r_k; tp.uT16 = uT16 + (size_t)k * n_pad * r_k;
         tp.u = md.u ? md.u + so : nullptr; tp.v = md.v ? md.v + so : nullptr;
         tp.dcol = md.dcol + (long long)k * md.n;
         if (real) {

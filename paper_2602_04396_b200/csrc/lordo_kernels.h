@@ -76,8 +76,12 @@ struct TcProblem {
   int m_k;                     // m rounded up to 64: k extent of PT16, rows of P16
   const __nv_bfloat16* PT16;   // [r_n][m_k]  P^T, zero padded
   const __nv_bfloat16* P16;    // [m_k][r_k]  P, zero padded
-  __nv_bfloat16* gT16;         // [n][r_k]    low-rank gradient, transposed
-  __nv_bfloat16* uT16;         // [n][r_k]    normalised low-rank update U~, transposed
+  // Low-rank gradient and normalised low-rank update U~, transposed, private to the projection and
+  // update kernels of one path. Register-staged kernels: [n][r_k]. TMA-fed kernels:
+  // [strip][r_k/8][128 columns][8], i.e. the 16-byte pieces of one k-chunk of a strip's columns lie
+  // side by side and a warp moves 512 contiguous bytes. Room for ceil(n/128)*128 columns either way.
+  __nv_bfloat16* gT16;
+  __nv_bfloat16* uT16;
   float* u;                    // [r][n] of this worker
   float* v;
   float* dcol;                 // [n]

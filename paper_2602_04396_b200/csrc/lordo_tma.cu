@@ -197,8 +197,10 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       const long long ecolc = e_ok ? ecol : (long long)n - 1;
       float* __restrict__ up_ = pr->u;
       float* __restrict__ vp_ = pr->v;
-      __nv_bfloat16* __restrict__ gT = pr->gT16 + ecolc * r_k;
-      __nv_bfloat16* __restrict__ uT = pr->uT16 + ecolc * r_k;
+      // this column's 16-byte pieces inside the strip's block [r_k/8][128][8]
+      const size_t lr_off = (size_t)(strip - pr->strip_start) * (size_t)r_k * 128 + (size_t)(q * 32 + lane) * 8;
+      __nv_bfloat16* __restrict__ gT = pr->gT16 + lr_off;
+      __nv_bfloat16* __restrict__ uT = pr->uT16 + lr_off;
       const uint32_t buf = BIG ? 0u : (si & 1u);
       ok = mbar_wait<64>(&acc_full[buf], (BIG ? si : (si >> 1)) & 1u, status);
       if (!ok) break;
@@ -240,10 +242,10 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           upk[i >> 1] = pack2_bf16(o[0], o[1]);
         }
         if (e_ok) {
-          uint4* gd = reinterpret_cast<uint4*>(gT + ch * 16);
-          uint4* ud = reinterpret_cast<uint4*>(uT + ch * 16);
-          gd[0] = make_uint4(gp[0], gp[1], gp[2], gp[3]); gd[1] = make_uint4(gp[4], gp[5], gp[6], gp[7]);
-          ud[0] = make_uint4(upk[0], upk[1], upk[2], upk[3]); ud[1] = make_uint4(upk[4], upk[5], upk[6], upk[7]);
+          uint4* gd = reinterpret_cast<uint4*>(gT + (size_t)ch * 2048);  // k-chunks 2ch and 2ch+1, 128 pieces apart
+          uint4* ud = reinterpret_cast<uint4*>(uT + (size_t)ch * 2048);
+          gd[0] = make_uint4(gp[0], gp[1], gp[2], gp[3]); gd[128] = make_uint4(gp[4], gp[5], gp[6], gp[7]);
+          ud[0] = make_uint4(upk[0], upk[1], upk[2], upk[3]); ud[128] = make_uint4(upk[4], upk[5], upk[6], upk[7]);
         }
       }
       tc_fence_before_sync();
@@ -424,17 +426,20 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       // this thread's quarter of its column's low-rank operands -> tensor memory (r_k/8 columns each)
       {
         const int per = r_k / 8;  // 32-bit columns of one operand handled by this row group
-        const __nv_bfloat16* __restrict__ g16 = pr->gT16 + colc * r_k + grp * (r_k / 4);
-        const __nv_bfloat16* __restrict__ u16 = pr->uT16 + colc * r_k + grp * (r_k / 4);
+        // strip block [r_k/8][128][8]: this row group's k-chunks, this lane's column; a warp reads 512
+        // contiguous bytes per instruction
+        const size_t lr_off = (size_t)(strip - pr->strip_start) * (size_t)r_k * 128 + (size_t)grp * (r_k / 32) * 1024 + (size_t)colq * 8;
+        const uint4* __restrict__ g16 = reinterpret_cast<const uint4*>(pr->gT16 + lr_off);
+        const uint4* __restrict__ u16 = reinterpret_cast<const uint4*>(pr->uT16 + lr_off);
         const bool live = col < n;
         for (int c0 = 0; c0 < per; c0 += 8) {
           if (DO_E) {
-            uint4 glo = *reinterpret_cast<const uint4*>(g16 + c0 * 2), ghi = *reinterpret_cast<const uint4*>(g16 + c0 * 2 + 8);
+            uint4 glo = g16[(c0 >> 2) * 128], ghi = g16[(c0 >> 2) * 128 + 128];
             if (!live) glo = ghi = make_uint4(0u, 0u, 0u, 0u);
             tmem_st8(tmem + lane_base + (uint32_t)(grp * per + c0), glo, ghi);
           }
           if (DO_W) {
-            uint4 ulo = *reinterpret_cast<const uint4*>(u16 + c0 * 2), uhi = *reinterpret_cast<const uint4*>(u16 + c0 * 2 + 8);
+            uint4 ulo = u16[(c0 >> 2) * 128], uhi = u16[(c0 >> 2) * 128 + 128];
             if (!live) ulo = uhi = make_uint4(0u, 0u, 0u, 0u);
             tmem_st8(tmem + lane_base + A2COL + (uint32_t)(grp * per + c0), ulo, uhi);
           }
