@@ -506,6 +506,47 @@ def test_config4_full_size_fast_mode_sampled_columns():
     opt.close()
 
 
+def _fold(t):
+    """Order-sensitive 64-bit fold of a tensor's bit pattern (computed on the device)."""
+    v = t.contiguous().view(-1)
+    v = (v.view(torch.int16) if v.element_size() == 2 else v.view(torch.int32)).to(torch.int64)
+    return int(v.sum().item()) ^ int((v * (torch.arange(v.numel(), device=v.device) % 8191 + 1)).sum().item())
+
+
+@pytest.mark.gpu
+def test_config4_full_size_fast_mode_repeatable():
+    """Two runs of the full-size launch configuration from the same seed give the same bits in every
+    matrix of W, E, u, v after the inner steps and in every P after the refresh, and raise no flag.
+    None of these kernels uses atomics on data, so any difference is a race between their roles."""
+    from paper_2602_04396_b200 import lordo
+    free, _total = torch.cuda.mem_get_info()
+    if free < 125 * 2 ** 30:
+        pytest.skip("needs about 120 GB of free device memory")
+    wl = synth.scaled(synth.config(4), H=2)
+    seed, lr, beta1, omega, form = 11, 0.004, 0.999, 0.97, 2
+    runs = []
+    for _rep in range(2):
+        W0 = synth.init_weights_device(wl, seed)
+        opt = lordo.Lordo(wl.mats, wl.K, wl.H, W0, g_dtype=torch.bfloat16, e_dtype=torch.bfloat16, variant=0, error_feedback=True,
+                          beta2=0.999, eps=0.05, clip_rho=wl.clip_rho, outer=lordo.OUTER_NESTEROV, outer_lr=0.8, outer_momentum=0.9,
+                          seed=seed, check_mode=0)
+        del W0
+        G = None
+        for h in range(2):
+            G = synth.gradients_device(wl, seed, 0, h, out=G)
+            opt.inner_step(G, lr, beta1, omega, form)
+        folds = [_fold(getattr(opt, name)[i]) for name in ("W", "E", "u", "v") for i in range(len(wl.mats))]
+        opt.outer_step()
+        opt.refresh_subspace(None, beta1)
+        assert opt.poll_status() == 0
+        folds += [_fold(opt.P[i]) for i in range(len(wl.mats))]
+        runs.append(folds)
+        opt.close()
+        del opt, G
+    differing = [k for k in range(len(runs[0])) if runs[0][k] != runs[1][k]]
+    assert not differing, differing[:8]
+
+
 # ------------------------------------------------------------------ determinism and checkpoint / resume
 
 def _run_rounds_gpu(opt, wl, seed, rounds, first_round, variant, form, lr=0.01, beta1=0.9, omega=0.9):
