@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kMaxK = 64;
 
-enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3, ST_SKETCH = 4, ST_CONVERT = 5 };
+enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3, ST_SKETCH = 4, ST_CONVERT = 5, ST_NORM = 6 };
 enum Phase { PH_SUBSPACE = 0, PH_ROTATE = 1, PH_COMMIT = 2 };
 
 // One launch of the refresh / init / inner-step plans. The entries it works on are a contiguous
@@ -40,6 +40,7 @@ struct SlotBuilder {
     std::vector<CopyProblem> cp;
     std::vector<SkProblem> sk;
     std::vector<ConvProblem> cv;
+    std::vector<NormProblem> nm;
   };
   std::vector<Slot> slots;
   size_t cur = 0;
@@ -89,6 +90,7 @@ struct lordo_ctx {
   CopyProblem* d_copies = nullptr;
   SkProblem* d_sks = nullptr;
   ConvProblem* d_convs = nullptr;
+  NormProblem* d_norms = nullptr;
   float* d_scratch = nullptr;
   long long total_chunks = 0, total_mom_tiles = 0, total_wblks = 0, total_sblks = 0;
 
@@ -120,7 +122,12 @@ struct lordo_ctx {
   std::vector<DiagProblem> h_diag;  // one per rotation matrix, ordered by matrix then batch entry
   DiagProblem* d_diag = nullptr;
   std::vector<ConvProblem> h_convs;
-  struct SketchBufs { __nv_bfloat16 *om16 = nullptr, *pn16 = nullptr, *zq16 = nullptr; };
+  std::vector<NormProblem> h_norms;
+  struct SketchBufs {
+    __nv_bfloat16 *om16 = nullptr, *pn16 = nullptr, *zq16 = nullptr;
+    // hi|lo planes of the tensor-core QR and rotation (null when those run in fp32)
+    __nv_bfloat16 *x16 = nullptr, *rinv16 = nullptr, *phl = nullptr, *rt16 = nullptr, *sq16 = nullptr, *uh16 = nullptr, *wr16 = nullptr;
+  };
   std::vector<SketchBufs> h_skbufs;  // per matrix: bf16 right-hand sides of the sketch products (refresh scratch)
   PlanStep inner_proj, inner_apply;
   std::vector<PlanStep> refresh_steps, init_steps;
@@ -253,7 +260,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   prefix_arrays(cfg, chunk_start, mom_start, wblk, sblk);
   // Refresh scratch: matrices are processed in groups whose scratch fits kRefreshScratchFloats;
   // every step of the refresh is one launch over a whole group.
-  constexpr size_t kRefreshScratchFloats = size_t(1) << 32;  // 16 GiB
+  constexpr size_t kRefreshScratchFloats = size_t(1) << 31;  // 8 GiB
   std::vector<size_t> mat_scratch(n_mats);
   std::vector<int> group_of(n_mats);
   size_t scratch_floats = 0;
@@ -268,7 +275,14 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
                    4 * (size_t)a.r * a.r;
       // bf16 right-hand sides of the tensor-core sketch products (Omega, P', Z), counted in floats
       per += ((size_t)a.n * a.r + (q > 0 ? (size_t)a.m * a.r + (size_t)a.n * a.r : 0)) / 2 + 64;
-      mat_scratch[i] = nb * per;
+      size_t states16 = 0;
+      if (cfg.check_mode == 0 && cfg.w_dtype == LORDO_BF16) {
+        // bf16 planes of the tensor-core QR and rotation: X and R^-1 in three planes, P, Rot^T, its square
+        // (per batch entry) and the two moment operands of every worker in two
+        per += 3 * (size_t)maxd * a.r / 2 + (size_t)a.m * a.r + 7 * (size_t)a.r * a.r / 2 + 128;
+        states16 = 2 * (size_t)K * a.r * a.n + 64;
+      }
+      mat_scratch[i] = nb * per + states16;
       if (acc > 0 && acc + mat_scratch[i] > kRefreshScratchFloats) { ++grp; acc = 0; }
       group_of[i] = grp;
       acc += mat_scratch[i];
@@ -364,7 +378,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
 
   // ---------------- launch plans ----------------
   std::vector<GemmProblem>& P = c->h_probs;
-  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear(); c->h_diag.clear();
+  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear(); c->h_norms.clear(); c->h_diag.clear();
   c->h_skbufs.assign(n_mats, lordo_ctx::SketchBufs());
   const bool tc_sketch = c->tc && c->tma;  // sketch products of the refresh on tensor cores
   auto gemm_prob = [&](int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
@@ -406,6 +420,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       } else if (st.type == ST_CONVERT) {
         st.first = (long long)c->h_convs.size(); st.count = (int)sl.cv.size(); st.tiles = 0;
         for (ConvProblem& x : sl.cv) { x.blk_start = st.tiles; st.tiles += (x.count + 1023) / 1024; c->h_convs.push_back(x); }
+      } else if (st.type == ST_NORM) {
+        st.first = (long long)c->h_norms.size(); st.count = (int)sl.nm.size(); st.tiles = 0;
+        for (NormProblem& x : sl.nm) { x.blk_start = st.tiles; st.tiles += (x.r + 31) / 32; c->h_norms.push_back(x); }
       } else {
         st.first = (long long)c->h_copies.size(); st.count = (int)sl.cp.size(); st.tiles = 0;
         for (CopyProblem& x : sl.cp) { x.blk_start = st.tiles; st.tiles += (x.chunks + 1023) / 1024; c->h_copies.push_back(x); }
@@ -516,6 +533,79 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         zq16 = reinterpret_cast<__nv_bfloat16*>(s); s += ((size_t)nb * n * r) / 2 + 16;
       }
       c->h_skbufs[i].om16 = om16; c->h_skbufs[i].pn16 = pn16; c->h_skbufs[i].zq16 = zq16;
+      // tensor-core QR and rotation: bf16 planes, plane p of batch entry b at index p * nb + b
+      __nv_bfloat16 *x16 = nullptr, *rinv16 = nullptr, *phl = nullptr, *rt16 = nullptr, *sq16 = nullptr, *uh16 = nullptr, *wr16 = nullptr;
+      if (tc_sketch) {
+        auto take16 = [&](size_t floats) { __nv_bfloat16* p16 = reinterpret_cast<__nv_bfloat16*>(s); s += floats + 16; return p16; };
+        x16 = take16(3 * (size_t)nb * maxd * r / 2);
+        phl = take16((size_t)nb * m * r);
+        rinv16 = take16(3 * (size_t)nb * r * r / 2);
+        rt16 = take16((size_t)nb * r * r);
+        sq16 = take16((size_t)nb * r * r);
+        uh16 = take16((size_t)K * r * n);
+        wr16 = take16((size_t)K * r * n);
+        lordo_ctx::SketchBufs& kb = c->h_skbufs[i];
+        kb.x16 = x16; kb.rinv16 = rinv16; kb.phl = phl; kb.rt16 = rt16; kb.sq16 = sq16; kb.uh16 = uh16; kb.wr16 = wr16;
+      }
+      TmaMatMaps* mmi = c->d_maps + i;
+      auto conv = [&](SlotBuilder& sb, int phase, const ConvProblem& cp) { sb.next(ST_CONVERT, phase).cv.push_back(cp); };
+      auto conv_split = [&](SlotBuilder& sb, int phase, const float* src, long long sstride, __nv_bfloat16* planes, long long elems, int np) {
+        SlotBuilder::Slot& sl = sb.next(ST_CONVERT, phase);
+        for (int b = 0; b < nb; ++b) {
+          ConvProblem cp;
+          std::memset(&cp, 0, sizeof(cp));
+          cp.mode = CONV_SPLIT; cp.src = src ? src + b * sstride : nullptr; cp.count = elems;
+          cp.dst = planes + (long long)b * elems; cp.plane = (long long)nb * elems; cp.planes = np;
+          sl.cv.push_back(cp);
+        }
+      };
+      // C = A B as the sum of the products of np-plane split operands; planes as above. a_mn: A stored [Kd][M].
+      auto sk_split = [&](SlotBuilder::Slot& sl, int a_mn, const unsigned char* map_a, int a_b, int a_nb, const unsigned char* map_b, int b_b, int b_nb,
+                          long long Mo, long long Kd, float* C, long long ldc, int c_trans, int np) {
+        SkProblem sp;
+        std::memset(&sp, 0, sizeof(sp));
+        sp.M = (int)Mo; sp.Kd = (int)Kd; sp.r = r; sp.r_n = (r + 15) / 16 * 16;
+        sp.a_mn = a_mn; sp.a_c2 = a_b; sp.a_pl = a_nb; sp.b_c2 = b_b; sp.b_pl = b_nb;
+        sp.split = np; sp.c_trans = c_trans;
+        sp.map_a = map_a; sp.map_b = map_b; sp.C = C; sp.ldc = ldc;
+        sl.sk.push_back(sp);
+      };
+      // CholeskyQR2 with the Gram matrices and the products with R^-1 on tensor cores, operands in three
+      // planes: the Gram matrix then carries fp32's rounding noise, which the breakdown threshold of the
+      // Cholesky step assumes
+      auto cholqr2_tc = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows) {
+        const bool by_m = rows == m;
+        const unsigned char* x_sw = by_m ? mmi->xm_sw : mmi->xn_sw;
+        const unsigned char* x_kb = by_m ? mmi->xm_kb : mmi->xn_kb;
+        float* src = X; long long ss = sx;
+        for (int pass = 0; pass < 2; ++pass) {
+          float* dst = pass == 0 ? T : O;
+          const long long sd = pass == 0 ? st : so;
+          conv_split(sb, phase, src, ss, x16, rows * r, 3);
+          SlotBuilder::Slot& g = sb.next(ST_SKETCH, phase);
+          for (int b = 0; b < nb; ++b) sk_split(g, 1, x_sw, b, nb, x_sw, b, nb, r, rows, gram + (long long)b * r * r, r, 0, 3);
+          SlotBuilder::Slot& ch = sb.next(ST_CHOL, phase);
+          for (int b = 0; b < nb; ++b) {
+            CholProblem cp;
+            cp.gram = gram + (long long)b * r * r; cp.lwork = lw + (long long)b * r * r; cp.rinv = rinv + (long long)b * r * r; cp.r = r; cp.pad = 0;
+            ch.ch.push_back(cp);
+          }
+          conv_split(sb, phase, rinv, (long long)r * r, rinv16, (long long)r * r, 3);
+          SlotBuilder::Slot& ap = sb.next(ST_SKETCH, phase);
+          for (int b = 0; b < nb; ++b) sk_split(ap, 0, x_kb, b, nb, mmi->rinv_sw, b, nb, rows, r, dst + b * sd, r, 0, 3);
+          src = dst; ss = sd;
+        }
+        SlotBuilder::Slot& nr = sb.next(ST_NORM, phase);  // the columns of Q back to unit length
+        for (int b = 0; b < nb; ++b) {
+          NormProblem np;
+          np.X = O + b * so; np.blk_start = 0; np.rows = (int)rows; np.r = r;
+          nr.nm.push_back(np);
+        }
+      };
+      auto qr2 = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows) {
+        if (tc_sketch) cholqr2_tc(sb, phase, X, sx, T, st, O, so, rows);
+        else cholqr2(sb, phase, X, sx, T, st, O, so, rows, r, nb, gram, lw, rinv);
+      };
       // S * B on tensor cores: a_mn = 0 -> S rows are the output rows (Y = S B), 1 -> S^T B
       auto sketch = [&](SlotBuilder& sb, int a_mn, unsigned char* map_b, float* C, long long cstride, long long Mo, long long Kd) {
         SlotBuilder::Slot& sl = sb.next(ST_SKETCH, PH_SUBSPACE);
@@ -539,7 +629,8 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       };
       auto convert = [&](SlotBuilder& sb, const float* src, __nv_bfloat16* dst, size_t count) {
         ConvProblem cp;
-        cp.src = src; cp.dst = dst; cp.count = (long long)count; cp.blk_start = 0;
+        std::memset(&cp, 0, sizeof(cp));
+        cp.mode = CONV_BF16; cp.src = src; cp.dst = dst; cp.count = (long long)count;
         sb.next(ST_CONVERT, PH_SUBSPACE).cv.push_back(cp);
       };
 
@@ -576,7 +667,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
         }
-        cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
+        qr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m);
       }
       for (int it = 0; it < q; ++it) {
         if (tc_sketch) {  // Z = S^T P'
@@ -586,7 +677,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, r, (int)m, signal(b), plain(Pn + (long long)b * m * r, r), nullptr, store_epi(Za + (long long)b * n * r, r)));
         }
-        cholqr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n, r, nb, gram, lw, rinv);
+        qr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n);
         if (tc_sketch) {  // Y = S Z
           convert(R, Zq, zq16, (size_t)nb * n * r);
           sketch(R, 0, (c->d_maps + i)->zq16, Ya, m * r, m, n);
@@ -594,31 +685,72 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Zq + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
         }
-        cholqr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r, nb, gram, lw, rinv);
+        qr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m);
       }
       for (int b = 0; b < nb; ++b) {
         DiagProblem dp;
         dp.rot = rot + (long long)b * r * r; dp.r = r; dp.pad = 0;
         c->h_diag.push_back(dp);
       }
-      {  // Rot = P'^T P (always formed: it also carries the MSSV diagnostic)
-        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
-        for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob(r, r, (int)m, plain(Pn + (long long)b * m * r, r), plain(md.P ? md.P + b * md.p_stride : nullptr, r), nullptr, store_epi(rot + (long long)b * r * r, r)));
-      }
-      {  // u', v' (into the transient g^ / U~ areas), then back
-        SlotBuilder::Slot& g = R.next(ST_GEMM, PH_ROTATE, 0, 1, 1);
-        for (int k = 0; k < K; ++k) {
-          const long long so = (long long)k * r * n;
-          Operand A = plain(rot + (long long)(local ? k : 0) * r * r, r);
-          Operand B = plain(md.u ? md.u + so : nullptr, n); B.kind = OP_UHAT;
-          Operand B2 = plain(md.u ? md.u + so : nullptr, n); B2.kind = OP_VRES; B2.p1 = md.v ? md.v + so : nullptr;
-          Epilogue e;
-          std::memset(&e, 0, sizeof(e));
-          e.kind = EPI_ROTATE; e.u_out = md.ghat + so; e.v_out = md.util + so;
-          g.g.push_back(gemm_prob(r, (int)n, r, A, B, &B2, e));
+      if (tc_sketch) {
+        // Rot = P'^T P and the rotated moments on tensor cores, operands in two planes (16 bits each)
+        conv_split(R, PH_SUBSPACE, Pn, m * r, x16, m * r, 2);
+        conv_split(R, PH_SUBSPACE, md.P, md.p_stride, phl, m * r, 2);
+        {
+          SlotBuilder::Slot& g = R.next(ST_SKETCH, PH_SUBSPACE);
+          for (int b = 0; b < nb; ++b) sk_split(g, 1, mmi->xm_sw, b, nb, mmi->phl_sw, b, nb, r, m, rot + (long long)b * r * r, r, 0, 2);
         }
-        add_copy(R, PH_ROTATE, md.u, md.ghat, (size_t)K * r * n * sizeof(float));
-        add_copy(R, PH_ROTATE, md.v, md.util, (size_t)K * r * n * sizeof(float));
+        {  // Rot^T and its element-wise square as right-hand sides
+          SlotBuilder::Slot& sl = R.next(ST_CONVERT, PH_ROTATE);
+          for (int b = 0; b < nb; ++b) {
+            ConvProblem cp;
+            std::memset(&cp, 0, sizeof(cp));
+            cp.mode = CONV_ROT_T; cp.src = rot + (long long)b * r * r; cp.count = (long long)r * r; cp.ld = r;
+            cp.dst = rt16 + (long long)b * r * r; cp.dst2 = sq16 + (long long)b * r * r; cp.plane = (long long)nb * r * r; cp.planes = 2;
+            sl.cv.push_back(cp);
+          }
+        }
+        {  // u^ and v^ - u^ u^ of all workers as hi|lo planes [2K][r][n]
+          ConvProblem cp;
+          std::memset(&cp, 0, sizeof(cp));
+          cp.mode = CONV_STATES; cp.src = md.u; cp.src2 = md.v; cp.count = (long long)K * r * n;
+          cp.dst = uh16; cp.dst2 = wr16; cp.plane = (long long)K * r * n; cp.planes = 2;
+          conv(R, PH_ROTATE, cp);
+        }
+        {  // (Rot u^)^T = u^^T Rot^T, stored back as [r][n] into the transient g^ area; same for the second moment
+          SlotBuilder::Slot& g1 = R.next(ST_SKETCH, PH_ROTATE);
+          for (int k = 0; k < K; ++k)
+            sk_split(g1, 1, mmi->uh_sw, k, K, mmi->rt_sw, local ? k : 0, nb, n, r, md.ghat + (long long)k * r * n, n, 1, 2);
+          SlotBuilder::Slot& g2 = R.next(ST_SKETCH, PH_ROTATE);
+          for (int k = 0; k < K; ++k)
+            sk_split(g2, 1, mmi->wr_sw, k, K, mmi->sq_sw, local ? k : 0, nb, n, r, md.util + (long long)k * r * n, n, 1, 2);
+        }
+        {  // u = bc1 (Rot u^), v = bc2 |Rot^2 (v^ - u^ u^) + (Rot u^)^2|
+          ConvProblem cp;
+          std::memset(&cp, 0, sizeof(cp));
+          cp.mode = CONV_COMBINE; cp.src = md.ghat; cp.src2 = md.util; cp.outf = md.u; cp.outf2 = md.v; cp.count = (long long)K * r * n;
+          conv(R, PH_ROTATE, cp);
+        }
+      } else {
+        {  // Rot = P'^T P (always formed: it also carries the MSSV diagnostic)
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob(r, r, (int)m, plain(Pn + (long long)b * m * r, r), plain(md.P ? md.P + b * md.p_stride : nullptr, r), nullptr, store_epi(rot + (long long)b * r * r, r)));
+        }
+        {  // u', v' (into the transient g^ / U~ areas), then back
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_ROTATE, 0, 1, 1);
+          for (int k = 0; k < K; ++k) {
+            const long long so = (long long)k * r * n;
+            Operand A = plain(rot + (long long)(local ? k : 0) * r * r, r);
+            Operand B = plain(md.u ? md.u + so : nullptr, n); B.kind = OP_UHAT;
+            Operand B2 = plain(md.u ? md.u + so : nullptr, n); B2.kind = OP_VRES; B2.p1 = md.v ? md.v + so : nullptr;
+            Epilogue e;
+            std::memset(&e, 0, sizeof(e));
+            e.kind = EPI_ROTATE; e.u_out = md.ghat + so; e.v_out = md.util + so;
+            g.g.push_back(gemm_prob(r, (int)n, r, A, B, &B2, e));
+          }
+          add_copy(R, PH_ROTATE, md.u, md.ghat, (size_t)K * r * n * sizeof(float));
+          add_copy(R, PH_ROTATE, md.v, md.util, (size_t)K * r * n * sizeof(float));
+        }
       }
       add_copy(R, PH_COMMIT, md.P, Pn, (size_t)nb * m * r * sizeof(float));
       if (!local) {  // P_0 = orthonormalised random m x r matrix
@@ -637,6 +769,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   c->d_copies = cv.take<CopyProblem>(c->h_copies.size() + 1);
   c->d_sks = cv.take<SkProblem>(c->h_sks.size() + 1);
   c->d_convs = cv.take<ConvProblem>(c->h_convs.size() + 1);
+  c->d_norms = cv.take<NormProblem>(c->h_norms.size() + 1);
   c->d_diag = cv.take<DiagProblem>(c->h_diag.size() + 1);
 
   c->last_G.assign(n_mats, nullptr);
@@ -705,9 +838,13 @@ int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t 
       c->launches += 1;
       return check_launch(c, "sketch");
     case ST_CONVERT:
-      launch_convert_grouped(c->d_convs + s.first, s.count, s.tiles, st);
+      launch_convert_grouped(c->d_convs + s.first, s.count, s.tiles, sc, st);
       c->launches += 1;
       return check_launch(c, "convert");
+    case ST_NORM:
+      launch_colnorm_grouped(c->d_norms + s.first, s.count, s.tiles, st);
+      c->launches += 1;
+      return check_launch(c, "colnorm");
     case ST_COPY:
       launch_copy_grouped(c->d_copies + s.first, s.count, s.tiles, st);
       c->launches += 1;
@@ -832,6 +969,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   if (!c->h_sks.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_sks, c->h_sks.data(), sizeof(SkProblem) * c->h_sks.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_diag.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_diag, c->h_diag.data(), sizeof(DiagProblem) * c->h_diag.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_convs.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_convs, c->h_convs.data(), sizeof(ConvProblem) * c->h_convs.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_norms.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_norms, c->h_norms.data(), sizeof(NormProblem) * c->h_norms.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
   if (c->tc) {
     if (!c->tma) INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));  // register-staged kernels (fp32 storage)
@@ -870,6 +1008,18 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         good = good && encode_map3(hm[i].om16, sb.om16, md.r, md.n, nbatch, 64, 64, true);
         if (sb.pn16) good = good && encode_map3(hm[i].pn16, sb.pn16, md.r, md.m, nbatch, 64, 64, true);
         if (sb.zq16) good = good && encode_map3(hm[i].zq16, sb.zq16, md.r, md.n, nbatch, 64, 64, true);
+        if (sb.x16) {  // hi|lo planes of the tensor-core QR and rotation
+          good = good && encode_map3(hm[i].xm_sw, sb.x16, md.r, md.m, 3 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].xm_kb, sb.x16, md.r, md.m, 3 * nbatch, 64, 128, true);
+          good = good && encode_map3(hm[i].xn_sw, sb.x16, md.r, md.n, 3 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].xn_kb, sb.x16, md.r, md.n, 3 * nbatch, 64, 128, true);
+          good = good && encode_map3(hm[i].rinv_sw, sb.rinv16, md.r, md.r, 3 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].phl_sw, sb.phl, md.r, md.m, 2 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].rt_sw, sb.rt16, md.r, md.r, 2 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].sq_sw, sb.sq16, md.r, md.r, 2 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].uh_sw, sb.uh16, md.n, md.r, 2 * c->K, 64, 64, true);
+          good = good && encode_map3(hm[i].wr_sw, sb.wr16, md.n, md.r, 2 * c->K, 64, 64, true);
+        }
       }
       if (good) {
         INIT_CUDA(cudaMemcpyAsync(c->d_maps, hm.data(), sizeof(TmaMatMaps) * nm, cudaMemcpyHostToDevice, st));

@@ -102,6 +102,10 @@ struct alignas(128) TmaMatMaps {
   // 64 x 64 swizzled boxes, and the three bf16 right-hand sides [batch][Kd][r]
   unsigned char e_kb[128], d_kb[128], d_sw[128], om16[128], pn16[128], zq16[128];
   unsigned char e_st[128], w_st[128];  // stores of one row group of the update epilogue
+  // refresh on tensor cores, all over hi|lo bf16 planes [2 x batch][rows][cols], 64 x 64 swizzled boxes
+  // unless noted: the matrix being orthonormalised with m rows and with n rows (also as 64 x 128 boxes,
+  // rows as MMA rows), R^-1, P, Rot^T, Rot^T o Rot^T, and the moment operands u^, v^ - u^ u^ as [r][n]
+  unsigned char xm_sw[128], xm_kb[128], xn_sw[128], xn_kb[128], rinv_sw[128], phl_sw[128], rt_sw[128], sq_sw[128], uh_sw[128], wr_sw[128];
 };
 struct alignas(128) TmaGradMaps {  // re-encoded whenever the caller's gradient pointer changes
   unsigned char g_sw[128], g_kb[128];
@@ -169,12 +173,39 @@ struct CopyProblem {
 void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long total_blocks, unsigned long long seed, long long index,
                                 cudaStream_t st);
 void launch_copy_grouped(const CopyProblem* probs, int nprobs, long long total_blocks, cudaStream_t st);
+// Element-wise preparation of tensor-core operands, many buffers per launch (1024 elements per block).
+// "Split" writes a value x as `planes` bf16 planes, plane p + 1 holding the rounding residual of the
+// planes before it (x ~ p0 + p1 (+ p2)), `plane` elements apart. Products of split operands sum the
+// plane pairs (0,0), (0,1), (1,0) [two planes: 16 bits of each operand] and (1,1), (0,2), (2,0)
+// [three planes: 24 bits, the accuracy of an fp32 product].
+enum ConvMode {
+  CONV_BF16 = 0,     // dst = bf16(src)
+  CONV_SPLIT = 1,    // dst = split(src)
+  CONV_STATES = 2,   // dst = split(u^ = inv_bc1 src), dst2 = split(inv_bc2 src2 - u^ u^)
+  CONV_ROT_T = 3,    // src is Rot [ld][ld]: dst = split(Rot^T), dst2 = split(Rot^T o Rot^T)
+  CONV_COMBINE = 4   // outf = bc1 src, outf2 = bc2 |src2 + src src|   (rotated moments from the two products)
+};
 struct ConvProblem {
   const float* src;
-  __nv_bfloat16* dst;
-  long long count, blk_start;  // 1024 elements per block
+  const float* src2;
+  __nv_bfloat16 *dst, *dst2;
+  float *outf, *outf2;
+  long long count, blk_start;  // count is a multiple of 8
+  long long plane;             // elements between the planes of dst and of dst2
+  int mode, ld, planes, pad;
 };
-void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long total_blocks, cudaStream_t st);
+void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long total_blocks, const GemmScalars& sc, cudaStream_t st);
+
+// Columns of X [rows][r] scaled to unit length (sums of squares in fp64), one block per 32 columns.
+// The tensor-core Gram matrix underestimates its diagonal (an fp32 accumulator that truncates, over
+// thousands of positive addends), which leaves every column of Q a few 1e-5 too long; the
+// off-diagonal part is already at fp32 level.
+struct NormProblem {
+  float* X;
+  long long blk_start;
+  int rows, r;
+};
+void launch_colnorm_grouped(const NormProblem* probs, int nprobs, long long total_blocks, cudaStream_t st);
 
 // Tensor-core sketch products of the refresh (lordo_tma.cu): C[M x r] (fp32) = S * B with the big
 // signal matrix S streamed by TMA as bf16 (optionally formed as c*G + E in shared memory) and
@@ -182,7 +213,10 @@ void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long tota
 struct SkProblem {
   long long tile_start;      // first 128-row tile of this problem within the launch
   int M, Kd, r, r_n;
-  int a_mn, a_c2, b_c2, pad;  // third TMA coordinate (worker / batch index) of A and of B
+  int a_mn, a_c2, b_c2;      // third TMA coordinate (worker / batch index) of A and of B
+  int split;                 // 0: one product; 2 or 3: operands split in that many bf16 planes, 3 or 6 passes over k
+  int a_pl, b_pl;            // third-coordinate distance between the planes of A and of B
+  int c_trans, pad;          // 1: C is stored transposed, C[col * ldc + row]
   const void* map_a;         // 64 x 64 swizzled boxes (a_mn) or 64 x 128 swizzled boxes
   const void* map_e;         // same shape over E, or null
   const void* map_b;         // 64 x 64 swizzled boxes over B [batch][Kd][r]

@@ -270,7 +270,17 @@ __global__ void __launch_bounds__(256) fill_random_grouped_kernel(const RandProb
 }
 
 // fp32 -> bf16 copies of many buffers in one launch (operands of the tensor-core sketch products)
-__global__ void __launch_bounds__(256) convert_grouped_kernel(const ConvProblem* __restrict__ probs, int nprobs) {
+__device__ __forceinline__ void split_store4(__nv_bfloat16* dst, long long plane, int planes, long long e, float4 v) {
+  for (int p = 0; p < planes; ++p) {
+    const float4 h = make_float4(__bfloat162float(__float2bfloat16_rn(v.x)), __bfloat162float(__float2bfloat16_rn(v.y)),
+                                 __bfloat162float(__float2bfloat16_rn(v.z)), __bfloat162float(__float2bfloat16_rn(v.w)));
+    store4(dst + p * plane, LORDO_BF16, e, h);
+    v = make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w);  // exact: the residual of a rounding to 8 bits
+  }
+}
+
+__global__ void __launch_bounds__(256) convert_grouped_kernel(const ConvProblem* __restrict__ probs, int nprobs, float inv_bc1, float inv_bc2,
+                                                              float bc1, float bc2) {
   const long long blk = blockIdx.x;
   int lo = 0, hi = nprobs - 1;
   while (lo < hi) {
@@ -280,8 +290,64 @@ __global__ void __launch_bounds__(256) convert_grouped_kernel(const ConvProblem*
   const ConvProblem pb = probs[lo];
   const long long e = ((blk - pb.blk_start) * 256 + threadIdx.x) * 4;  // count is a multiple of 8
   if (e >= pb.count) return;
+  if (pb.mode == CONV_ROT_T) {  // element e of the transposed matrix: (k, j) <- Rot[j][k]
+    float t[4];
+    for (int x = 0; x < 4; ++x) {
+      const long long k = (e + x) / pb.ld, j = (e + x) - k * pb.ld;
+      t[x] = pb.src[j * pb.ld + k];
+    }
+    split_store4(pb.dst, pb.plane, pb.planes, e, make_float4(t[0], t[1], t[2], t[3]));
+    split_store4(pb.dst2, pb.plane, pb.planes, e, make_float4(t[0] * t[0], t[1] * t[1], t[2] * t[2], t[3] * t[3]));
+    return;
+  }
   const float4 v = *reinterpret_cast<const float4*>(pb.src + e);
-  store4(pb.dst, LORDO_BF16, e, v);
+  if (pb.mode == CONV_BF16) {
+    store4(pb.dst, LORDO_BF16, e, v);
+  } else if (pb.mode == CONV_SPLIT) {
+    split_store4(pb.dst, pb.plane, pb.planes, e, v);
+  } else if (pb.mode == CONV_STATES) {
+    const float4 w = *reinterpret_cast<const float4*>(pb.src2 + e);
+    const float4 uh = make_float4(inv_bc1 * v.x, inv_bc1 * v.y, inv_bc1 * v.z, inv_bc1 * v.w);
+    split_store4(pb.dst, pb.plane, pb.planes, e, uh);
+    split_store4(pb.dst2, pb.plane, pb.planes, e,
+                 make_float4(inv_bc2 * w.x - uh.x * uh.x, inv_bc2 * w.y - uh.y * uh.y, inv_bc2 * w.z - uh.z * uh.z, inv_bc2 * w.w - uh.w * uh.w));
+  } else {  // CONV_COMBINE
+    const float4 w = *reinterpret_cast<const float4*>(pb.src2 + e);
+    *reinterpret_cast<float4*>(pb.outf + e) = make_float4(bc1 * v.x, bc1 * v.y, bc1 * v.z, bc1 * v.w);
+    *reinterpret_cast<float4*>(pb.outf2 + e) = make_float4(bc2 * fabsf(w.x + v.x * v.x), bc2 * fabsf(w.y + v.y * v.y),
+                                                           bc2 * fabsf(w.z + v.z * v.z), bc2 * fabsf(w.w + v.w * v.w));
+  }
+}
+
+__global__ void __launch_bounds__(256) colnorm_grouped_kernel(const NormProblem* __restrict__ probs, int nprobs) {
+  __shared__ double part[8][32];
+  const long long blk = blockIdx.x;
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].blk_start <= blk) lo = mid; else hi = mid - 1;
+  }
+  const NormProblem pb = probs[lo];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int col = (int)(blk - pb.blk_start) * 32 + lane;
+  const bool live = col < pb.r;
+  double s = 0.0;
+  if (live)
+    for (int row = w; row < pb.rows; row += 8) {
+      const float x = pb.X[(long long)row * pb.r + col];
+      s += (double)x * (double)x;
+    }
+  part[w][lane] = s;
+  __syncthreads();
+  if (w == 0) {
+    double t = 0.0;
+    for (int k = 0; k < 8; ++k) t += part[k][lane];
+    part[0][lane] = t > 0.0 ? 1.0 / sqrt(t) : 1.0;
+  }
+  __syncthreads();
+  const float sc = (float)part[0][lane];
+  if (live)
+    for (int row = w; row < pb.rows; row += 8) pb.X[(long long)row * pb.r + col] *= sc;
 }
 
 // Device-to-device copies of many buffers in one launch (16-byte chunks).
@@ -353,8 +419,11 @@ void launch_fill_random_grouped(const RandProblem* probs, int nprobs, long long 
                                 cudaStream_t st) {
   fill_random_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs, seed, index);
 }
-void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long total_blocks, cudaStream_t st) {
-  convert_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs);
+void launch_convert_grouped(const ConvProblem* probs, int nprobs, long long total_blocks, const GemmScalars& sc, cudaStream_t st) {
+  convert_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs, sc.inv_bc1, sc.inv_bc2, sc.bc1, sc.bc2);
+}
+void launch_colnorm_grouped(const NormProblem* probs, int nprobs, long long total_blocks, cudaStream_t st) {
+  colnorm_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs);
 }
 void launch_copy_grouped(const CopyProblem* probs, int nprobs, long long total_blocks, cudaStream_t st) {
   copy_grouped_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(probs, nprobs);

@@ -570,6 +570,7 @@ constexpr int kSStages = 3;
 constexpr uint32_t kSStageBytes = 65536;  // A 16 KB | E 16 KB | B up to 32 KB
 constexpr int kSThreads = (2 + 4 + 4) * 32;  // TMA, MMA, 4 transform warps, 4 epilogue warps
 constexpr uint32_t kIdescBMajorMN = 1u << 16;
+__device__ __forceinline__ int sk_passes(int split) { return split == 3 ? 6 : (split == 2 ? 3 : 1); }
 
 __device__ __forceinline__ int find_sk(const SkProblem* __restrict__ probs, int nprobs, long long tile) {
   int lo = 0, hi = nprobs - 1;
@@ -610,27 +611,30 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
       for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
         const int m0 = (int)(tile - pr->tile_start) * 128;
-        const int nkb = (pr->Kd + 63) / 64, nbox = (pr->r_n + 63) / 64;
+        const int nkb1 = (pr->Kd + 63) / 64, nbox = (pr->r_n + 63) / 64;
+        const int nkb = nkb1 * sk_passes(pr->split);
         const bool has_e = pr->map_e != nullptr;
         const uint32_t tx = 16384u + (has_e ? 16384u : 0u) + (uint32_t)nbox * 8192u;
-        for (int kb = 0; kb < nkb; ++kb, ++it) {
+        for (int j = 0; j < nkb; ++j, ++it) {
+          const int seg = j / nkb1, kb = j - seg * nkb1;  // plane pairs (0,0) (0,1) (1,0) (1,1) (0,2) (2,0)
+          const int a_c2 = pr->a_c2 + ((0x201100 >> (4 * seg)) & 3) * pr->a_pl, b_c2 = pr->b_c2 + ((0x021010 >> (4 * seg)) & 3) * pr->b_pl;
           const int s = it % ST;
           ok = mbar_wait(&empty_bar[s], ((it / ST) & 1u) ^ 1u, status);
           if (!ok) break;
           unsigned char* base = smem + s * SB;
           mbar_expect_tx(&full_bar[s], tx);
           if (pr->a_mn) {  // S stored [Kd][M]: two boxes of 64 k-rows x 64 columns
-            tma_load_3d(base, pr->map_a, m0, kb * 64, pr->a_c2, &full_bar[s]);
-            tma_load_3d(base + 8192, pr->map_a, m0 + 64, kb * 64, pr->a_c2, &full_bar[s]);
+            tma_load_3d(base, pr->map_a, m0, kb * 64, a_c2, &full_bar[s]);
+            tma_load_3d(base + 8192, pr->map_a, m0 + 64, kb * 64, a_c2, &full_bar[s]);
             if (has_e) {
-              tma_load_3d(base + 16384, pr->map_e, m0, kb * 64, pr->a_c2, &full_bar[s]);
-              tma_load_3d(base + 24576, pr->map_e, m0 + 64, kb * 64, pr->a_c2, &full_bar[s]);
+              tma_load_3d(base + 16384, pr->map_e, m0, kb * 64, a_c2, &full_bar[s]);
+              tma_load_3d(base + 24576, pr->map_e, m0 + 64, kb * 64, a_c2, &full_bar[s]);
             }
           } else {         // S stored [M][Kd]: one box of 128 rows x 64 k
-            tma_load_3d(base, pr->map_a, kb * 64, m0, pr->a_c2, &full_bar[s]);
-            if (has_e) tma_load_3d(base + 16384, pr->map_e, kb * 64, m0, pr->a_c2, &full_bar[s]);
+            tma_load_3d(base, pr->map_a, kb * 64, m0, a_c2, &full_bar[s]);
+            if (has_e) tma_load_3d(base + 16384, pr->map_e, kb * 64, m0, a_c2, &full_bar[s]);
           }
-          for (int j = 0; j < nbox; ++j) tma_load_3d(base + 32768 + j * 8192, pr->map_b, j * 64, kb * 64, pr->b_c2, &full_bar[s]);
+          for (int x = 0; x < nbox; ++x) tma_load_3d(base + 32768 + x * 8192, pr->map_b, x * 64, kb * 64, b_c2, &full_bar[s]);
         }
       }
     }
@@ -640,7 +644,7 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
       bool ok = true;
       for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++si) {
         const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
-        const int nkb = (pr->Kd + 63) / 64;
+        const int nkb = ((pr->Kd + 63) / 64) * sk_passes(pr->split);
         const bool a_mn = pr->a_mn != 0;
         const uint32_t n_lo = pr->r_n < 256 ? (uint32_t)pr->r_n : 256u, n_hi = (uint32_t)pr->r_n - n_lo;
         const uint32_t majors = kIdescBMajorMN | (a_mn ? kIdescAMajorMN : 0u);
@@ -671,7 +675,7 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
     bool ok = true;
     for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
-      const int nkb = (pr->Kd + 63) / 64;
+      const int nkb = ((pr->Kd + 63) / 64) * sk_passes(pr->split);
       const bool has_e = pr->map_e != nullptr;
       const float c = pr->cptr ? *pr->cptr : 1.f;
       for (int kb = 0; kb < nkb; ++kb, ++it) {
@@ -715,10 +719,14 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
       for (int ch = 0; ch < r_n / 16; ++ch) {
         float v[16];
         tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + buf * 256 + (uint32_t)(ch * 16), v);
-        if (row_ok) {
+        if (row_ok && !pr->c_trans) {
 #pragma unroll
           for (int j = 0; j < 16; j += 4)
             if (ch * 16 + j < r) *reinterpret_cast<float4*>(crow + ch * 16 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        } else if (row_ok) {  // transposed: the warp's lanes write 32 neighbouring floats of each output row
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (ch * 16 + j < r) pr->C[(long long)(ch * 16 + j) * pr->ldc + row] = v[j];
         }
       }
       tc_fence_before_sync();

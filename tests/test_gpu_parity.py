@@ -92,6 +92,9 @@ def test_nonfinite_gradient_sets_flag():
 # size, and so are u, sqrt(v) and the normalised update. The tolerances below are 8 * 2^-9 of the
 # largest entry for the states and the matching share of the weight movement for W.
 FAST_TOL = 8 * 2.0 ** -9
+# Fast mode with bf16 storage orthonormalises on tensor cores (operands split in three bf16 planes,
+# columns renormalised in fp32): P^T P = I is held to the same bound as on the fp32 path.
+TC_ORTH_TOL = 1e-5
 
 
 def _update_error(opt, orc, spec):
@@ -178,8 +181,8 @@ def test_fast_mode_no_error_feedback_fp32_and_bf16():
 
 
 def test_fast_mode_full_loop_with_refresh():
-    """Whole loop in fast mode. The refresh stays on the fp32 path, so each refresh, taken on the
-    CUDA path's own state, must match the oracle as tightly as in check mode."""
+    """Whole loop in fast mode with fp32 storage. The refresh then stays on the fp32 path, so each
+    refresh, taken on the CUDA path's own state, must match the oracle as tightly as in check mode."""
     wl = _small(m=264, n=200, r=32, K=2, H=2, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0)
     for variant, form in ((0, 2), (1, 1)):
         spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0)
@@ -203,7 +206,7 @@ def test_fast_mode_refresh_on_tensor_cores(variant, form, q, shape):
     spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0, eps=0.05)
     opt, orc, worst = hz.run_lockstep_refresh(spec)
     assert opt.poll_status() == 0
-    assert worst["P_orth"] < 1e-5 and abs(worst["energy"] - 1.0) < 1e-2, worst
+    assert worst["P_orth"] < TC_ORTH_TOL and abs(worst["energy"] - 1.0) < 1e-2, worst
     for t in list(opt.u) + list(opt.v) + list(opt.P):
         assert bool(torch.isfinite(t).all())
 
@@ -281,7 +284,7 @@ def test_refresh_warm_started_fast_mode_bf16():
         spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0, eps=0.05, warm_start=True)
         opt, orc, worst = hz.run_lockstep_refresh(spec)
         assert opt.poll_status() == 0
-        assert worst["P_orth"] < 1e-5 and abs(worst["energy"] - 1.0) < 1e-2, worst
+        assert worst["P_orth"] < TC_ORTH_TOL and abs(worst["energy"] - 1.0) < 1e-2, worst
 
 
 def test_rank_deficient_sketch_raises_flag_and_stays_finite():
@@ -448,6 +451,9 @@ def test_config4_full_size_fast_mode_sampled_columns():
     of one matrix per shape class one by one; the clip coefficients are checked against a plain
     torch reduction over all gradients."""
     from paper_2602_04396_b200 import lordo
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _total = torch.cuda.mem_get_info()
     if free < 125 * 2 ** 30:
         pytest.skip("needs about 120 GB of free device memory")
@@ -502,7 +508,7 @@ def test_config4_full_size_fast_mode_sampled_columns():
         assert bool((W == W[0:1]).all())  # every worker holds the broadcast model
         assert float((opt.X0[i] - W[0].float()).abs().max()) <= 2.0 ** -8 * float(opt.X0[i].abs().max())
         P = opt.P[i].double()
-        assert float((P.T @ P - torch.eye(P.shape[1], device="cuda", dtype=torch.float64)).abs().max()) < 1e-5
+        assert float((P.T @ P - torch.eye(P.shape[1], device="cuda", dtype=torch.float64)).abs().max()) < TC_ORTH_TOL
     opt.close()
 
 
@@ -519,6 +525,9 @@ def test_config4_full_size_fast_mode_repeatable():
     matrix of W, E, u, v after the inner steps and in every P after the refresh, and raise no flag.
     None of these kernels uses atomics on data, so any difference is a race between their roles."""
     from paper_2602_04396_b200 import lordo
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _total = torch.cuda.mem_get_info()
     if free < 125 * 2 ** 30:
         pytest.skip("needs about 120 GB of free device memory")
