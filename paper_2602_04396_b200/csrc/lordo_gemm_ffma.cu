@@ -249,11 +249,8 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
   const CholProblem pb = probs[blockIdx.x];
   const int r = pb.r;
   const float* __restrict__ A = pb.gram;
-  // Lt and X are written and re-read by different threads of the block: no __restrict__ and no const
-  // views of them, so that every load takes the coherent path (a read-only load could return a stale
-  // line holding the head of a row that was written after the line was fetched).
-  float* Lt = pb.lwork;
-  float* X = pb.rinv;
+  float* __restrict__ Lt = pb.lwork;  // distinct buffers; every other view of them below is derived from these
+  float* __restrict__ X = pb.rinv;
   const int t = threadIdx.x, nt = blockDim.x;
 
   if (t == 0) {
@@ -274,7 +271,7 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
     __syncthreads();
     // s_i = A[i][j] - sum_{k<j} L[i][k] L[j][k] for i >= j   (A is symmetric: row j is read)
     for (int i = j + t; i < r; i += nt) {
-      const float* col = Lt + i;
+      const float* col = Lt + i;  // derived from Lt (rows < j are final and were published by the barriers above)
       double s0 = (double)A[(long long)j * r + i], s1 = 0.0, s2 = 0.0, s3 = 0.0;
       int k = 0;
       for (; k + 4 <= j; k += 4) {
