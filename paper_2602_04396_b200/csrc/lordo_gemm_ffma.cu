@@ -238,12 +238,22 @@ void launch_gemm(const GemmProblem* probs, int nprobs, long long total_tiles, in
 
 // ---------------------------------------------------------------------------------------------
 // Cholesky of the Gram matrix + inverse of the triangular factor, one block per problem.
-// Left-looking column Cholesky with fp64 accumulation. The factor is kept TRANSPOSED in global
-// memory (Lt[k][i] = L[i][k], L2-resident) so that thread i's sweep over its own row of L reads
-// consecutive addresses across the block; the row of the pivot column is staged in shared memory.
+// Blocked left-looking Cholesky with fp64 accumulation, panels of 32 columns: a thread owns a row i
+// of L and keeps that row's 32 panel entries in registers; the contribution of the columns before
+// the panel is a rank-j0 update in which every value of L loaded from memory meets 32 values of a
+// 32 x 32 tile in shared memory, so that the column-by-column part (two barriers per column) is left
+// with at most 31 multiply-adds. The factor is kept TRANSPOSED in global memory (Lt[k][i] = L[i][k],
+// L2-resident) so that the threads' reads of their own rows are consecutive addresses.
+// L^-1 the same way with a thread per column: 32 rows of X at a time, the part below the panel's
+// diagonal block as a tile product, the block itself by substitution in registers.
 // ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int kCB = 32;
+}
+
 __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __restrict__ probs, unsigned* __restrict__ status) {
-  extern __shared__ float row_s[];  // r floats: row j of L (columns < j), later row i of L
+  __shared__ double tile[kCB][kCB + 1];  // [panel entry][k within the chunk]
+  __shared__ float dblk[kCB][kCB + 1];   // diagonal block of L, row-major
   __shared__ float pivot_s;
   __shared__ float maxdiag_s;
   const CholProblem pb = probs[blockIdx.x];
@@ -266,68 +276,136 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
   constexpr float kBreakdown = 3e-5f;
   const float abs_floor = maxdiag_s > 0.f ? maxdiag_s * 1e-12f : 1.f;
 
-  for (int j = 0; j < r; ++j) {
-    for (int k = t; k < j; k += nt) row_s[k] = Lt[(long long)k * r + j];  // L[j][k]
-    __syncthreads();
-    // s_i = A[i][j] - sum_{k<j} L[i][k] L[j][k] for i >= j   (A is symmetric: row j is read)
-    for (int i = j + t; i < r; i += nt) {
-      const float* col = Lt + i;  // derived from Lt (rows < j are final and were published by the barriers above)
-      double s0 = (double)A[(long long)j * r + i], s1 = 0.0, s2 = 0.0, s3 = 0.0;
-      int k = 0;
-      for (; k + 4 <= j; k += 4) {
-        const float l0 = col[(long long)k * r], l1 = col[(long long)(k + 1) * r], l2 = col[(long long)(k + 2) * r],
-                    l3 = col[(long long)(k + 3) * r];
-        s0 -= (double)l0 * (double)row_s[k];
-        s1 -= (double)l1 * (double)row_s[k + 1];
-        s2 -= (double)l2 * (double)row_s[k + 2];
-        s3 -= (double)l3 * (double)row_s[k + 3];
-      }
-      for (; k < j; ++k) s0 -= (double)col[(long long)k * r] * (double)row_s[k];
-      const double s = (s0 + s1) + (s2 + s3);
-      if (i == j) {
-        float d = (float)s;
-        const float floor_pivot = fmaxf(kBreakdown * A[(long long)j * r + j], abs_floor);
-        if (!(d > floor_pivot)) {  // also catches NaN
-          atomicOr(status, LORDO_FLAG_QR_BREAKDOWN);
-          d = floor_pivot;
+  for (int j0 = 0; j0 < r; j0 += kCB) {
+    const int nbw = r - j0 < kCB ? r - j0 : kCB;
+    for (int ib = j0; ib < r; ib += nt) {  // one pass unless r - j0 exceeds the block
+      const int i = ib + t;
+      const bool live = i < r;
+      // s_i[jj] = A[i][j0+jj] - sum_{k<j0} L[i][k] L[j0+jj][k]   (A is symmetric: row j0+jj is read)
+      double acc[kCB];
+#pragma unroll
+      for (int jj = 0; jj < kCB; ++jj) acc[jj] = (live && jj < nbw) ? (double)A[(long long)(j0 + jj) * r + i] : 0.0;
+      for (int k0 = 0; k0 < j0; k0 += kCB) {
+        __syncthreads();
+        for (int e = t; e < kCB * kCB; e += nt) {
+          const int jj = e / kCB, kk = e - jj * kCB;
+          tile[jj][kk] = jj < nbw ? (double)Lt[(long long)(k0 + kk) * r + j0 + jj] : 0.0;
         }
-        pivot_s = sqrtf(d);
+        __syncthreads();
+        if (live) {
+#pragma unroll 4
+          for (int kk = 0; kk < kCB; ++kk) {
+            const double l = (double)Lt[(long long)(k0 + kk) * r + i];
+#pragma unroll
+            for (int jj = 0; jj < kCB; ++jj) acc[jj] -= l * tile[jj][kk];
+          }
+        }
       }
-      Lt[(long long)j * r + i] = (float)s;  // unscaled for now; written and re-read by the same thread
+      if (ib == j0) {
+        // the chunk that holds the diagonal block: column by column, the finished column of the block
+        // published in shared memory for the multiply-adds of the columns after it
+#pragma unroll
+        for (int jj = 0; jj < kCB; ++jj) {
+          if (jj < nbw) {
+            const int j = j0 + jj;
+            if (live && i == j) {
+              float d = (float)acc[jj];
+              const float floor_pivot = fmaxf(kBreakdown * A[(long long)j * r + j], abs_floor);
+              if (!(d > floor_pivot)) {  // also catches NaN
+                atomicOr(status, LORDO_FLAG_QR_BREAKDOWN);
+                d = floor_pivot;
+              }
+              pivot_s = sqrtf(d);
+            }
+            __syncthreads();
+            const float piv = pivot_s;
+            float lij = 0.f;
+            if (live && i >= j) {
+              lij = (i == j) ? piv : (float)acc[jj] / piv;
+              Lt[(long long)j * r + i] = lij;
+              if (i < j0 + nbw) dblk[i - j0][jj] = lij;
+            }
+            __syncthreads();
+            if (live && i > j) {
+#pragma unroll
+              for (int j2 = jj + 1; j2 < kCB; ++j2)
+                if (j2 < nbw) acc[j2] -= (double)lij * (double)dblk[j2][jj];
+            }
+          }
+        }
+      } else {
+        // rows below the first chunk: the whole diagonal block is known
+        __syncthreads();
+        if (live) {
+#pragma unroll
+          for (int jj = 0; jj < kCB; ++jj) {
+            if (jj < nbw) {
+              const float lij = (float)acc[jj] / dblk[jj][jj];
+              Lt[(long long)(j0 + jj) * r + i] = lij;
+#pragma unroll
+              for (int j2 = jj + 1; j2 < kCB; ++j2)
+                if (j2 < nbw) acc[j2] -= (double)lij * (double)dblk[j2][jj];
+            }
+          }
+        }
+      }
     }
-    __syncthreads();
-    const float piv = pivot_s;
-    for (int i = j + t; i < r; i += nt) {
-      float* Lji = Lt + (long long)j * r + i;
-      *Lji = (i == j) ? piv : (*Lji / piv);
-    }
-    __syncthreads();
+    __syncthreads();  // the panel's columns are in memory for everybody
   }
 
-  // X = L^-1 (lower triangular), column c by thread c: X[i][c] = -(sum_{k=c}^{i-1} L[i][k] X[k][c]) / L[i][i].
-  // Row i of L is staged in shared memory for everybody; X[k][c] is read along rows (consecutive c).
+  // X = L^-1 (lower triangular), column c by thread c, 32 rows at a time:
+  // X[i][c] = ([i == c] - sum_{k<i} L[i][k] X[k][c]) / L[i][i], zero above the diagonal.
   for (int c = t; c < r; c += nt)
     for (int i = 0; i < r; ++i)
       if (i < c) X[(long long)i * r + c] = 0.f;
-  for (int i = 0; i < r; ++i) {
-    for (int k = t; k <= i; k += nt) row_s[k] = Lt[(long long)k * r + i];  // L[i][k]
-    __syncthreads();
-    for (int c = t; c <= i; c += nt) {
-      if (c == i) {
-        X[(long long)i * r + c] = 1.f / row_s[i];
-      } else {
-        double s0 = 0.0, s1 = 0.0;
-        int k = c;
-        for (; k + 2 <= i; k += 2) {
-          s0 += (double)row_s[k] * (double)X[(long long)k * r + c];
-          s1 += (double)row_s[k + 1] * (double)X[(long long)(k + 1) * r + c];
+  for (int i0 = 0; i0 < r; i0 += kCB) {
+    const int nbw = r - i0 < kCB ? r - i0 : kCB;
+    for (int cb = 0; cb < r; cb += nt) {
+      const int c = cb + t;
+      const bool live = c < r && c < i0 + nbw;  // columns right of the panel's last row are zero in it
+      double sum[kCB];
+#pragma unroll
+      for (int ii = 0; ii < kCB; ++ii) sum[ii] = 0.0;
+      for (int k0 = 0; k0 < i0; k0 += kCB) {
+        __syncthreads();
+        for (int e = t; e < kCB * kCB; e += nt) {
+          const int ii = e / kCB, kk = e - ii * kCB;
+          tile[ii][kk] = ii < nbw ? (double)Lt[(long long)(k0 + kk) * r + i0 + ii] : 0.0;
         }
-        for (; k < i; ++k) s0 += (double)row_s[k] * (double)X[(long long)k * r + c];
-        X[(long long)i * r + c] = (float)(-(s0 + s1) / (double)row_s[i]);
+        __syncthreads();
+        if (live && c < k0 + kCB) {  // X[k][c] = 0 for k < c
+#pragma unroll 4
+          for (int kk = 0; kk < kCB; ++kk) {
+            const double x = (double)X[(long long)(k0 + kk) * r + c];
+#pragma unroll
+            for (int ii = 0; ii < kCB; ++ii) sum[ii] += tile[ii][kk] * x;
+          }
+        }
+      }
+      __syncthreads();
+      for (int e = t; e < kCB * kCB; e += nt) {
+        const int ii = e / kCB, p = e - ii * kCB;
+        dblk[ii][p] = (ii < nbw && p <= ii) ? Lt[(long long)(i0 + p) * r + i0 + ii] : 0.f;
+      }
+      __syncthreads();
+      if (live) {
+        float xs[kCB];
+#pragma unroll
+        for (int ii = 0; ii < kCB; ++ii) {
+          xs[ii] = 0.f;
+          if (ii < nbw) {
+            const int i = i0 + ii;
+            double s = sum[ii];
+#pragma unroll
+            for (int p = 0; p < ii; ++p) s += (double)dblk[ii][p] * (double)xs[p];
+            xs[ii] = i < c ? 0.f : (float)(((i == c ? 1.0 : 0.0) - s) / (double)dblk[ii][ii]);
+            X[(long long)i * r + c] = xs[ii];
+          }
+        }
       }
     }
-    __syncthreads();
   }
+  __syncthreads();
   // R^-1 = (L^-1)^T : transpose X through Lt's storage (the factor is no longer needed)
   for (long long e = t; e < (long long)r * r; e += nt) Lt[e] = X[e];
   __syncthreads();
@@ -338,7 +416,8 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
 }
 
 void launch_chol_inverse(const CholProblem* probs, int nprobs, int r_max, unsigned* status, cudaStream_t st) {
-  chol_inverse_kernel<<<nprobs, 512, r_max * sizeof(float), st>>>(probs, status);
+  (void)r_max;
+  chol_inverse_kernel<<<nprobs, 512, 0, st>>>(probs, status);
 }
 
 }  // namespace lordo
