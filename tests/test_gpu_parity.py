@@ -23,6 +23,16 @@ def _small(m=200, n=136, r=24, K=3, H=2, rounds=2, grad="gauss", **kw):
     return synth.Workload(f"t{m}x{n}r{r}", ((m, n, r),), K=K, H=H, rounds=rounds, grad=grad, **kw)
 
 
+def test_init_state_rank_above_one_cholesky_block():
+    """r = 600: the Cholesky kernel's rows no longer fit one pass of its 512 threads, so the panels'
+    rows below the first chunk take the path that reads the finished diagonal block."""
+    spec = RunSpec(_small(m=1100, n=608, r=600, K=1), variant=0, rounds=0)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert st["P_orth"] < 1e-5 and st["P_angle"] < ANGLE_TOL and st["P_cols"] < 1e-5, st
+    assert opt.poll_status() == 0
+
+
 # ------------------------------------------------------------------ integer work: bit-exact
 
 @pytest.mark.parametrize("rows,cols", [(8, 8), (300, 24), (1000, 136)])
