@@ -31,6 +31,11 @@ Readings of points the paper leaves open (each is restated where it is used):
   R13 The error buffer is left untouched by a refresh; there is no weight decay.
   R14 Random matrices come from a counter-based integer generator (below): entries are
       popcount(64-bit word) - 32, i.e. centred Binomial(64, 1/2) integers, variance 16.
+  R15 Up-link time buffer (App. "Worker Communication", the server-side repacked updates): with
+      `time_buffer` every worker accumulates T <- T + eta * alpha, alpha being the low-rank update of
+      the step (no QHM or low-rank QHM only), and the pseudo-gradient of the synchronisation is
+      rebuilt as Delta = (1/M) sum_m Q^m T^m instead of being read off the weights; T is cleared
+      after every synchronisation. The basis must stay fixed between two synchronisations.
 
 Parity status: every function here is pinned by tests/test_oracle_pins.py against closed forms,
 invariants, library routines (torch.optim.Adam / SGD, numpy.linalg.svd / qr) or brute force.
@@ -253,6 +258,7 @@ class OracleConfig:
     e_dtype: str = "f32"
     state_dtype: str = "f32"  # u, v, P, X0, B, Delta
     warm_start: bool = False   # refresh by block power iteration from the current P (no sketch)
+    time_buffer: bool = False  # R15: pseudo-gradient rebuilt from the accumulated low-rank updates
 
 
 class LordoOracle:
@@ -264,6 +270,8 @@ class LordoOracle:
         self.s = 0  # moment updates done so far (R3)
         self.refreshes = 0
         self.W, self.E, self.P, self.u, self.v, self.X0, self.B, self.Delta = [], [], [], [], [], [], [], []
+        self.T = []  # R15: accumulated eta * alpha per worker, r x n
+        self.steps_in_round = 0
         self.last_clip = None
         self.last_mssv = None  # [n_mats][1 or K] MSSV of the last refresh that rotated (diagnostic)
         for i, (m, n, r) in enumerate(c.mats):
@@ -272,6 +280,7 @@ class LordoOracle:
             self.E.append(np.zeros((c.K, m, n)))
             self.u.append(np.zeros((c.K, r, n)))
             self.v.append(np.zeros((c.K, r, n)))
+            self.T.append(np.zeros((c.K, r, n)))
             self.X0.append(store(w0, c.state_dtype))
             self.B.append(np.zeros((m, n)))
             self.Delta.append(np.zeros((m, n)))
@@ -298,6 +307,9 @@ class LordoOracle:
         self.last_clip = coef
         bc1 = 1.0 - beta1 ** s
         bc2 = 1.0 - c.beta2 ** s
+        if c.time_buffer and form == QHM_FULL:
+            raise ValueError("the full-rank QHM update has no low-rank factorisation (R15)")
+        self.steps_in_round += 1
         for i, (m, n, r) in enumerate(c.mats):
             for k in range(c.K):
                 P = self._P(i, k)
@@ -314,15 +326,19 @@ class LordoOracle:
                 v_hat = self.v[i][k] / bc2
                 D = np.sqrt(v_hat) + c.eps
                 if form == QHM_NONE:
-                    upd = P @ (u_hat / D)
+                    alpha = u_hat / D
+                    upd = P @ alpha
                 elif form == QHM_LOW:
-                    upd = P @ ((omega * u_hat + (1.0 - omega) * g) / D)
+                    alpha = (omega * u_hat + (1.0 - omega) * g) / D
+                    upd = P @ alpha
                 elif form == QHM_FULL:
                     d = D.mean(axis=0)  # R6: mean over the rank axis, one value per column
                     upd = (1.0 - omega) * Ghat / d[None, :] + omega * (P @ (u_hat / D))  # R7
                 else:
                     raise ValueError(form)
                 self.W[i][k] = store(self.W[i][k] - lr * upd, c.w_dtype)
+                if c.time_buffer:
+                    self.T[i][k] = store(self.T[i][k] + lr * alpha, c.state_dtype)
 
     # -- Algorithm 1, the two state-synchronisation lines on their own (K_u, K_v != K_x) ------------
     def sync_states(self, sync_u: bool, sync_v: bool) -> None:
@@ -341,7 +357,11 @@ class LordoOracle:
                 self.u[i][:] = store(self.u[i].mean(axis=0), c.state_dtype)[None]
             if c.sync_v:
                 self.v[i][:] = store(self.v[i].mean(axis=0), c.state_dtype)[None]
-            delta = self.X0[i] - self.W[i].mean(axis=0)  # R9
+            if c.time_buffer:  # R15: (1/M) sum_m Q^m T^m
+                delta = np.mean([self._P(i, k) @ self.T[i][k] for k in range(c.K)], axis=0)
+                self.T[i][:] = 0.0
+            else:
+                delta = self.X0[i] - self.W[i].mean(axis=0)  # R9
             if c.outer == OUTER_AVG:
                 x_new = self.X0[i] - delta
             else:  # R10
@@ -350,10 +370,13 @@ class LordoOracle:
             self.Delta[i] = store(delta, c.state_dtype)
             self.X0[i] = store(x_new, c.state_dtype)
             self.W[i][:] = store(self.X0[i], c.w_dtype)[None]
+        self.steps_in_round = 0
 
     # -- ComputeProjection + moment rotation ------------------------------------------------------
     def refresh_subspace(self, G: Optional[Sequence[np.ndarray]] = None, beta1: float = 0.9) -> None:
         c = self.cfg
+        if c.time_buffer and self.steps_in_round > 0:
+            raise ValueError("the basis must stay fixed between two synchronisations (R15)")
         coef = None
         if c.variant == LOCAL:
             assert G is not None

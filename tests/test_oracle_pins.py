@@ -546,3 +546,70 @@ def test_sync_states_is_the_mean_over_workers():
     assert np.allclose(orc.u[0], mu[None]) and np.array_equal(orc.v[0], v_before)
     orc.sync_states(False, True)
     assert np.allclose(orc.v[0], v_before.mean(axis=0)[None])
+
+
+# ---------------------------------------------------------------------------------------------
+# Up-link time buffer (App. "Worker Communication"): the pseudo-gradient rebuilt from the low-rank
+# accumulators equals the one read off the weights, because every inner step moved the weights by
+# exactly eta * Q * alpha (App. "Extended Mathematical Derivations", the telescoped sum).
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("variant", [lo.GLOBAL, lo.LOCAL])
+@pytest.mark.parametrize("form", [lo.QHM_NONE, lo.QHM_LOW])
+def test_time_buffer_rebuilds_the_dense_pseudo_gradient(variant, form):
+    rng = np.random.default_rng(3)
+    mats = ((12, 10, 3), (9, 14, 4))
+    K, H = 3, 4
+    W0 = [rng.standard_normal((m, n)) for m, n, r in mats]
+    runs = []
+    for tb in (False, True):
+        cfg = lo.OracleConfig(mats=mats, K=K, H=H, variant=variant, state_dtype="f64", w_dtype="f64", e_dtype="f64", eps=1e-3,
+                              outer=lo.OUTER_NESTEROV, outer_lr=0.7, outer_momentum=0.9, time_buffer=tb)
+        orc = lo.LordoOracle(cfg, W0)
+        g_rng = np.random.default_rng(4)
+        for rnd in range(2):
+            for h in range(H):
+                G = [g_rng.standard_normal((K, m, n)) for m, n, r in mats]
+                if variant == lo.LOCAL and h == 0:
+                    orc.refresh_subspace(G, 0.9)
+                orc.inner_step(G, 0.01 * (h + 1), 0.9, 0.8, form)  # a different eta every step
+            orc.outer_step()
+            if variant == lo.GLOBAL:
+                orc.refresh_subspace(None, 0.9)
+        runs.append(orc)
+    dense, tb = runs
+    for i in range(len(mats)):
+        assert np.allclose(tb.Delta[i], dense.Delta[i], rtol=0, atol=1e-12)
+        assert np.allclose(tb.X0[i], dense.X0[i], rtol=0, atol=1e-12)
+        assert float(np.abs(tb.T[i]).max()) == 0.0  # cleared by the synchronisation
+
+
+def test_time_buffer_is_the_sum_of_eta_alpha():
+    """One worker, one matrix, no QHM: T after H steps = sum eta_t u^_t / (sqrt(v^_t) + eps), every term
+    recomputed here from the low-rank gradients of the run."""
+    rng = np.random.default_rng(8)
+    m, n, r, H = 7, 6, 2, 3
+    cfg = lo.OracleConfig(mats=((m, n, r),), K=1, H=H, variant=lo.GLOBAL, state_dtype="f64", w_dtype="f64", e_dtype="f64",
+                          error_feedback=False, eps=1e-2, beta2=0.95, time_buffer=True)
+    orc = lo.LordoOracle(cfg, [rng.standard_normal((m, n))])
+    P = orc.P[0].copy()
+    u = np.zeros((r, n)); v = np.zeros((r, n)); want = np.zeros((r, n))
+    for t in range(1, H + 1):
+        G = rng.standard_normal((1, m, n))
+        eta = 0.1 / t
+        orc.inner_step([G], eta, 0.9, 1.0, lo.QHM_NONE)
+        g = P.T @ G[0]
+        u = 0.9 * u + 0.1 * g
+        v = 0.95 * v + 0.05 * g * g
+        want += eta * (u / (1 - 0.9 ** t)) / (np.sqrt(v / (1 - 0.95 ** t)) + 1e-2)
+    assert np.allclose(orc.T[0][0], want, rtol=1e-12, atol=1e-14)
+
+
+def test_time_buffer_refuses_what_does_not_factorise():
+    cfg = lo.OracleConfig(mats=((6, 6, 2),), K=2, H=2, state_dtype="f64", w_dtype="f64", e_dtype="f64", time_buffer=True)
+    orc = lo.LordoOracle(cfg, [np.zeros((6, 6))])
+    G = [np.ones((2, 6, 6))]
+    with pytest.raises(ValueError):
+        orc.inner_step(G, 0.1, 0.9, 0.9, lo.QHM_FULL)
+    orc.inner_step(G, 0.1, 0.9, 0.9, lo.QHM_LOW)
+    with pytest.raises(ValueError):
+        orc.refresh_subspace(None, 0.9)  # the basis may not move inside a round
