@@ -103,6 +103,13 @@ typedef struct {
   int32_t warm_start;      /* 0: every refresh starts from a fresh random sketch; 1: block power iteration
                               started from the current P (max(power_iters, 1) iterations, no sketch), the
                               cheaper estimator the paper names as an alternative ComputeProjection */
+  int32_t time_buffer;     /* 1: the up-link time buffer of App. "Worker Communication": every worker accumulates
+                              T += eta * alpha (alpha = the step's low-rank update, r x n, workspace memory) and
+                              lordo_outer_step rebuilds the pseudo-gradient as (1/K) sum_k P_k T_k instead of
+                              reading it off the K weight replicas. Only the update forms without the full-rank
+                              term factorise: lordo_inner_step with LORDO_QHM_FULL returns LORDO_ERR_UNSUPPORTED.
+                              The basis does not move between two synchronisations (the call order that
+                              lordo_refresh_subspace enforces), which the factorisation needs. 0: off */
 } lordo_config;
 
 /* Host tables of device pointers, one entry per matrix. fp32 unless stated. */

@@ -131,6 +131,7 @@ struct lordo_ctx {
   std::vector<SketchBufs> h_skbufs;  // per matrix: bf16 right-hand sides of the sketch products (refresh scratch)
   PlanStep inner_proj, inner_apply;
   std::vector<PlanStep> refresh_steps, init_steps;
+  std::vector<PlanStep> tb_steps;  // Delta rebuilt from the time buffers (lordo_outer_step with time_buffer)
 
   // pinned host staging
   const void** h_Gtab = nullptr;  // pinned
@@ -205,6 +206,7 @@ int validate_config(const lordo_config* cfg, std::string& why) {
   if (!(cfg->beta2 >= 0.f && cfg->beta2 < 1.f) || !(cfg->eps >= 0.f)) { why = "beta2 or eps out of range"; return LORDO_ERR_INVALID_ARG; }
   if (cfg->power_iters < 0 || cfg->power_iters > 8) { why = "power_iters out of range (0..8)"; return LORDO_ERR_INVALID_ARG; }
   if (cfg->clip_scope != 0 && cfg->clip_scope != 1) { why = "clip_scope must be 0 or 1"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->time_buffer != 0 && cfg->time_buffer != 1) { why = "time_buffer must be 0 or 1"; return LORDO_ERR_INVALID_ARG; }
   for (int i = 0; i < cfg->n_mats; ++i) {
     const lordo_mat& a = cfg->mats[i];
     if (a.m < 1 || a.n < 1 || a.r < 1) { why = "non-positive shape"; return LORDO_ERR_SHAPE; }
@@ -303,6 +305,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     md.ghat = cv.take<float>((size_t)K * a.r * a.n);
     md.util = cv.take<float>((size_t)K * a.r * a.n);
     md.dcol = cv.take<float>((size_t)K * a.n);
+    md.T = cfg.time_buffer ? cv.take<float>((size_t)K * a.r * a.n) : nullptr;
     md.p_stride = local ? a.m * a.r : 0;
     if (real) {
       md.W = buf->W[i]; md.E = buf->E ? buf->E[i] : nullptr; md.P = buf->P[i]; md.u = buf->u[i]; md.v = buf->v[i];
@@ -352,6 +355,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         tp.gT16 = gT16 + (size_t)k * n_pad * r_k; tp.uT16 = uT16 + (size_t)k * n_pad * r_k;
         tp.u = md.u ? md.u + so : nullptr; tp.v = md.v ? md.v + so : nullptr;
         tp.dcol = md.dcol + (long long)k * md.n;
+        tp.tb = md.T ? md.T + so : nullptr;
         if (real) {
           tp.W = cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
           tp.E = md.E ? (cfg.e_dtype == LORDO_F32 ? (void*)((float*)md.E + wo) : (void*)((unsigned short*)md.E + wo)) : nullptr;
@@ -763,6 +767,24 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     flatten(R, c->refresh_steps);
     flatten(I, c->init_steps);
   }
+  // Up-link time buffer: Delta = P T_mean (Global, after the buffers were averaged) or the sum over
+  // the workers of P_k T_k (Local; the outer kernel divides by K), one grouped GEMM per term.
+  c->tb_steps.clear();
+  if (cfg.time_buffer) {
+    SlotBuilder TB;
+    for (int i = 0; i < n_mats; ++i) {
+      TB.rewind();
+      const MatDev& md = c->h_mats[i];
+      const int terms = local ? K : 1;
+      for (int k = 0; k < terms; ++k) {
+        Epilogue e = store_epi(md.Delta, md.n);
+        e.pad = k > 0;  // accumulate
+        TB.next(ST_GEMM, 0, 0, 0, 0).g.push_back(gemm_prob((int)md.m, (int)md.n, md.r, plain(md.P ? md.P + (long long)k * md.p_stride : nullptr, md.r),
+                                                            plain(md.T + (long long)k * md.r * md.n, md.n), nullptr, e));
+      }
+    }
+    flatten(TB, c->tb_steps);
+  }
   c->d_probs = cv.take<GemmProblem>(P.size());
   c->d_chols = cv.take<CholProblem>(c->h_chols.size() + 1);
   c->d_rands = cv.take<RandProblem>(c->h_rands.size() + 1);
@@ -1044,6 +1066,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
     if (md.E) INIT_CUDA(cudaMemsetAsync(md.E, 0, (size_t)c->K * wn * (c->cfg.e_dtype == LORDO_F32 ? 4 : 2), st));
     INIT_CUDA(cudaMemsetAsync(md.u, 0, sn * 4, st));
     INIT_CUDA(cudaMemsetAsync(md.v, 0, sn * 4, st));
+    if (md.T) INIT_CUDA(cudaMemsetAsync(md.T, 0, sn * 4, st));
     if (md.B) INIT_CUDA(cudaMemsetAsync(md.B, 0, wn * 4, st));
     INIT_CUDA(cudaMemsetAsync(md.Delta, 0, wn * 4, st));
     if (c->cfg.variant == LORDO_LOCAL) {
@@ -1071,6 +1094,8 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
   if (!c) return LORDO_ERR_INVALID_ARG;
   if (!G) return fail(c, LORDO_ERR_INVALID_ARG, "G is null");
   if (form != LORDO_QHM_NONE && form != LORDO_QHM_LOW && form != LORDO_QHM_FULL) return fail(c, LORDO_ERR_INVALID_ARG, "unknown QHM form");
+  if (c->cfg.time_buffer && form == LORDO_QHM_FULL)
+    return fail(c, LORDO_ERR_UNSUPPORTED, "time_buffer: the full-rank QHM update has no low-rank factorisation");
   if (!(beta1 >= 0.f && beta1 < 1.f) || !(omega >= 0.f && omega <= 1.f)) return fail(c, LORDO_ERR_INVALID_ARG, "beta1 or omega out of range");
   if (c->steps_in_round >= c->cfg.H) return fail(c, LORDO_ERR_STATE, "H inner steps done: lordo_outer_step is due");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
@@ -1181,20 +1206,32 @@ int lordo_outer_step(lordo_ctx* c, void* stream) {
   if (!c) return LORDO_ERR_INVALID_ARG;
   if (c->steps_in_round != c->cfg.H) return fail(c, LORDO_ERR_STATE, "lordo_outer_step needs exactly H inner steps since the last one");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-  const int which = (c->cfg.sync_u ? 1 : 0) | (c->cfg.sync_v ? 2 : 0);
+  const bool tb = c->cfg.time_buffer != 0, local = c->cfg.variant == LORDO_LOCAL;
+  const int which = (c->cfg.sync_u ? 1 : 0) | (c->cfg.sync_v ? 2 : 0) | ((tb && !local) ? 4 : 0);
   if (which) {
     ProfScope ps(c, st, PC_OUTER_STATES);
     launch_outer_states(c->d_mats, c->d_sblk_start, c->n_mats, c->total_sblks, c->K, which, st);
     c->launches += 1;
   }
+  int rc;
   {
     ProfScope ps(c, st, PC_OUTER_WEIGHTS);
+    if (tb) {  // Delta from the low-rank accumulators instead of the weight replicas
+      const GemmScalars gs = base_scalars(c);
+      for (const PlanStep& s : c->tb_steps) {
+        rc = run_plan_step(c, s, gs, st);
+        if (rc != LORDO_OK) return rc;
+      }
+    }
     launch_outer_weights(c->d_mats, c->d_wblk_start, c->n_mats, c->total_wblks, c->K, c->cfg.w_dtype, c->cfg.outer, c->cfg.outer_lr,
-                         c->cfg.outer_momentum, st);
+                         c->cfg.outer_momentum, tb ? (local ? 1.f / (float)c->K : 1.f) : 0.f, st);
   }
   c->launches += 1;
-  int rc = check_launch(c, "outer");
+  rc = check_launch(c, "outer");
   if (rc != LORDO_OK) return rc;
+  if (tb)
+    for (int i = 0; i < c->n_mats; ++i)
+      CUDA_OK(c, cudaMemsetAsync(c->h_mats[i].T, 0, sizeof(float) * (size_t)c->K * c->h_mats[i].r * c->h_mats[i].n, st));
   c->steps_in_round = 0;
   c->outers += 1;
   c->after_outer = true;

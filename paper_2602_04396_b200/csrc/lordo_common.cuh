@@ -28,6 +28,7 @@ struct MatDev {
   float* dcol;        // [K][n]    column scale of the full-rank QHM term (workspace)
   long long p_stride; // elements between the P of consecutive replicas (0 for Global)
   __nv_bfloat16* Delta16;  // [m][n] bf16 copy of Delta, made at the start of a Global refresh for the tensor-core sketch (workspace; may be null)
+  float* T;           // [K][r][n] up-link time buffer: sum over the round of lr * U~ (workspace; null unless enabled)
 };
 
 // Scalars of one inner step (Algorithm 1, per-step lines).

@@ -177,7 +177,13 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
     const long long row = m0 + ty * 4 + i;
     if (row >= M) break;
     if (ep.kind == EPI_STORE) {
-      *reinterpret_cast<float4*>(ep.C + row * ep.ldc + col) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+      float4* cp = reinterpret_cast<float4*>(ep.C + row * ep.ldc + col);
+      float4 o = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+      if (ep.pad) {  // accumulate into C
+        const float4 old = *cp;
+        o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+      }
+      *cp = o;
     } else if (ep.kind == EPI_APPLY) {
       if constexpr (DUAL) {
         const long long idx = row * (long long)N + col;

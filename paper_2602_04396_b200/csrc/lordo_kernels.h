@@ -35,7 +35,7 @@ enum EpilogueKind { EPI_STORE = 0, EPI_APPLY = 1, EPI_ROTATE = 2 };
 
 struct Epilogue {
   int kind, pad;
-  float* C;         // STORE: C[row*ldc + col] = acc
+  float* C;         // STORE: C[row*ldc + col] = acc (pad != 0: += acc)
   long long ldc;
   // APPLY (Algorithm 1: error-feedback line and the model update), row = weight row, col = column
   void* W;
@@ -91,6 +91,7 @@ struct TcProblem {
   long long G_off;             // element offset of this worker inside it
   const float* cptr;           // clip coefficient
   int mat, replica, pcopy, pad;  // matrix index, worker index, which copy of P (0 for Global)
+  float* tb;                   // [r][n] time buffer of this worker (+= lr * U~ every step), or null
 };
 
 // Tensor maps (opaque 128-byte objects encoded on the host) of one matrix for the TMA-fed kernels.
@@ -235,7 +236,7 @@ void launch_fill_float(float* p, long long count, float value, cudaStream_t st);
 void launch_moments(const MatDev* mats, const long long* tile_start, int n_mats, long long total_tiles, const StepScalars& sc,
                     cudaStream_t st);
 void launch_outer_weights(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int w_dt,
-                          int outer, float eta_s, float mu_s, cudaStream_t st);
+                          int outer, float eta_s, float mu_s, float delta_scale, cudaStream_t st);
 void launch_outer_states(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int which,
                          cudaStream_t st);
 void launch_init_weights(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int w_dt,

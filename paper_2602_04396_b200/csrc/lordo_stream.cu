@@ -132,6 +132,11 @@ __global__ void __launch_bounds__(256) moments_kernel(const MatDev* __restrict__
       *reinterpret_cast<float4*>(md.u + idx) = u;
       *reinterpret_cast<float4*>(md.v + idx) = v;
       *reinterpret_cast<float4*>(md.util + idx) = o;
+      if (md.T) {  // up-link time buffer
+        float4 tb = *reinterpret_cast<const float4*>(md.T + idx);
+        tb.x += sc.lr * o.x; tb.y += sc.lr * o.y; tb.z += sc.lr * o.z; tb.w += sc.lr * o.w;
+        *reinterpret_cast<float4*>(md.T + idx) = tb;
+      }
     }
   }
   if (sc.form == LORDO_QHM_FULL) {  // uniform over the grid
@@ -157,23 +162,29 @@ __global__ void __launch_bounds__(256) moments_kernel(const MatDev* __restrict__
 // One thread = 4 consecutive weights of one matrix, all K replicas.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) outer_weights_kernel(const MatDev* __restrict__ mats, const long long* __restrict__ blk_start,
-                                                            int n_mats, int K, int w_dt, int outer, float eta_s, float mu_s) {
+                                                            int n_mats, int K, int w_dt, int outer, float eta_s, float mu_s,
+                                                            float delta_scale) {
   const long long blk = blockIdx.x;
   const int i = find_segment(blk_start, n_mats, blk);
   const MatDev md = mats[i];
   const long long elems = md.m * md.n;
   const long long e = ((blk - blk_start[i]) * 256 + threadIdx.x) * 4;
   if (e >= elems) return;
-  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-  for (int k = 0; k < K; ++k) {
-    const float4 w = load4(md.W, w_dt, (long long)k * elems + e);
-    s.x += w.x; s.y += w.y; s.z += w.z; s.w += w.w;
-  }
-  const float inv_k = 1.f / (float)K;
   const float4 x0 = *reinterpret_cast<const float4*>(md.X0 + e);
   float4 d, xn;
-  d.x = x0.x - s.x * inv_k; d.y = x0.y - s.y * inv_k; d.z = x0.z - s.z * inv_k; d.w = x0.w - s.w * inv_k;
+  if (delta_scale != 0.f) {  // the pseudo-gradient was rebuilt from the time buffers into Delta
+    d = *reinterpret_cast<const float4*>(md.Delta + e);
+    d.x *= delta_scale; d.y *= delta_scale; d.z *= delta_scale; d.w *= delta_scale;
+  } else {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int k = 0; k < K; ++k) {
+      const float4 w = load4(md.W, w_dt, (long long)k * elems + e);
+      s.x += w.x; s.y += w.y; s.z += w.z; s.w += w.w;
+    }
+    const float inv_k = 1.f / (float)K;
+    d.x = x0.x - s.x * inv_k; d.y = x0.y - s.y * inv_k; d.z = x0.z - s.z * inv_k; d.w = x0.w - s.w * inv_k;
+  }
   if (outer == LORDO_OUTER_NESTEROV) {
     float4 b = *reinterpret_cast<const float4*>(md.B + e);
     b.x = mu_s * b.x + d.x; b.y = mu_s * b.y + d.y; b.z = mu_s * b.z + d.z; b.w = mu_s * b.w + d.w;
@@ -189,7 +200,8 @@ __global__ void __launch_bounds__(256) outer_weights_kernel(const MatDev* __rest
   for (int k = 0; k < K; ++k) store4(md.W, w_dt, (long long)k * elems + e, xn);
 }
 
-// u, v <- mean over replicas (Algorithm 1, "Sync u / v" lines). which: bit 0 = u, bit 1 = v.
+// u, v <- mean over replicas (Algorithm 1, "Sync u / v" lines). which: bit 0 = u, bit 1 = v,
+// bit 2 = the time buffers (Global rule: one basis, so their mean is all the rebuilt pseudo-gradient needs).
 __global__ void __launch_bounds__(256) outer_states_kernel(const MatDev* __restrict__ mats, const long long* __restrict__ blk_start,
                                                            int n_mats, int K, int which) {
   const long long blk = blockIdx.x;
@@ -199,9 +211,9 @@ __global__ void __launch_bounds__(256) outer_states_kernel(const MatDev* __restr
   const long long e = ((blk - blk_start[i]) * 256 + threadIdx.x) * 4;
   if (e >= elems) return;
   const float inv_k = 1.f / (float)K;
-  for (int t = 0; t < 2; ++t) {
+  for (int t = 0; t < 3; ++t) {
     if (!((which >> t) & 1)) continue;
-    float* p = t == 0 ? md.u : md.v;
+    float* p = t == 0 ? md.u : (t == 1 ? md.v : md.T);
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
     for (int k = 0; k < K; ++k) {
@@ -445,8 +457,8 @@ void launch_moments(const MatDev* mats, const long long* tile_start, int n_mats,
   moments_kernel<<<(unsigned)total_tiles, dim3(32, 8), 0, st>>>(mats, tile_start, n_mats, sc);
 }
 void launch_outer_weights(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int w_dt,
-                          int outer, float eta_s, float mu_s, cudaStream_t st) {
-  outer_weights_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(mats, blk_start, n_mats, K, w_dt, outer, eta_s, mu_s);
+                          int outer, float eta_s, float mu_s, float delta_scale, cudaStream_t st) {
+  outer_weights_kernel<<<(unsigned)total_blocks, 256, 0, st>>>(mats, blk_start, n_mats, K, w_dt, outer, eta_s, mu_s, delta_scale);
 }
 void launch_outer_states(const MatDev* mats, const long long* blk_start, int n_mats, long long total_blocks, int K, int which,
                          cudaStream_t st) {

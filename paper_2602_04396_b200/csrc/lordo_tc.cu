@@ -233,6 +233,7 @@ __global__ void __launch_bounds__(kProjThreads, 2) project_tc_kernel(const TcPro
             const size_t idx = (size_t)(unsigned)row * (size_t)n + (size_t)ecol;
             up_[idx] = un;
             vp_[idx] = vn;
+            if (prp->tb) prp->tb[idx] += sc.lr * o[t];
             dsum += D;
           } else {
             o[t] = 0.f;

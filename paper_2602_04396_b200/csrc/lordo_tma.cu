@@ -197,6 +197,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       const long long ecolc = e_ok ? ecol : (long long)n - 1;
       float* __restrict__ up_ = pr->u;
       float* __restrict__ vp_ = pr->v;
+      float* __restrict__ tb_ = pr->tb;
       // this column's 16-byte pieces inside the strip's block [r_k/8][128][8]
       const size_t lr_off = (size_t)(strip - pr->strip_start) * (size_t)r_k * 128 + (size_t)(q * 32 + lane) * 8;
       __nv_bfloat16* __restrict__ gT = pr->gT16 + lr_off;
@@ -233,6 +234,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
               const size_t idx = (size_t)(unsigned)row * (size_t)n + (size_t)ecol;
               up_[idx] = un;
               vp_[idx] = vn;
+              if (tb_) tb_[idx] += sc.lr * o[t];
               dsum += D;
             } else {
               o[t] = 0.f;

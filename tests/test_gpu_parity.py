@@ -566,6 +566,56 @@ def test_config4_full_size_fast_mode_repeatable():
     assert not differing, differing[:8]
 
 
+# ------------------------------------------------------------------ up-link time buffer
+
+@pytest.mark.parametrize("variant,form", [(0, 0), (0, 1), (1, 1)])
+def test_time_buffer_check_mode(variant, form):
+    """Pseudo-gradient rebuilt as (1/K) sum_k P_k T_k from the accumulated low-rank updates
+    (App. "Worker Communication"), both rules, against the oracle that does the same."""
+    wl = _small(m=264, n=200, r=32, K=3, H=3, rounds=2, grad="lowrank", signal_rank=8, clip_rho=30.0)
+    spec = RunSpec(wl, variant=variant, form=form, lr=0.01, omega=0.9, outer=1, outer_lr=0.7, outer_momentum=0.9, time_buffer=True)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert opt.poll_status() == 0
+    assert st["Delta"] < 1e-3 and st["X0"] < W_TOL and st["W"] < W_TOL and st["B"] < 1e-3, st
+    assert st["P_angle"] < ANGLE_TOL and st["u"] < 1e-3 and st["v"] < 1e-3, st
+
+
+def test_time_buffer_matches_dense_pseudo_gradient_on_device():
+    """fp32 storage, no refresh: the weights moved by exactly lr * P * alpha every step, so Delta from
+    the time buffers and Delta read off the weight replicas agree to fp32 rounding of the sums."""
+    wl = _small(m=320, n=264, r=72, K=3, H=4, rounds=1, clip_rho=30.0)
+    got = {}
+    for tb in (False, True):
+        spec = RunSpec(wl, variant=0, form=1, refresh=False, lr=0.01, omega=0.9, time_buffer=tb)
+        opt = hz.run_gpu(spec)
+        got[tb] = opt.Delta[0].double().cpu().numpy()
+        assert opt.poll_status() == 0
+    assert hz.scaled_error(got[True], got[False]) < 1e-4, hz.scaled_error(got[True], got[False])
+
+
+@pytest.mark.parametrize("w_dtype", ["f32", "bf16"])
+def test_time_buffer_fast_mode(w_dtype):
+    wl = _small(m=320, n=264, r=72, K=2, H=3, rounds=1, clip_rho=30.0, w_dtype=w_dtype, g_dtype=w_dtype, e_dtype=w_dtype)
+    spec = RunSpec(wl, variant=0, form=1, refresh=False, lr=0.01, omega=0.9, check_mode=0, eps=0.05, time_buffer=True)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert opt.poll_status() == 0
+    assert st["Delta"] < FAST_TOL and st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL, st
+
+
+def test_time_buffer_refuses_full_rank_qhm():
+    from paper_2602_04396_b200 import lordo
+    wl = _small(m=200, n=136, r=24, K=2, H=2, rounds=1)
+    spec = RunSpec(wl, variant=0, form=2, time_buffer=True)
+    opt = hz.make_gpu(spec)
+    G = hz.device_grads(wl, synth.gradients(wl, spec.seed, 0, 0))
+    with pytest.raises(lordo.LordoError):
+        opt.inner_step(G, 0.01, 0.9, 0.9, 2)
+    opt.inner_step(G, 0.01, 0.9, 0.9, 1)  # the low-rank form is accepted
+    opt.close()
+
+
 # ------------------------------------------------------------------ determinism and checkpoint / resume
 
 def _run_rounds_gpu(opt, wl, seed, rounds, first_round, variant, form, lr=0.01, beta1=0.9, omega=0.9):
