@@ -31,6 +31,10 @@ Readings of points the paper leaves open (each is restated where it is used):
   R13 The error buffer is left untouched by a refresh; there is no weight decay.
   R14 Random matrices come from a counter-based integer generator (below): entries are
       popcount(64-bit word) - 32, i.e. centred Binomial(64, 1/2) integers, variance 16.
+  R16 Oversampled sketch (`oversample` = p > 0): the range finder runs with r + p columns and the
+      basis is truncated to the top-r left singular subspace of its projection of the signal
+      (Rayleigh-Ritz), see compute_projection_rr. Not in the paper: the randomized-SVD refinement of
+      R1, closer to the paper's SVD definition of the projection at the same rank.
   R15 Up-link time buffer (App. "Worker Communication", the server-side repacked updates): with
       `time_buffer` every worker accumulates T <- T + eta * alpha, alpha being the low-rank update of
       the step (no QHM or low-rank QHM only), and the pseudo-gradient of the synchronisation is
@@ -185,6 +189,22 @@ def compute_projection(S: np.ndarray, Omega: np.ndarray, power_iters: int) -> np
     return Pn
 
 
+def compute_projection_rr(S: np.ndarray, Omega: np.ndarray, power_iters: int, r: int) -> np.ndarray:
+    """R16: range finder with an oversampled sketch (Omega is n x (r + p)) and Rayleigh-Ritz truncation
+    back to rank r. Q = the range finder's (r + p)-column basis; the top-r left singular subspace of
+    Q Q^T S is Q V_r, V_r the eigenvectors of the r largest eigenvalues of (Q^T S)(Q^T S)^T
+    (`numpy.linalg.eigh` serves as that step). A basis of a subspace is not unique, and the moments
+    live in the basis's coordinates, so the basis returned is fixed by the subspace alone:
+    P' = qr(Q M[:, :r]) with the projector M = V_r V_r^T."""
+    S = np.asarray(S, dtype=np.float64)
+    Q = compute_projection(S, Omega, power_iters)          # m x (r + p), orthonormal
+    Z = S.T @ Q                                            # n x (r + p)
+    lam, V = np.linalg.eigh(Z.T @ Z)                       # ascending eigenvalues
+    Vr = V[:, np.argsort(lam)[::-1][:r]]                   # (r + p) x r
+    M_r = Vr @ Vr[:r, :].T                                 # first r columns of the projector V_r V_r^T
+    return householder_qr_q(Q @ M_r)
+
+
 def compute_projection_warm(S: np.ndarray, P_old: np.ndarray, iters: int) -> np.ndarray:
     """Block power iteration started from the previous basis (the cheaper ComputeProjection the paper
     names, Sec. 2 "PowerSGD / block power iteration" and App. "Limitations"): `iters` >= 1 times
@@ -259,6 +279,7 @@ class OracleConfig:
     state_dtype: str = "f32"  # u, v, P, X0, B, Delta
     warm_start: bool = False   # refresh by block power iteration from the current P (no sketch)
     time_buffer: bool = False  # R15: pseudo-gradient rebuilt from the accumulated low-rank updates
+    oversample: int = 0        # R16: extra sketch columns p, Rayleigh-Ritz truncation back to rank r
 
 
 class LordoOracle:
@@ -387,8 +408,11 @@ class LordoOracle:
                 if c.warm_start:
                     P_new = store(compute_projection_warm(self.Delta[i], self.P[i], c.power_iters), c.state_dtype)
                 else:
-                    Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, 0, n, r)
-                    P_new = store(compute_projection(self.Delta[i], Om, c.power_iters), c.state_dtype)
+                    Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, 0, n, r + c.oversample)
+                    if c.oversample:
+                        P_new = store(compute_projection_rr(self.Delta[i], Om, c.power_iters, r), c.state_dtype)
+                    else:
+                        P_new = store(compute_projection(self.Delta[i], Om, c.power_iters), c.state_dtype)
                 diag[i].append(mssv(P_new, self.P[i]))
                 if self.s > 0:
                     for k in range(c.K):
@@ -404,8 +428,11 @@ class LordoOracle:
                     if c.warm_start:
                         P_new = store(compute_projection_warm(S, self.P[i][k], c.power_iters), c.state_dtype)
                     else:
-                        Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, n, r)
-                        P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
+                        Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, n, r + c.oversample)
+                        if c.oversample:
+                            P_new = store(compute_projection_rr(S, Om, c.power_iters, r), c.state_dtype)
+                        else:
+                            P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
                     diag[i].append(mssv(P_new, self.P[i][k]))
                     if self.s > 0:
                         un, vn = rotate_moments(self.u[i][k], self.v[i][k], P_new, self.P[i][k], beta1, c.beta2, self.s)

@@ -613,3 +613,58 @@ def test_time_buffer_refuses_what_does_not_factorise():
     orc.inner_step(G, 0.1, 0.9, 0.9, lo.QHM_LOW)
     with pytest.raises(ValueError):
         orc.refresh_subspace(None, 0.9)  # the basis may not move inside a round
+
+
+# ---------------------------------------------------------------------------------------------
+# R16: oversampled sketch with Rayleigh-Ritz truncation.
+# ---------------------------------------------------------------------------------------------
+def _angle(A, B):
+    s = np.linalg.svd(np.linalg.qr(A)[0].T @ np.linalg.qr(B)[0], compute_uv=False)
+    return float(np.arccos(np.clip(s.min(), -1.0, 1.0)))
+
+
+def test_rayleigh_ritz_is_the_truncated_svd_of_the_projected_signal():
+    """The returned basis spans the top-r left singular vectors of Q Q^T S (numpy's SVD of that matrix)."""
+    rng = np.random.default_rng(21)
+    m, n, r, p = 40, 30, 5, 4
+    S = rng.standard_normal((m, n)) * (0.7 ** np.arange(n))[None, :]
+    Om = rng.standard_normal((n, r + p))
+    Q = lo.compute_projection(S, Om, 1)
+    U = np.linalg.svd(Q @ (Q.T @ S))[0][:, :r]
+    P = lo.compute_projection_rr(S, Om, 1, r)
+    assert P.shape == (m, r)
+    assert np.abs(P.T @ P - np.eye(r)).max() < 1e-12
+    assert _angle(P, U) < 1e-6
+
+
+def test_rayleigh_ritz_recovers_an_exact_rank_r_range_and_beats_the_plain_sketch():
+    rng = np.random.default_rng(22)
+    m, n, r, p = 36, 28, 4, 4
+    L = np.linalg.qr(rng.standard_normal((m, r)))[0]
+    S0 = L @ rng.standard_normal((r, n))
+    Om = rng.standard_normal((n, r + p))
+    assert _angle(lo.compute_projection_rr(S0, Om, 0, r), L) < 1e-7  # exact rank r: the range itself
+    # rank r signal + noise: energy captured by r columns, oversampled + truncated vs r-column sketch
+    S = S0 + 0.2 * rng.standard_normal((m, n))
+    P_rr = lo.compute_projection_rr(S, Om, 0, r)
+    P_pl = lo.compute_projection(S, Om[:, :r], 0)
+    e_rr, e_pl = np.linalg.norm(P_rr.T @ S), np.linalg.norm(P_pl.T @ S)
+    e_best = np.sqrt((np.linalg.svd(S, compute_uv=False)[:r] ** 2).sum())
+    assert e_pl < e_rr <= e_best * (1 + 1e-12)
+
+
+def test_rayleigh_ritz_basis_depends_on_the_subspace_only():
+    """Any orthonormal basis of the same (r + p)-dimensional range gives the same P: the eigenvectors'
+    signs and order, which a solver is free to choose, do not show in the result."""
+    rng = np.random.default_rng(23)
+    m, n, r, p = 30, 24, 4, 3
+    S = rng.standard_normal((m, n)) * (0.6 ** np.arange(n))[None, :]
+    Om = rng.standard_normal((n, r + p))
+    P1 = lo.compute_projection_rr(S, Om, 0, r)
+    # the same steps with the eigenvectors negated and taken in another order
+    Q = lo.compute_projection(S, Om, 0)
+    Z = S.T @ Q
+    lam, V = np.linalg.eigh(Z.T @ Z)
+    Vr = -V[:, np.argsort(lam)[::-1][:r]][:, ::-1]
+    P2 = lo.householder_qr_q(Q @ (Vr @ Vr[:r, :].T))
+    assert np.abs(P1 - P2).max() < 1e-10
