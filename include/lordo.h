@@ -110,6 +110,11 @@ typedef struct {
                               term factorise: lordo_inner_step with LORDO_QHM_FULL returns LORDO_ERR_UNSUPPORTED.
                               The basis does not move between two synchronisations (the call order that
                               lordo_refresh_subspace enforces), which the factorisation needs. 0: off */
+  int32_t oversample;      /* p >= 0, a multiple of 8: the range finder of the refresh runs with r + p columns and its
+                              basis is truncated to the top-r left singular subspace of its projection of the
+                              signal (Rayleigh-Ritz; not in the paper, the randomized-SVD refinement of the range
+                              finder). The refresh then runs in fp32 in both modes. Needs r + p <= min(m, n) and
+                              <= 600 for every matrix and warm_start = 0. 0: off */
 } lordo_config;
 
 /* Host tables of device pointers, one entry per matrix. fp32 unless stated. */

@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kMaxK = 64;
 
-enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3, ST_SKETCH = 4, ST_CONVERT = 5, ST_NORM = 6 };
+enum StepType { ST_GEMM = 0, ST_CHOL = 1, ST_RANDOM = 2, ST_COPY = 3, ST_SKETCH = 4, ST_CONVERT = 5, ST_NORM = 6, ST_EIG = 7 };
 enum Phase { PH_SUBSPACE = 0, PH_ROTATE = 1, PH_COMMIT = 2 };
 
 // One launch of the refresh / init / inner-step plans. The entries it works on are a contiguous
@@ -41,6 +41,7 @@ struct SlotBuilder {
     std::vector<SkProblem> sk;
     std::vector<ConvProblem> cv;
     std::vector<NormProblem> nm;
+    std::vector<EigProblem> eg;
   };
   std::vector<Slot> slots;
   size_t cur = 0;
@@ -91,6 +92,7 @@ struct lordo_ctx {
   SkProblem* d_sks = nullptr;
   ConvProblem* d_convs = nullptr;
   NormProblem* d_norms = nullptr;
+  EigProblem* d_eigs = nullptr;
   float* d_scratch = nullptr;
   long long total_chunks = 0, total_mom_tiles = 0, total_wblks = 0, total_sblks = 0;
 
@@ -123,6 +125,7 @@ struct lordo_ctx {
   DiagProblem* d_diag = nullptr;
   std::vector<ConvProblem> h_convs;
   std::vector<NormProblem> h_norms;
+  std::vector<EigProblem> h_eigs;
   struct SketchBufs {
     __nv_bfloat16 *om16 = nullptr, *pn16 = nullptr, *zq16 = nullptr;
     // hi|lo planes of the tensor-core QR and rotation (null when those run in fp32)
@@ -207,11 +210,17 @@ int validate_config(const lordo_config* cfg, std::string& why) {
   if (cfg->power_iters < 0 || cfg->power_iters > 8) { why = "power_iters out of range (0..8)"; return LORDO_ERR_INVALID_ARG; }
   if (cfg->clip_scope != 0 && cfg->clip_scope != 1) { why = "clip_scope must be 0 or 1"; return LORDO_ERR_INVALID_ARG; }
   if (cfg->time_buffer != 0 && cfg->time_buffer != 1) { why = "time_buffer must be 0 or 1"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->oversample < 0 || cfg->oversample % 8 != 0) { why = "oversample must be a non-negative multiple of 8"; return LORDO_ERR_INVALID_ARG; }
+  if (cfg->oversample > 0 && cfg->warm_start) { why = "oversample needs a fresh sketch: warm_start must be 0"; return LORDO_ERR_UNSUPPORTED; }
   for (int i = 0; i < cfg->n_mats; ++i) {
     const lordo_mat& a = cfg->mats[i];
     if (a.m < 1 || a.n < 1 || a.r < 1) { why = "non-positive shape"; return LORDO_ERR_SHAPE; }
     if (a.n % 8 != 0 || a.r % 8 != 0) { why = "n and r must be multiples of 8"; return LORDO_ERR_ALIGN; }
     if (a.r > a.m || a.r > a.n) { why = "r must not exceed min(m, n)"; return LORDO_ERR_SHAPE; }
+    if (cfg->oversample > 0 && (a.r + cfg->oversample > a.m || a.r + cfg->oversample > a.n || a.r + cfg->oversample > 600)) {
+      why = "r + oversample must not exceed min(m, n) nor 600";
+      return LORDO_ERR_SHAPE;
+    }
     if (a.r > 4096) { why = "r above 4096 is not supported"; return LORDO_ERR_UNSUPPORTED; }
   }
   return LORDO_OK;
@@ -273,8 +282,10 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       const lordo_mat& a = cfg.mats[i];
       const long long maxd = a.m > a.n ? a.m : a.n;
       const size_t nb = local ? K : 1;
-      size_t per = (size_t)a.n * a.r + 2 * (size_t)a.m * a.r + (size_t)maxd * a.r + (q > 0 ? 2 * (size_t)a.n * a.r : 0) +
-                   4 * (size_t)a.r * a.r;
+      const size_t rs = (size_t)a.r + cfg.oversample;  // columns of the sketch and of everything up to the truncation
+      size_t per = (size_t)a.n * rs + 2 * (size_t)a.m * rs + (size_t)maxd * rs + ((q > 0 || cfg.oversample > 0) ? 2 * (size_t)a.n * rs : 0) +
+                   4 * rs * rs;
+      if (cfg.oversample > 0) per += 3 * rs * rs + rs * a.r;  // eigen-solver work and the truncating projector
       // bf16 right-hand sides of the tensor-core sketch products (Omega, P', Z), counted in floats
       per += ((size_t)a.n * a.r + (q > 0 ? (size_t)a.m * a.r + (size_t)a.n * a.r : 0)) / 2 + 64;
       size_t states16 = 0;
@@ -382,9 +393,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
 
   // ---------------- launch plans ----------------
   std::vector<GemmProblem>& P = c->h_probs;
-  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear(); c->h_norms.clear(); c->h_diag.clear();
+  P.clear(); c->h_chols.clear(); c->h_rands.clear(); c->h_copies.clear(); c->h_sks.clear(); c->h_convs.clear(); c->h_norms.clear(); c->h_eigs.clear(); c->h_diag.clear();
   c->h_skbufs.assign(n_mats, lordo_ctx::SketchBufs());
-  const bool tc_sketch = c->tc && c->tma;  // sketch products of the refresh on tensor cores
+  const bool tc_sketch = c->tc && c->tma && cfg.oversample == 0;  // products of the refresh on tensor cores
   auto gemm_prob = [&](int M, int N, int Kd, const Operand& A, const Operand& B, const Operand* B2, const Epilogue& ep) {
     GemmProblem g;
     std::memset(&g, 0, sizeof(g));
@@ -424,6 +435,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       } else if (st.type == ST_CONVERT) {
         st.first = (long long)c->h_convs.size(); st.count = (int)sl.cv.size(); st.tiles = 0;
         for (ConvProblem& x : sl.cv) { x.blk_start = st.tiles; st.tiles += (x.count + 1023) / 1024; c->h_convs.push_back(x); }
+      } else if (st.type == ST_EIG) {
+        st.first = (long long)c->h_eigs.size(); st.count = (int)sl.eg.size(); st.r_max = 0;
+        for (const EigProblem& x : sl.eg) { if (x.w > st.r_max) st.r_max = x.w; c->h_eigs.push_back(x); }
       } else if (st.type == ST_NORM) {
         st.first = (long long)c->h_norms.size(); st.count = (int)sl.nm.size(); st.tiles = 0;
         for (NormProblem& x : sl.nm) { x.blk_start = st.tiles; st.tiles += (x.r + 31) / 32; c->h_norms.push_back(x); }
@@ -520,16 +534,20 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       // scratch carve of this matrix inside its group (batch-strided arrays)
       float* s = c->d_scratch + goff;
       goff += mat_scratch[i];
-      float* Om = s; s += (size_t)nb * n * r;
-      float* Ya = s; s += (size_t)nb * m * r;
-      float* Pn = s; s += (size_t)nb * m * r;
-      float* Yb = s; s += (size_t)nb * maxd * r;
+      const bool rr = cfg.oversample > 0;  // oversampled sketch, Rayleigh-Ritz truncation back to r columns
+      const int rs = r + cfg.oversample;   // equals r on the tensor-core path
+      float* Om = s; s += (size_t)nb * n * rs;
+      float* Ya = s; s += (size_t)nb * m * rs;
+      float* Pn = s; s += (size_t)nb * m * rs;
+      float* Yb = s; s += (size_t)nb * maxd * rs;
       float *Za = nullptr, *Zq = nullptr;
-      if (q > 0) { Za = s; s += (size_t)nb * n * r; Zq = s; s += (size_t)nb * n * r; }
-      float* gram = s; s += (size_t)nb * r * r;
-      float* lw = s; s += (size_t)nb * r * r;
-      float* rinv = s; s += (size_t)nb * r * r;
-      float* rot = s; s += (size_t)nb * r * r;
+      if (q > 0 || rr) { Za = s; s += (size_t)nb * n * rs; Zq = s; s += (size_t)nb * n * rs; }
+      float* gram = s; s += (size_t)nb * rs * rs;
+      float* lw = s; s += (size_t)nb * rs * rs;
+      float* rinv = s; s += (size_t)nb * rs * rs;
+      float* rot = s; s += (size_t)nb * rs * rs;
+      float *eigw = nullptr, *mr = nullptr;
+      if (rr) { eigw = s; s += (size_t)nb * 3 * rs * rs; mr = s; s += (size_t)nb * rs * r; }
       __nv_bfloat16* om16 = reinterpret_cast<__nv_bfloat16*>(s); s += ((size_t)nb * n * r) / 2 + 16;
       __nv_bfloat16 *pn16 = nullptr, *zq16 = nullptr;
       if (q > 0) {
@@ -606,9 +624,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           nr.nm.push_back(np);
         }
       };
-      auto qr2 = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows) {
+      auto qr2 = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows, int w) {
         if (tc_sketch) cholqr2_tc(sb, phase, X, sx, T, st, O, so, rows);
-        else cholqr2(sb, phase, X, sx, T, st, O, so, rows, r, nb, gram, lw, rinv);
+        else cholqr2(sb, phase, X, sx, T, st, O, so, rows, w, nb, gram, lw, rinv);
       };
       // S * B on tensor cores: a_mn = 0 -> S rows are the output rows (Y = S B), 1 -> S^T B
       auto sketch = [&](SlotBuilder& sb, int a_mn, unsigned char* map_b, float* C, long long cstride, long long Mo, long long Kd) {
@@ -658,9 +676,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& f = R.next(ST_RANDOM, PH_SUBSPACE);
           for (int b = 0; b < nb; ++b) {
             RandProblem rp;
-            rp.out = tc_sketch ? nullptr : Om + (long long)b * n * r;
+            rp.out = tc_sketch ? nullptr : Om + (long long)b * n * rs;
             rp.out16 = tc_sketch ? om16 + (long long)b * n * r : nullptr;
-            rp.count = n * r; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
+            rp.count = n * rs; rp.blk_start = 0; rp.purpose = 2; rp.mat = i; rp.replica = local ? b : 0; rp.pad = 0;
             f.rn.push_back(rp);
           }
         }
@@ -669,9 +687,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           sketch(R, 0, (c->d_maps + i)->om16, Ya, m * r, m, n);
         } else {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
-          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Om + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, rs, (int)n, signal(b), plain(Om + (long long)b * n * rs, rs), nullptr, store_epi(Ya + (long long)b * m * rs, rs)));
         }
-        qr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m);
+        qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs);
       }
       for (int it = 0; it < q; ++it) {
         if (tc_sketch) {  // Z = S^T P'
@@ -679,17 +697,42 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           sketch(R, 1, (c->d_maps + i)->pn16, Za, n * r, n, m);
         } else {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
-          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, r, (int)m, signal(b), plain(Pn + (long long)b * m * r, r), nullptr, store_epi(Za + (long long)b * n * r, r)));
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, rs, (int)m, signal(b), plain(Pn + (long long)b * m * rs, rs), nullptr, store_epi(Za + (long long)b * n * rs, rs)));
         }
-        qr2(R, PH_SUBSPACE, Za, n * r, Yb, maxd * r, Zq, n * r, n);
+        qr2(R, PH_SUBSPACE, Za, n * rs, Yb, maxd * rs, Zq, n * rs, n, rs);
         if (tc_sketch) {  // Y = S Z
           convert(R, Zq, zq16, (size_t)nb * n * r);
           sketch(R, 0, (c->d_maps + i)->zq16, Ya, m * r, m, n);
         } else {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
-          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, (int)n, signal(b), plain(Zq + (long long)b * n * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, rs, (int)n, signal(b), plain(Zq + (long long)b * n * rs, rs), nullptr, store_epi(Ya + (long long)b * m * rs, rs)));
         }
-        qr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m);
+        qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs);
+      }
+      if (rr) {
+        // Rayleigh-Ritz truncation of the (r + p)-column basis Q (in Pn): Z = S^T Q, C = Z^T Z, the
+        // projector onto the r leading eigenvectors of C, P' = qr(Q M[:, :r])
+        {
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, rs, (int)m, signal(b), plain(Pn + (long long)b * m * rs, rs), nullptr, store_epi(Za + (long long)b * n * rs, rs)));
+        }
+        {
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob(rs, rs, (int)n, plain(Za + (long long)b * n * rs, rs), plain(Za + (long long)b * n * rs, rs), nullptr, store_epi(gram + (long long)b * rs * rs, rs)));
+        }
+        {
+          SlotBuilder::Slot& e = R.next(ST_EIG, PH_SUBSPACE);
+          for (int b = 0; b < nb; ++b) {
+            EigProblem ep;
+            ep.C = gram + (long long)b * rs * rs; ep.work = eigw + (long long)b * 3 * rs * rs; ep.Mr = mr + (long long)b * rs * r; ep.w = rs; ep.r = r;
+            e.eg.push_back(ep);
+          }
+        }
+        {
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
+          for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, r, rs, plain(Pn + (long long)b * m * rs, rs), plain(mr + (long long)b * rs * r, r), nullptr, store_epi(Ya + (long long)b * m * r, r)));
+        }
+        qr2(R, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, Pn, m * r, m, r);
       }
       for (int b = 0; b < nb; ++b) {
         DiagProblem dp;
@@ -792,6 +835,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   c->d_sks = cv.take<SkProblem>(c->h_sks.size() + 1);
   c->d_convs = cv.take<ConvProblem>(c->h_convs.size() + 1);
   c->d_norms = cv.take<NormProblem>(c->h_norms.size() + 1);
+  c->d_eigs = cv.take<EigProblem>(c->h_eigs.size() + 1);
   c->d_diag = cv.take<DiagProblem>(c->h_diag.size() + 1);
 
   c->last_G.assign(n_mats, nullptr);
@@ -863,6 +907,10 @@ int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t 
       launch_convert_grouped(c->d_convs + s.first, s.count, s.tiles, sc, st);
       c->launches += 1;
       return check_launch(c, "convert");
+    case ST_EIG:
+      launch_jacobi_projector(c->d_eigs + s.first, s.count, s.r_max, st);
+      c->launches += 1;
+      return check_launch(c, "jacobi_projector");
     case ST_NORM:
       launch_colnorm_grouped(c->d_norms + s.first, s.count, s.tiles, st);
       c->launches += 1;
@@ -992,6 +1040,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   if (!c->h_diag.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_diag, c->h_diag.data(), sizeof(DiagProblem) * c->h_diag.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_convs.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_convs, c->h_convs.data(), sizeof(ConvProblem) * c->h_convs.size(), cudaMemcpyHostToDevice, st));
   if (!c->h_norms.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_norms, c->h_norms.data(), sizeof(NormProblem) * c->h_norms.size(), cudaMemcpyHostToDevice, st));
+  if (!c->h_eigs.empty()) INIT_CUDA(cudaMemcpyAsync(c->d_eigs, c->h_eigs.data(), sizeof(EigProblem) * c->h_eigs.size(), cudaMemcpyHostToDevice, st));
   INIT_CUDA(cudaMemsetAsync(c->d_status, 0, 256, st));
   if (c->tc) {
     if (!c->tma) INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));  // register-staged kernels (fp32 storage)

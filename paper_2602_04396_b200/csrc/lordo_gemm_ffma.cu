@@ -421,6 +421,127 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Parallel cyclic Jacobi eigen-solver of a small symmetric matrix + the projector it is wanted for.
+// A sweep is w - 1 steps (w made even with a dummy index); a step rotates w/2 disjoint index pairs
+// (round-robin tournament order). Rotations of disjoint pairs commute, so a step is
+//   C <- J^T C J,  V^T <- J^T V^T,  J = product of the step's plane rotations,
+// done row by row: a warp forms row i of J^T C from rows i and partner(i) (coalesced reads), keeps
+// it in shared memory, applies the column rotations there and writes row i of the new matrix.
+// Old and new matrices are separate buffers, swapped after every step.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512) jacobi_projector_kernel(const EigProblem* __restrict__ probs) {
+  extern __shared__ float jsm[];
+  const EigProblem pb = probs[blockIdx.x];
+  const int w = pb.w, r = pb.r;
+  const int we = (w + 1) & ~1;           // even number of players
+  float* cc = jsm;                       // [we] own-row coefficient
+  float* ss = cc + we;                   // [we] partner-row coefficient
+  int* partner = reinterpret_cast<int*>(ss + we);  // [we]
+  float* rowbuf = reinterpret_cast<float*>(partner + we);  // [16][w]
+  __shared__ double red[16];
+  __shared__ int done_s;
+  const int t = threadIdx.x, lane = t & 31, wp = t >> 5;
+  float* Ca = pb.C;
+  float* Cb = pb.work;
+  float* Va = pb.work + (long long)w * w;
+  float* Vb = pb.work + 2LL * w * w;
+  for (long long e = t; e < (long long)w * w; e += 512) Va[e] = (e / w == e % w) ? 1.f : 0.f;  // V^T = I
+  __syncthreads();
+
+  for (int sweep = 0; sweep < 14; ++sweep) {
+    // off-diagonal and diagonal weight: stop when the matrix is diagonal to fp32 accuracy
+    double off = 0.0, dg = 0.0;
+    for (long long e = t; e < (long long)w * w; e += 512) {
+      const double x = (double)Ca[e];
+      if (e / w == e % w) dg += x * x; else off += x * x;
+    }
+    for (int o = 16; o > 0; o >>= 1) { off += __shfl_xor_sync(0xffffffffu, off, o); dg += __shfl_xor_sync(0xffffffffu, dg, o); }
+    if (lane == 0) red[wp] = off;
+    __syncthreads();
+    if (t == 0) { double s0 = 0.0; for (int k = 0; k < 16; ++k) s0 += red[k]; red[0] = s0; }
+    __syncthreads();
+    const double off_all = red[0];
+    __syncthreads();
+    if (lane == 0) red[wp] = dg;
+    __syncthreads();
+    if (t == 0) { double s0 = 0.0; for (int k = 0; k < 16; ++k) s0 += red[k]; done_s = off_all <= 1e-14 * (double)w * (double)w * s0; }
+    __syncthreads();
+    if (done_s) break;
+
+    for (int step = 0; step < we - 1; ++step) {
+      // ---- rotations of this step's pairs
+      for (int k = t; k < we / 2; k += 512) {
+        const int p = (step + k) % (we - 1);
+        const int q = (k == 0) ? we - 1 : (step + we - 1 - k) % (we - 1);
+        float c = 1.f, s = 0.f;
+        if (p < w && q < w) {
+          const double apq = (double)Ca[(long long)p * w + q];
+          if (apq != 0.0) {
+            const double app = (double)Ca[(long long)p * w + p], aqq = (double)Ca[(long long)q * w + q];
+            const double theta = (aqq - app) / (2.0 * apq);
+            const double tt = (theta >= 0.0 ? 1.0 : -1.0) / (fabs(theta) + sqrt(theta * theta + 1.0));
+            const double cd = 1.0 / sqrt(tt * tt + 1.0);
+            c = (float)cd; s = (float)(tt * cd);
+          }
+        }
+        // new row p = c row p - s row q ; new row q = s row p + c row q
+        if (p < we) { partner[p] = q; cc[p] = c; ss[p] = -s; }
+        if (q < we) { partner[q] = p; cc[q] = c; ss[q] = s; }
+      }
+      __syncthreads();
+      // ---- rows of J^T C J and of J^T V^T
+      float* rb = rowbuf + wp * w;
+      for (int i = wp; i < w; i += 16) {
+        int pi = partner[i];
+        float ci = cc[i], si = ss[i];
+        if (pi >= w) { pi = i; ci = 1.f; si = 0.f; }  // paired with the dummy index
+        for (int j = lane; j < w; j += 32) {
+          rb[j] = ci * Ca[(long long)i * w + j] + si * Ca[(long long)pi * w + j];
+          Vb[(long long)i * w + j] = ci * Va[(long long)i * w + j] + si * Va[(long long)pi * w + j];
+        }
+        __syncwarp();
+        for (int j = lane; j < w; j += 32) {
+          int pj = partner[j];
+          float cj = cc[j], sj = ss[j];
+          if (pj >= w) { pj = j; cj = 1.f; sj = 0.f; }
+          Cb[(long long)i * w + j] = cj * rb[j] + sj * rb[pj];
+        }
+        __syncwarp();
+      }
+      __syncthreads();
+      float* x = Ca; Ca = Cb; Cb = x;
+      x = Va; Va = Vb; Vb = x;
+    }
+  }
+  __syncthreads();
+  // ---- eigenvalues = diagonal of Ca; rank of each (0 = largest), kept in `partner`
+  for (int i = t; i < w; i += 512) {
+    const float li = Ca[(long long)i * w + i];
+    int rk = 0;
+    for (int j = 0; j < w; ++j) {
+      const float lj = Ca[(long long)j * w + j];
+      rk += (lj > li || (lj == li && j < i)) ? 1 : 0;
+    }
+    partner[i] = rk;
+  }
+  __syncthreads();
+  // ---- Mr[a][b] = sum over the r leading eigenvectors v of v[a] v[b], b < r  (rows of V^T are eigenvectors)
+  for (long long e = t; e < (long long)w * r; e += 512) {
+    const int a = (int)(e / r), b = (int)(e - (long long)a * r);
+    double acc = 0.0;
+    for (int i = 0; i < w; ++i)
+      if (partner[i] < r) acc += (double)Va[(long long)i * w + a] * (double)Va[(long long)i * w + b];
+    pb.Mr[e] = (float)acc;
+  }
+}
+
+void launch_jacobi_projector(const EigProblem* probs, int nprobs, int w_max, cudaStream_t st) {
+  const int we = (w_max + 1) & ~1;
+  const size_t smem = sizeof(float) * (size_t)(3 * we + 16 * w_max);
+  jacobi_projector_kernel<<<nprobs, 512, smem, st>>>(probs);
+}
+
 void launch_chol_inverse(const CholProblem* probs, int nprobs, int r_max, unsigned* status, cudaStream_t st) {
   (void)r_max;
   chol_inverse_kernel<<<nprobs, 512, 0, st>>>(probs, status);

@@ -158,6 +158,18 @@ struct CholProblem {
 };
 void launch_chol_inverse(const CholProblem* probs, int nprobs, int r_max, unsigned* status, cudaStream_t st);
 
+// Rayleigh-Ritz truncation of an oversampled basis: C = (Q^T S)(Q^T S)^T is w x w symmetric (w = r + p
+// <= 600). The kernel diagonalises C with a parallel cyclic Jacobi method (one CTA per problem) and
+// writes Mr [w][r] = the first r columns of the projector V_r V_r^T onto the eigenvectors of the r
+// largest eigenvalues. C is destroyed; work holds 3 w*w floats.
+struct EigProblem {
+  float* C;
+  float* work;
+  float* Mr;
+  int w, r;
+};
+void launch_jacobi_projector(const EigProblem* probs, int nprobs, int w_max, cudaStream_t st);
+
 // Grouped helpers of the refresh: random sketches and device-to-device copies for many matrices
 // in one launch each. blk_start is the first 256-thread block of the entry within the launch.
 struct RandProblem {

@@ -46,7 +46,7 @@ class _Config(C.Structure):
         ("error_feedback", C.c_int32), ("beta2", C.c_float), ("eps", C.c_float), ("clip_rho", C.c_float),
         ("clip_scope", C.c_int32), ("sync_u", C.c_int32), ("sync_v", C.c_int32), ("outer", C.c_int32),
         ("outer_lr", C.c_float), ("outer_momentum", C.c_float), ("power_iters", C.c_int32), ("seed", C.c_uint64),
-        ("check_mode", C.c_int32), ("warm_start", C.c_int32), ("time_buffer", C.c_int32),
+        ("check_mode", C.c_int32), ("warm_start", C.c_int32), ("time_buffer", C.c_int32), ("oversample", C.c_int32),
     ]
 
 
@@ -123,13 +123,13 @@ def _stream_handle(stream: Optional[torch.cuda.Stream]) -> C.c_void_p:
 
 def make_config(mats: Sequence[Tuple[int, int, int]], K: int, H: int, *, w_dtype=F32, g_dtype=F32, e_dtype=F32,
                 variant=GLOBAL, error_feedback=True, beta2=0.999, eps=1e-8, clip_rho=0.0, clip_scope=0, sync_u=True,
-                sync_v=True, outer=OUTER_AVG, outer_lr=1.0, outer_momentum=0.0, power_iters=0, seed=0, check_mode=1, warm_start=0, time_buffer=0):
+                sync_v=True, outer=OUTER_AVG, outer_lr=1.0, outer_momentum=0.0, power_iters=0, seed=0, check_mode=1, warm_start=0, time_buffer=0, oversample=0):
     """Returns (config struct, keep-alive matrix array)."""
     arr = (_Mat * len(mats))()
     for i, (m, n, r) in enumerate(mats):
         arr[i] = _Mat(m, n, r, 0)
     cfg = _Config(len(mats), arr, K, H, w_dtype, g_dtype, e_dtype, variant, int(error_feedback), beta2, eps, clip_rho,
-                  clip_scope, int(sync_u), int(sync_v), outer, outer_lr, outer_momentum, power_iters, seed, check_mode, int(warm_start), int(time_buffer))
+                  clip_scope, int(sync_u), int(sync_v), outer, outer_lr, outer_momentum, power_iters, seed, check_mode, int(warm_start), int(time_buffer), int(oversample))
     return cfg, arr
 
 

@@ -37,6 +37,7 @@ class RunSpec:
     check_mode: int = 1
     warm_start: bool = False
     time_buffer: bool = False
+    oversample: int = 0
 
     @property
     def n_rounds(self) -> int:
@@ -73,7 +74,7 @@ def make_gpu(spec: RunSpec):
                        beta2=spec.beta2, eps=spec.eps, clip_rho=wl.clip_rho, clip_scope=spec.clip_scope,
                        sync_u=spec.sync_u, sync_v=spec.sync_v, outer=spec.outer, outer_lr=spec.outer_lr,
                        outer_momentum=spec.outer_momentum, power_iters=wl.power_iters, seed=spec.seed,
-                       check_mode=spec.check_mode, warm_start=int(spec.warm_start), time_buffer=int(spec.time_buffer))
+                       check_mode=spec.check_mode, warm_start=int(spec.warm_start), time_buffer=int(spec.time_buffer), oversample=spec.oversample)
 
 
 def device_grads(wl: synth.Workload, G: List[np.ndarray]) -> List[torch.Tensor]:
@@ -103,7 +104,7 @@ def make_oracle(spec: RunSpec) -> lo.LordoOracle:
                           beta2=f32(spec.beta2), eps=f32(spec.eps), clip_rho=f32(wl.clip_rho), clip_scope=spec.clip_scope,
                           sync_u=spec.sync_u, sync_v=spec.sync_v, outer=spec.outer, outer_lr=f32(spec.outer_lr),
                           outer_momentum=f32(spec.outer_momentum), power_iters=wl.power_iters, seed=spec.seed,
-                          w_dtype=wl.w_dtype, e_dtype=wl.e_dtype, state_dtype="f32", warm_start=spec.warm_start, time_buffer=spec.time_buffer)
+                          w_dtype=wl.w_dtype, e_dtype=wl.e_dtype, state_dtype="f32", warm_start=spec.warm_start, time_buffer=spec.time_buffer, oversample=spec.oversample)
     return lo.LordoOracle(cfg, synth.init_weights(wl, spec.seed))
 
 

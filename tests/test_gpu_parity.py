@@ -566,6 +566,32 @@ def test_config4_full_size_fast_mode_repeatable():
     assert not differing, differing[:8]
 
 
+# ------------------------------------------------------------------ oversampled sketch, Rayleigh-Ritz truncation
+
+@pytest.mark.parametrize("variant,form", [(0, 2), (1, 1)])
+@pytest.mark.parametrize("q", [0, 1])
+def test_refresh_oversampled_rayleigh_ritz(variant, form, q):
+    """Sketch of r + 8 columns truncated to the top-r subspace of the projected signal. The signal has
+    rank r plus noise, so that subspace is well separated and the basis (fixed by the subspace alone)
+    can be compared with the oracle's column by column."""
+    wl = _small(m=264, n=200, r=24, K=2, H=2, rounds=2, grad="lowrank", power_iters=q, signal_rank=24, clip_rho=30.0)
+    spec = RunSpec(wl, variant=variant, form=form, lr=0.01, oversample=8)
+    opt, orc, worst = hz.run_lockstep_refresh(spec)
+    assert opt.poll_status() == 0
+    assert worst["P_orth"] < 1e-5 and worst["P_angle"] < ANGLE_TOL and worst["u"] < 1e-3 and worst["v"] < 1e-3, worst
+
+
+def test_refresh_oversampled_fast_mode_bf16():
+    """bf16 storage in fast mode with an oversampled sketch: the inner step stays on the TMA-fed kernels,
+    the refresh runs in fp32."""
+    wl = _small(m=520, n=392, r=136, K=2, H=2, rounds=2, grad="lowrank", signal_rank=136, clip_rho=30.0, power_iters=1,
+                w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    spec = RunSpec(wl, variant=0, form=2, lr=0.01, check_mode=0, eps=0.05, oversample=16)
+    opt, orc, worst = hz.run_lockstep_refresh(spec)
+    assert opt.poll_status() == 0
+    assert worst["P_orth"] < 1e-5 and worst["P_angle"] < ANGLE_TOL and abs(worst["energy"] - 1.0) < 1e-2, worst
+
+
 # ------------------------------------------------------------------ up-link time buffer
 
 @pytest.mark.parametrize("variant,form", [(0, 0), (0, 1), (1, 1)])
