@@ -35,11 +35,6 @@ __device__ __forceinline__ int find_problem(const TcProblem* __restrict__ probs,
 
 __device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
-__device__ __forceinline__ float bf16_to_f(unsigned short x) { return __uint_as_float(((uint32_t)x) << 16); }
-__device__ __forceinline__ unsigned short f_to_bf16(float v) {
-  const __nv_bfloat16 h = __float2bfloat16_rn(v);
-  return *reinterpret_cast<const unsigned short*>(&h);
-}
 
 // ---- projection ---------------------------------------------------------------------------------
 constexpr int kPStages = 3;
@@ -417,7 +412,6 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       const int rep = pr->replica;
       const int nsteps = (pr->m + kARows - 1) / kARows;
       const long long col = (long long)n0 + colq;
-      const long long colc = col < n ? col : (long long)n - 1;
       const float c = *pr->cptr;
       float cd[4];
 #pragma unroll
