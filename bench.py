@@ -66,6 +66,7 @@ def parse_args():
     ap.add_argument("--inner-steps", type=int, default=0, help="override H (non-standard; recorded in config)")
     ap.add_argument("--layers", type=int, default=0, help="keep only the first N decoder layers (profiling; recorded in config)")
     ap.add_argument("--matrices", type=int, default=0, help="keep only the first N matrices (profiling / memory; recorded in config)")
+    ap.add_argument("--oversample", type=int, default=0, help="extra sketch columns of the refresh, Rayleigh-Ritz truncation (non-standard; recorded in config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -295,7 +296,7 @@ def main():
     opt = lordo.Lordo(wl.mats, wl.K, H, W0, device=str(dev), g_dtype=synth.torch_dtype(wl.g_dtype),
                       e_dtype=synth.torch_dtype(wl.e_dtype), variant=hp["variant"], error_feedback=True, beta2=0.999,
                       eps=1e-8, clip_rho=wl.clip_rho, outer=lordo.OUTER_NESTEROV, outer_lr=0.8, outer_momentum=0.9,
-                      power_iters=wl.power_iters, seed=seed, check_mode=1 if args.mode == "check" else 0)
+                      power_iters=wl.power_iters, seed=seed, check_mode=1 if args.mode == "check" else 0, oversample=args.oversample)
     del W0
     # two gradient sets (round-level signal + per-replica noise), used alternately
     pool = [synth.gradients_device(wl, seed, 0, s, device=str(dev)) for s in range(2)]
@@ -423,7 +424,8 @@ def main():
                        "outer": "nesterov", "mode": args.mode, "w_dtype": wl.w_dtype, "g_dtype": wl.g_dtype,
                        "step": "one round = H inner steps + outer step + subspace refresh",
                        "l2": "inputs larger than L2 (no flush)" if wl.weight_replicas * 2 > 4e8 else "inputs fit L2",
-                       "parallelism": "replicas only" if world > 1 else "1 gpu"},
+                       "parallelism": "replicas only" if world > 1 else "1 gpu",
+                       **({"oversample": args.oversample} if args.oversample else {})},
             "clocks": sampler.summary(t_wall0, t_wall1),
             "gpu_launches": launches,
             "inner_step": {"ms": inner_ms, "params_per_s": wl.weight_replicas / (inner_ms * 1e-3) if inner_ms else None},

@@ -426,8 +426,8 @@ __global__ void __launch_bounds__(512) chol_inverse_kernel(const CholProblem* __
 // A sweep is w - 1 steps (w made even with a dummy index); a step rotates w/2 disjoint index pairs
 // (round-robin tournament order). Rotations of disjoint pairs commute, so a step is
 //   C <- J^T C J,  V^T <- J^T V^T,  J = product of the step's plane rotations,
-// done row by row: a warp forms row i of J^T C from rows i and partner(i) (coalesced reads), keeps
-// it in shared memory, applies the column rotations there and writes row i of the new matrix.
+// done pair by pair: a warp forms rows p and q of J^T C from the old rows p and q (coalesced reads),
+// keeps them in shared memory, applies the column rotations there and writes the two new rows.
 // Old and new matrices are separate buffers, swapped after every step.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(512) jacobi_projector_kernel(const EigProblem* __restrict__ probs) {
@@ -438,7 +438,7 @@ __global__ void __launch_bounds__(512) jacobi_projector_kernel(const EigProblem*
   float* cc = jsm;                       // [we] own-row coefficient
   float* ss = cc + we;                   // [we] partner-row coefficient
   int* partner = reinterpret_cast<int*>(ss + we);  // [we]
-  float* rowbuf = reinterpret_cast<float*>(partner + we);  // [16][w]
+  float* rowbuf = reinterpret_cast<float*>(partner + we);  // [16][2][w]
   __shared__ double red[16];
   __shared__ int done_s;
   const int t = threadIdx.x, lane = t & 31, wp = t >> 5;
@@ -490,22 +490,34 @@ __global__ void __launch_bounds__(512) jacobi_projector_kernel(const EigProblem*
         if (q < we) { partner[q] = p; cc[q] = c; ss[q] = s; }
       }
       __syncthreads();
-      // ---- rows of J^T C J and of J^T V^T
-      float* rb = rowbuf + wp * w;
-      for (int i = wp; i < w; i += 16) {
-        int pi = partner[i];
-        float ci = cc[i], si = ss[i];
-        if (pi >= w) { pi = i; ci = 1.f; si = 0.f; }  // paired with the dummy index
+      // ---- rows of J^T C J and of J^T V^T, a pair of rows per warp: both new rows come from the same two
+      // old rows, which are read once
+      float* rbp = rowbuf + wp * 2 * w;
+      float* rbq = rbp + w;
+      for (int k = wp; k < we / 2; k += 16) {
+        int p = (step + k) % (we - 1);
+        int q = (k == 0) ? we - 1 : (step + we - 1 - k) % (we - 1);
+        float c = cc[p], sn = -ss[p];  // new row p = c row p - sn row q ; new row q = sn row p + c row q
+        const bool single = q >= w || p >= w;  // paired with the dummy index: the row is copied
+        if (p >= w) p = q;
+        if (single) { q = p; c = 1.f; sn = 0.f; }
+#pragma unroll 4
         for (int j = lane; j < w; j += 32) {
-          rb[j] = ci * Ca[(long long)i * w + j] + si * Ca[(long long)pi * w + j];
-          Vb[(long long)i * w + j] = ci * Va[(long long)i * w + j] + si * Va[(long long)pi * w + j];
+          const float cp = Ca[(long long)p * w + j], cq = Ca[(long long)q * w + j];
+          const float vp = Va[(long long)p * w + j], vq = Va[(long long)q * w + j];
+          rbp[j] = c * cp - sn * cq;
+          rbq[j] = sn * cp + c * cq;
+          Vb[(long long)p * w + j] = c * vp - sn * vq;
+          if (!single) Vb[(long long)q * w + j] = sn * vp + c * vq;
         }
         __syncwarp();
+#pragma unroll 4
         for (int j = lane; j < w; j += 32) {
           int pj = partner[j];
           float cj = cc[j], sj = ss[j];
           if (pj >= w) { pj = j; cj = 1.f; sj = 0.f; }
-          Cb[(long long)i * w + j] = cj * rb[j] + sj * rb[pj];
+          Cb[(long long)p * w + j] = cj * rbp[j] + sj * rbp[pj];
+          if (!single) Cb[(long long)q * w + j] = cj * rbq[j] + sj * rbq[pj];
         }
         __syncwarp();
       }
@@ -538,7 +550,12 @@ __global__ void __launch_bounds__(512) jacobi_projector_kernel(const EigProblem*
 
 void launch_jacobi_projector(const EigProblem* probs, int nprobs, int w_max, cudaStream_t st) {
   const int we = (w_max + 1) & ~1;
-  const size_t smem = sizeof(float) * (size_t)(3 * we + 16 * w_max);
+  const size_t smem = sizeof(float) * (size_t)(3 * we + 32 * w_max);
+  static bool configured = false;  // w <= 600 (checked at init): at most 84 KB
+  if (!configured) {
+    cudaFuncSetAttribute(jacobi_projector_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(float) * (3 * 600 + 32 * 600)));
+    configured = true;
+  }
   jacobi_projector_kernel<<<nprobs, 512, smem, st>>>(probs);
 }
 
