@@ -46,12 +46,24 @@ def test_workspace_query_and_validation(lib):
         ([(256, 256, 16)], dict(beta2=1.0), 1),  # beta2 out of range
         ([(256, 256, 16)], dict(power_iters=9), 1),
         ([(256, 256, 16)], dict(variant=5), 1),
+        ([(256, 256, 16)], dict(time_buffer=2), 1),
+        ([(256, 256, 16)], dict(oversample=4), 1),                  # not a multiple of 8
+        ([(256, 256, 16)], dict(oversample=8, warm_start=1), 8),    # needs a fresh sketch
+        ([(256, 24, 16)], dict(oversample=16), 2),                  # r + p > n
+        ([(1024, 1024, 512)], dict(oversample=96), 2),              # r + p > 600
     ]
     for mats, kw, code in bad:
         cfg, _k = lordo.make_config(mats, 2, 4, **kw)
         with pytest.raises(lordo.LordoError) as ei:
             lordo.query_workspace(cfg)
         assert ei.value.status == code
+    # both options cost workspace: the time buffers (K r n floats) and the wider sketch
+    c0, _k0 = lordo.make_config([(256, 256, 16)], 2, 4)
+    c1, _k1 = lordo.make_config([(256, 256, 16)], 2, 4, time_buffer=1)
+    c2, _k2 = lordo.make_config([(256, 256, 16)], 2, 4, oversample=8)
+    base = lordo.query_workspace(c0)
+    assert lordo.query_workspace(c1) >= base + 2 * 16 * 256 * 4
+    assert lordo.query_workspace(c2) > base
     cfg, _k = lordo.make_config([(256, 256, 16)], 65, 4)
     with pytest.raises(lordo.LordoError):
         lordo.query_workspace(cfg)
