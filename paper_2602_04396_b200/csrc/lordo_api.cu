@@ -353,7 +353,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         pp.P16 = P16 + (size_t)k * m_k * r_k; pp.PT16 = PT16 + (size_t)k * r_n * m_k;
         pp.m = md.m; pp.r = md.r; pp.r_k = r_k; pp.m_k = m_k;
         c->h_prep.push_back(pp);
-        c->h_prep_start.push_back(c->h_prep_start.back() + (md.m * md.r + 255) / 256);
+        c->h_prep_start.push_back(c->h_prep_start.back() + ((md.m + 63) / 64) * ((md.r + 63) / 64));  // 64 x 64 tiles
       }
       for (int k = 0; k < K; ++k) {
         const long long wo = (long long)k * md.m * md.n, so = (long long)k * md.r * md.n;

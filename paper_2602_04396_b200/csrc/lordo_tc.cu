@@ -65,18 +65,35 @@ struct Elem<false> {
 // ---------------------------------------------------------------------------------------------
 // P (fp32 [m][r]) -> P16 [m_r][r_k] and PT16 [r_n][m_k] in bf16; the pads stay zero.
 // ---------------------------------------------------------------------------------------------
+// One block per 64 x 64 tile of P: rows of P16 and, through a transposed tile in shared memory, rows of
+// PT16 are both written as runs of consecutive addresses.
 __global__ void __launch_bounds__(256) prep_projection_kernel(const TcPrep* __restrict__ items, const long long* __restrict__ blk_start,
                                                               int nitems) {
+  __shared__ __nv_bfloat16 tile[64][66];
   const long long blk = blockIdx.x;
   const int i = find_segment(blk_start, nitems, blk);
   const TcPrep it = items[i];
-  const long long e = (blk - blk_start[i]) * 256 + threadIdx.x;
-  if (e >= it.m * it.r) return;
-  const long long row = e / it.r;
-  const int col = (int)(e - row * it.r);
-  const __nv_bfloat16 h = __float2bfloat16_rn(it.P[e]);
-  it.P16[row * it.r_k + col] = h;
-  it.PT16[(long long)col * it.m_k + row] = h;
+  const long long local = blk - blk_start[i];
+  const int tiles_c = (it.r + 63) / 64;
+  const long long row0 = (local / tiles_c) * 64;
+  const int col0 = (int)(local % tiles_c) * 64;
+  for (int e = threadIdx.x; e < 64 * 64; e += 256) {
+    const int rr = e >> 6, cc = e & 63;
+    const long long row = row0 + rr;
+    const int col = col0 + cc;
+    if (row < it.m && col < it.r) {
+      const __nv_bfloat16 h = __float2bfloat16_rn(it.P[row * it.r + col]);
+      it.P16[row * it.r_k + col] = h;
+      tile[rr][cc] = h;
+    }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < 64 * 64; e += 256) {
+    const int cc = e >> 6, rr = e & 63;
+    const long long row = row0 + rr;
+    const int col = col0 + cc;
+    if (row < it.m && col < it.r) it.PT16[(long long)col * it.m_k + row] = tile[rr][cc];
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
