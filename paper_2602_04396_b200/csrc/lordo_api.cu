@@ -428,7 +428,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         for (const CholProblem& x : sl.ch) { if (x.r > st.r_max) st.r_max = x.r; c->h_chols.push_back(x); }
       } else if (st.type == ST_RANDOM) {
         st.first = (long long)c->h_rands.size(); st.count = (int)sl.rn.size(); st.tiles = 0;
-        for (RandProblem& x : sl.rn) { x.blk_start = st.tiles; st.tiles += (x.count + 255) / 256; c->h_rands.push_back(x); }
+        for (RandProblem& x : sl.rn) { x.blk_start = st.tiles; st.tiles += (x.count + 2047) / 2048; c->h_rands.push_back(x); }  // 8 per thread
       } else if (st.type == ST_SKETCH) {
         st.first = (long long)c->h_sks.size(); st.count = (int)sl.sk.size(); st.tiles = 0;
         for (SkProblem& x : sl.sk) { x.tile_start = st.tiles; st.tiles += (x.M + 127) / 128; c->h_sks.push_back(x); }

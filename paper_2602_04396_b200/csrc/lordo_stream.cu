@@ -272,13 +272,20 @@ __global__ void __launch_bounds__(256) fill_random_grouped_kernel(const RandProb
     if (probs[mid].blk_start <= blk) lo = mid; else hi = mid - 1;
   }
   const RandProblem pb = probs[lo];
-  const long long c = (blk - pb.blk_start) * 256 + threadIdx.x;
-  if (c >= pb.count) return;
+  const long long c0 = ((blk - pb.blk_start) * 256 + threadIdx.x) * 8;  // eight consecutive entries per thread (count is a multiple of 8)
+  if (c0 >= pb.count) return;
   const unsigned long long key = stream_key(seed, pb.purpose, pb.mat, index, pb.replica);
-  const unsigned long long w = mix64(key + kGolden * (unsigned long long)(c + 1));
-  const float val = (float)(__popcll(w) - 32);
-  if (pb.out) pb.out[c] = val;
-  if (pb.out16) pb.out16[c] = __float2bfloat16_rn(val);  // integers in [-32, 32]: exact in bf16
+  float val[8];
+#pragma unroll
+  for (int x = 0; x < 8; ++x) val[x] = (float)(__popcll(mix64(key + kGolden * (unsigned long long)(c0 + x + 1))) - 32);
+  if (pb.out) {
+    *reinterpret_cast<float4*>(pb.out + c0) = make_float4(val[0], val[1], val[2], val[3]);
+    *reinterpret_cast<float4*>(pb.out + c0 + 4) = make_float4(val[4], val[5], val[6], val[7]);
+  }
+  if (pb.out16) {  // integers in [-32, 32]: exact in bf16
+    store4(pb.out16, LORDO_BF16, c0, make_float4(val[0], val[1], val[2], val[3]));
+    store4(pb.out16, LORDO_BF16, c0 + 4, make_float4(val[4], val[5], val[6], val[7]));
+  }
 }
 
 // fp32 -> bf16 copies of many buffers in one launch (operands of the tensor-core sketch products)
