@@ -437,6 +437,7 @@ def main():
             "e2e": e2e,
             "cpu_baseline": cpu,
             "device_flags": flags,
+            "memory": {"workspace_bytes": int(opt.workspace_bytes), "peak_allocated_bytes": int(torch.cuda.max_memory_allocated(dev))},
         }
         print(json.dumps(out))
     opt.close()
