@@ -213,7 +213,9 @@ LORDO_API int lordo_selftest_wait_timeout(lordo_ctx* ctx, void* stream);
  * done in the current round}. A checkpoint is the caller's tensors (W, E, P, u, v, X0, B, Delta) plus
  * these four numbers: restore the tensors into the buffers of a context made with the same
  * configuration, then call lordo_set_counters (which also makes the library rebuild its internal
- * copies of P before the next step). */
+ * copies of P before the next step). With time_buffer the low-rank accumulators of a round live in the
+ * workspace and are not part of a checkpoint: lordo_set_counters then accepts round boundaries only
+ * (in[3] == 0, where the accumulators are zero) and returns LORDO_ERR_UNSUPPORTED otherwise. */
 LORDO_API int lordo_get_counters(const lordo_ctx* ctx, int64_t out[4]);
 LORDO_API int lordo_set_counters(lordo_ctx* ctx, const int64_t in[4]);
 

@@ -1391,6 +1391,8 @@ int lordo_get_counters(const lordo_ctx* c, int64_t out[4]) {
 int lordo_set_counters(lordo_ctx* c, const int64_t in[4]) {
   if (!c || !in) return LORDO_ERR_INVALID_ARG;
   if (in[0] < 0 || in[1] < 0 || in[2] < 0 || in[3] < 0 || in[3] > c->cfg.H) return fail(c, LORDO_ERR_INVALID_ARG, "counter out of range");
+  if (c->cfg.time_buffer && in[3] != 0)
+    return fail(c, LORDO_ERR_UNSUPPORTED, "time_buffer: the accumulators live in the workspace, so a checkpoint can only be restored at a round boundary");
   c->steps = in[0]; c->refreshes = in[1]; c->outers = in[2]; c->steps_in_round = (int)in[3];
   c->after_outer = false;
   c->p_copies_stale = true;  // a restored checkpoint brings its own P

@@ -639,6 +639,11 @@ def test_time_buffer_refuses_full_rank_qhm():
     with pytest.raises(lordo.LordoError):
         opt.inner_step(G, 0.01, 0.9, 0.9, 2)
     opt.inner_step(G, 0.01, 0.9, 0.9, 1)  # the low-rank form is accepted
+    # the accumulators are workspace state: a checkpoint inside a round cannot be restored
+    steps, refreshes, outers, in_round = opt.counters()
+    assert in_round == 1
+    with pytest.raises(lordo.LordoError):
+        opt.set_counters([steps, refreshes, outers, in_round])
     opt.close()
 
 
