@@ -42,8 +42,11 @@ Readings of points the paper leaves open (each is restated where it is used):
       after every synchronisation. The basis must stay fixed between two synchronisations.
 
 Parity status: every function here is pinned by tests/test_oracle_pins.py against closed forms,
-invariants, library routines (torch.optim.Adam / SGD, numpy.linalg.svd / qr) or brute force.
-Agreement with the authors' own (unpublished) code on R1-R14 is "parity unpinned".
+invariants, library routines (torch.optim.Adam / SGD, numpy.linalg.svd / qr) or brute force; the
+wiring of refresh_subspace and run_rounds (which basis is old and which new in the rotation, the
+step count it uses, the Local signal, the sketch index, when a refresh happens) by closed forms
+that hold after one moment update, by a subspace that cannot move and by signals of known range.
+Agreement with the authors' own (unpublished) code on R1-R16 is "parity unpinned".
 """
 from __future__ import annotations
 

@@ -473,6 +473,8 @@ def test_bf16_storage_rounds_once_per_step():
 # stored outputs (tests/golden/, written by tests/golden/make_golden.py from the oracle alone)
 # ---------------------------------------------------------------------------------------------
 def test_golden_files_match_the_oracle():
+    """Regression guard, not a pin: the stored values were written by the oracle itself, so this only
+    shows that its arithmetic has not changed since (the pins are the other tests of this file)."""
     import importlib.util
     import os
     here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
@@ -668,3 +670,168 @@ def test_rayleigh_ritz_basis_depends_on_the_subspace_only():
     Vr = -V[:, np.argsort(lam)[::-1][:r]][:, ::-1]
     P2 = lo.householder_qr_q(Q @ (Vr @ Vr[:r, :].T))
     assert np.abs(P1 - P2).max() < 1e-10
+
+
+# ---------------------------------------------------------------------------------------------
+# Wiring of the refresh and of the driver loop: which basis is "old" and which "new" in the
+# rotation, which step count it uses, what the Local signal is, which sketch a refresh draws and
+# when a refresh happens. Each test below is built on something fixed outside the oracle: a closed
+# form that holds after exactly one moment update, the geometry of a subspace that cannot move, a
+# signal whose range is known by construction.
+# ---------------------------------------------------------------------------------------------
+def _one_step_then_refresh(variant):
+    """One worker, one inner step with gradient G1 (so s = 1, E = 0 before it, no clipping), one
+    synchronisation, then a refresh that moves the basis. Returns everything a closed form needs."""
+    rng = np.random.default_rng(31)
+    m, n, r = 24, 18, 4
+    b1, b2 = 0.8, 0.95
+    cfg, W0 = make([(m, n, r)], K=1, H=1, variant=variant, beta2=b2, eps=1e-3, seed=11)
+    o = LordoOracle(cfg, W0)
+    G1 = [rng.standard_normal((1, m, n))]
+    if variant == LOCAL:
+        o.refresh_subspace(G1, b1)  # s = 0: no rotation, only the first basis
+    P_old = (o.P[0][0] if variant == LOCAL else o.P[0]).copy()
+    o.inner_step(G1, 1e-2, b1, 0.7, QHM_FULL if variant == GLOBAL else QHM_LOW)
+    o.outer_step()
+    G2 = [rng.standard_normal((1, m, n))]
+    o.refresh_subspace(G2 if variant == LOCAL else None, b1)
+    P_new = o.P[0][0] if variant == LOCAL else o.P[0]
+    return o, P_old, P_new, G1[0][0], b1, b2
+
+
+@pytest.mark.parametrize("variant", [GLOBAL, LOCAL])
+def test_refresh_after_one_step_gives_the_moments_of_that_step_in_the_new_basis(variant):
+    """After exactly one moment update u = (1 - b1) g and v = (1 - b2) g o g, so u^ = g and
+    v^ - u^ o u^ = 0: the rotation lines of Algorithm 1 then reduce to u' = (1 - b1) g' and
+    v' = (1 - b2) g' o g' with g' = P_new^T P_old g, the moments the same step would have left in
+    the new basis. The closed form fails if the two bases are swapped in the call (Rot transposed),
+    if the rotation is skipped, and if the step count handed to it is not s = 1 (the factor
+    (1 - b2^s) / (1 - b1^s)^2 in front of g' o g' is 1 - b2 only for s = 1)."""
+    o, P_old, P_new, G1, b1, b2 = _one_step_then_refresh(variant)
+    assert subspace_angle(P_old, P_new) > 0.1  # the basis did move
+    g = P_old.T @ G1
+    g_new = P_new.T @ (P_old @ g)
+    assert np.abs(o.u[0][0] - (1 - b1) * g_new).max() < 1e-13
+    assert np.abs(o.v[0][0] - (1 - b2) * g_new * g_new).max() < 1e-13
+    assert np.abs(o.u[0][0] - (1 - b1) * g).max() > 1e-3  # and differ from the unrotated ones
+
+
+@pytest.mark.parametrize("variant", [GLOBAL, LOCAL])
+def test_refresh_that_cannot_move_the_subspace_keeps_the_first_moment_vector(variant):
+    """Stagnation case (Sec. "Enabling Full Subspace Exploration"): the refresh signal has exact rank
+    r and lies in span(P), so the new basis spans the same subspace, P_new = P_old Q with Q
+    orthogonal, and the first moment, seen in the full space, must not move: P_new u_new = P_old u_old.
+    Swapped bases give P_old Q Q u, a skipped rotation P_old Q u."""
+    rng = np.random.default_rng(32)
+    m, n, r, K = 30, 22, 5, 2
+    cfg, W0 = make([(m, n, r)], K=K, H=1, variant=variant, seed=3)
+    P0 = np.linalg.qr(rng.standard_normal((m, r)))[0]
+    o = LordoOracle(cfg, W0, P0=[P0])
+    o.s = 7
+    o.u[0] = rng.standard_normal((K, r, n))
+    o.v[0] = rng.random((K, r, n)) + 0.5
+    u_full = np.stack([P0 @ o.u[0][k] for k in range(K)])
+    inside = [P0 @ rng.standard_normal((r, n)) for _ in range(K)]  # rank r, inside span(P)
+    if variant == GLOBAL:
+        o.Delta[0] = inside[0]
+        o.refresh_subspace(None, 0.9)
+    else:
+        o.refresh_subspace([np.stack(inside)], 0.9)
+    for k in range(K):
+        P_new = o.P[0][k] if variant == LOCAL else o.P[0]
+        assert subspace_angle(P_new, P0) < 1e-7
+        assert np.abs(P_new - P0).max() > 1e-2  # another basis of the same subspace
+        assert np.abs(P_new @ o.u[0][k] - u_full[k]).max() < 1e-12
+
+
+def test_local_refresh_signal_is_the_clipped_gradient_plus_the_error_buffer():
+    """Algorithm 2, ComputeProjection(G^ + E): with E = L - c G set by hand, L of exact rank r, the
+    signal is L whatever G is, and the refresh must return range(L). Dropping E leaves c G (full
+    rank), dropping c leaves L + (1 - c) G."""
+    rng = np.random.default_rng(33)
+    m, n, r, K, rho = 28, 20, 4, 2, 2.0
+    cfg, W0 = make([(m, n, r)], K=K, H=1, variant=LOCAL, clip_rho=rho, power_iters=1)
+    o = LordoOracle(cfg, W0)
+    G = rng.standard_normal((K, m, n))
+    L = [np.linalg.qr(rng.standard_normal((m, r)))[0] @ rng.standard_normal((r, n)) for _ in range(K)]
+    for k in range(K):
+        c = min(1.0, rho / (math.sqrt(float(np.sum(G[k] ** 2))) + 1e-6))
+        assert c < 0.2  # the gradient is clipped, so a dropped coefficient shows
+        o.E[0][k] = L[k] - c * G[k]
+    o.refresh_subspace([G], 0.9)
+    for k in range(K):
+        P = o.P[0][k]
+        assert np.linalg.norm(L[k] - P @ (P.T @ L[k])) / np.linalg.norm(L[k]) < 1e-6
+    # without error feedback the signal is the clipped gradient alone: E must then be ignored
+    cfg2, _ = make([(m, n, r)], K=K, H=1, variant=LOCAL, clip_rho=rho, error_feedback=False)
+    o2 = LordoOracle(cfg2, W0)
+    o2.E[0][:] = 5.0 * rng.standard_normal((K, m, n))
+    Glow = np.stack([np.linalg.qr(rng.standard_normal((m, r)))[0] @ rng.standard_normal((r, n)) for _ in range(K)])
+    o2.refresh_subspace([Glow], 0.9)
+    for k in range(K):
+        P = o2.P[0][k]
+        assert np.linalg.norm(Glow[k] - P @ (P.T @ Glow[k])) / np.linalg.norm(Glow[k]) < 1e-6
+
+
+@pytest.mark.parametrize("variant", [GLOBAL, LOCAL])
+def test_every_refresh_draws_its_own_sketch(variant):
+    """The sketch of refresh number j of matrix i (and worker k under the Local rule) is the
+    generator's stream (seed, sketch, i, j, k): two refreshes of the same full-rank signal give two
+    different bases, each the range finder's answer for its own stream. A refresh counter that
+    stands still would repeat the first basis."""
+    rng = np.random.default_rng(34)
+    mats = [(20, 16, 3), (18, 24, 4)]
+    K, seed = 2, 9
+    cfg, W0 = make(mats, K=K, H=1, variant=variant, seed=seed)
+    o = LordoOracle(cfg, W0)
+    S = [rng.standard_normal((K, m, n)) for m, n, _ in mats]
+    seen = []
+    for j in range(3):
+        if variant == GLOBAL:
+            for i in range(len(mats)):
+                o.Delta[i] = S[i][0]
+            o.refresh_subspace(None, 0.9)
+        else:
+            o.refresh_subspace(S, 0.9)
+        for i, (m, n, r) in enumerate(mats):
+            for k in range(K if variant == LOCAL else 1):
+                Om = lo.random_matrix(seed, lo.PURPOSE_OMEGA, i, j, k, n, r)
+                want = np.linalg.qr(S[i][k] @ Om)[0]  # any orthonormal basis of range(S Omega)
+                got = o.P[i][k] if variant == LOCAL else o.P[i]
+                assert subspace_angle(got, want) < 1e-7, (j, i, k)
+        seen.append(np.concatenate([p.ravel() for p in o.P]))
+    assert np.abs(seen[0] - seen[1]).max() > 1e-2 and np.abs(seen[1] - seen[2]).max() > 1e-2
+    if variant == LOCAL:  # workers draw different sketches
+        assert subspace_angle(o.P[0][0], np.linalg.qr(S[0][0] @ lo.random_matrix(seed, lo.PURPOSE_OMEGA, 0, 2, 1, 16, 3))[0]) > 1e-2
+
+
+def test_driver_loop_refreshes_local_before_the_step_and_global_after_the_sync():
+    """R11. Local: the basis is refreshed from the first gradient of a round before that gradient is
+    projected, so a gradient of exact rank r is represented without loss and leaves E = 0 (a refresh
+    after the step would have projected it onto Q_0 = I[:, :r] and left E != 0). Global: the basis a
+    round works with is the range of the previous round's pseudo-gradient, hence after the sync and
+    before the next step; with the full-rank QHM term and H = 1 that pseudo-gradient is known in
+    closed form from the first basis."""
+    rng = np.random.default_rng(35)
+    m, n, r, K = 26, 20, 4, 2
+    cfg, W0 = make([(m, n, r)], K=K, H=1, variant=LOCAL)
+    o = LordoOracle(cfg, W0)
+    Glow = np.stack([rng.standard_normal((m, r)) @ rng.standard_normal((r, n)) for _ in range(K)])
+    lo.run_rounds(o, lambda rnd, h: [Glow], 1, 1e-2, 0.9, 0.9, QHM_LOW)
+    assert np.abs(o.E[0]).max() < 1e-10 * np.abs(Glow).max()
+    assert o.refreshes == 1 and o.s == 1
+    # Global: two rounds; the second round's low-rank gradient must be taken in the refreshed basis
+    cfg, W0 = make([(m, n, r)], K=1, H=1, variant=GLOBAL, seed=4, eps=1e-3)
+    o = LordoOracle(cfg, W0)
+    P0 = o.P[0].copy()
+    G = [rng.standard_normal((1, m, n)) for _ in range(2)]
+    lo.run_rounds(o, lambda rnd, h: [G[rnd]], 2, 1e-2, 0.9, 0.5, QHM_FULL)
+    assert o.refreshes == 2 and o.s == 2
+    # round 1 by hand (s = 1, E = 0, K = 1, averaging outer step): Delta_1 = lr * update
+    g = P0.T @ G[0][0]
+    D = np.abs(g) + 1e-3                                  # sqrt(v^) + eps with v^ = g o g
+    delta1 = 1e-2 * (0.5 * G[0][0] / D.mean(axis=0)[None, :] + 0.5 * P0 @ (g / D))
+    P1 = np.linalg.qr(delta1 @ lo.random_matrix(4, lo.PURPOSE_OMEGA, 0, 0, 0, n, r))[0]
+    # the error buffer after round 2 is orthogonal to the basis that round 2 projected with
+    assert np.abs(P1.T @ o.E[0][0]).max() < 1e-9
+    assert np.abs(P0.T @ o.E[0][0]).max() > 1e-3
