@@ -70,6 +70,7 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="skip the short legs on the other configurations")
     return ap.parse_args()
 
 
@@ -177,18 +178,19 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # the CPU oracle on a bounded sample (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample(wl, variant_name: str):
+def oracle_sample(wl, variant_name: str, K: int = 0, H: int = 6):
     """Returns (sample workload, description). One matrix of the most common shape class with all
-    K replicas, a round of up to 6 inner steps + outer step + refresh."""
+    K replicas (or the first `K` of them), a round of up to `H` inner steps + outer step + refresh."""
     from paper_2602_04396_b200 import synth
     shapes = {}
     for mat in wl.mats:
         shapes[mat] = shapes.get(mat, 0) + 1
     mat = max(shapes, key=lambda s: (shapes[s], -s[0] * s[1]))
-    H = min(wl.H, 6)
-    sample = synth.scaled(wl, mats=[mat], H=H, rounds=1)
-    desc = (f"1 matrix {mat[0]}x{mat[1]} r{mat[2]} of {len(wl.mats)}, all K={wl.K} replicas, one round of "
-            f"{H} inner steps + outer step + refresh, {variant_name} rule")
+    H = min(wl.H, H)
+    Ks = min(wl.K, K) if K > 0 else wl.K
+    sample = synth.scaled(wl, mats=[mat], H=H, rounds=1, K=Ks)
+    desc = (f"1 matrix {mat[0]}x{mat[1]} r{mat[2]} of {len(wl.mats)}, {'all ' if Ks == wl.K else ''}K={Ks} replicas"
+            f"{'' if Ks == wl.K else f' of {wl.K}'}, one round of {H} inner steps + outer step + refresh, {variant_name} rule")
     return sample, desc
 
 
@@ -244,8 +246,10 @@ def reference_main(args):
     if rank != 0:
         return 0
     wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
-    sample, desc = oracle_sample(wl, args.variant)
-    for _ in range(min(args.warmup, 1)):
+    # one step = one pass of the oracle over the sample; the sample shrinks with the number of passes asked
+    # for, so that the whole run stays within a few minutes
+    sample, desc = oracle_sample(wl, args.variant, H=6 if args.steps + args.warmup <= 8 else 2)
+    for _ in range(args.warmup):
         run_oracle_sample(sample, args.variant)
     total_t, total_p = 0.0, 0
     for _ in range(args.steps):
@@ -256,7 +260,7 @@ def reference_main(args):
     cores = cpu_threads()
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "variant": args.variant, "sample": desc},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
@@ -268,35 +272,25 @@ def reference_main(args):
 # ------------------------------------------------------------------------------------------------
 # the CUDA path
 # ------------------------------------------------------------------------------------------------
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        return reference_main(args)
-
+def run_leg(wl, variant_name: str, mode: str, steps: int, warmup: int, *, dev, rank: int, world: int, local_rank: int,
+            oversample: int = 0, e2e_steps: int = 0, peaks=None):
+    """One timed leg: builds the workload on the device, runs `warmup` + `steps` rounds (a round = H inner
+    steps, with the Local refresh before the first; the outer step; the Global refresh), and returns the
+    figures of that leg: whole-round throughput, per-kernel-class times from the library's CUDA events,
+    the dominant kernel's roofline fraction, the clock sample of the timed region."""
     import torch
     import torch.distributed as dist
     from paper_2602_04396_b200 import lordo, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
-    hp = HYPER[args.variant]
+    hp = HYPER[variant_name]
     H = wl.H
     seed = 1000 + rank  # every rank runs its own copy of the workload on its own inputs
-
+    torch.cuda.reset_peak_memory_stats(dev)
     W0 = synth.init_weights_device(wl, seed, device=str(dev))
     opt = lordo.Lordo(wl.mats, wl.K, H, W0, device=str(dev), g_dtype=synth.torch_dtype(wl.g_dtype),
                       e_dtype=synth.torch_dtype(wl.e_dtype), variant=hp["variant"], error_feedback=True, beta2=0.999,
                       eps=1e-8, clip_rho=wl.clip_rho, outer=lordo.OUTER_NESTEROV, outer_lr=0.8, outer_momentum=0.9,
-                      power_iters=wl.power_iters, seed=seed, check_mode=1 if args.mode == "check" else 0, oversample=args.oversample)
+                      power_iters=wl.power_iters, seed=seed, check_mode=1 if mode == "check" else 0, oversample=oversample)
     del W0
     # two gradient sets (round-level signal + per-replica noise), used alternately
     pool = [synth.gradients_device(wl, seed, 0, s, device=str(dev)) for s in range(2)]
@@ -304,7 +298,7 @@ def main():
 
     def one_round(rnd: int):
         for h in range(H):
-            G = pool[h & 1]
+            G = pool[(rnd * H + h) & 1]
             if hp["variant"] == 1 and h == 0:
                 opt.refresh_subspace(G, hp["beta1"])
             opt.inner_step(G, LR, hp["beta1"], hp["omega"], hp["form"])
@@ -318,7 +312,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for w in range(args.warmup):
+    for w in range(warmup):
         one_round(w)
     barrier()
     opt.profile_enable(True)
@@ -332,8 +326,8 @@ def main():
     barrier()
     t_wall0 = time.time()
     ev0.record()
-    for s in range(args.steps):
-        one_round(args.warmup + s)
+    for s in range(steps):
+        one_round(warmup + s)
     ev1.record()
     barrier()
     t_wall1 = time.time()
@@ -347,15 +341,15 @@ def main():
     flags = opt.poll_status()
 
     ms_total = max_over_ranks(ms_total, dev)
-    n_inner = H * args.steps
+    n_inner = H * steps
     value = aggregate_value(wl.weight_replicas * n_inner, world, ms_total)
 
     # ---- per-class figures and the roofline of the dominant kernel -----------------------------
-    tc_active = (args.mode == "fast" and wl.w_dtype == wl.g_dtype == wl.e_dtype and
+    tc_active = (mode == "fast" and wl.w_dtype == wl.g_dtype == wl.e_dtype and
                  max(r for _, _, r in wl.mats) <= (512 if wl.w_dtype == "bf16" else 256))
     abytes = algorithmic_bytes(wl, hp["variant"], hp["form"], True, tc_active)
-    per_launch = {"clip": n_inner, "project": n_inner, "moments": n_inner, "apply": n_inner, "outer_states": args.steps,
-                  "outer_weights": args.steps, "refresh": args.steps * (H if wl.refresh_every_step else 1)}
+    per_launch = {"clip": n_inner, "project": n_inner, "moments": n_inner, "apply": n_inner, "outer_states": steps,
+                  "outer_weights": steps, "refresh": steps * (H if wl.refresh_every_step else 1)}
     kernels = {}
     for name, ms in classes.items():
         cnt = per_launch[name]
@@ -365,33 +359,33 @@ def main():
             ent["algorithmic_GB"] = abytes[name] / 1e9
             ent["GB_per_s"] = abytes[name] / 1e9 / (avg * 1e-3)
         kernels[name] = ent
-    peaks = {}
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
-            peaks = json.load(fh)
-    except Exception:
-        pass
+    peaks = peaks or {}
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
     dom = max((k for k in kernels if k in abytes), key=lambda k: kernels[k]["share"])
-    ent = NCU_TRAFFIC.get(f"{wl.name}:{args.variant}:{args.mode}:{dom}")
+    ent = NCU_TRAFFIC.get(f"{wl.name}:{variant_name}:{mode}:{dom}")
     traffic = ent[0] if ent else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom].get("GB_per_s"), "peak": hbm_peak, "unit": "GB/s",
                 "frac": (kernels[dom].get("GB_per_s") or 0.0) / hbm_peak, "peak_source": peak_src, "traffic": traffic,
                 "algorithmic_bytes_per_launch": abytes[dom]}
     inner_ms = sum(classes[k] for k in ("clip", "project", "moments", "apply")) / n_inner
-    outer_ms = (classes["outer_states"] + classes["outer_weights"]) / args.steps
+    outer_ms = (classes["outer_states"] + classes["outer_weights"]) / steps
     outer_bytes = abytes["outer_states"] + abytes["outer_weights"]
+    # the three tensor-core contractions of an inner step (project, error feedback, back-projection)
+    inner_flops = sum(6.0 * r * m * n for m, n, r in wl.mats) * wl.K
+    tf_peak = float(peaks.get("bf16_tflops_sustained", 1400.0))
 
     # ---- end to end: inner steps fed from pinned host memory ------------------------------------
     e2e = None
-    if not args.no_e2e:
-        n_e2e = max(1, min(args.e2e_steps, H))
+    if e2e_steps > 0:
+        n_e2e = max(1, min(e2e_steps, H))
         G_host = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True).copy_(g) for g in pool[0]]
         clip_host = torch.empty(wl.K, dtype=torch.float32, pin_memory=True)
         h2d = sum(g.numel() * g.element_size() for g in G_host)
         stage = pool[1]
         torch.cuda.synchronize()
+        if hp["variant"] == 1:
+            opt.refresh_subspace(stage, hp["beta1"])
         opt.inner_step_host(G_host, stage, LR, hp["beta1"], hp["omega"], hp["form"], clip_host)  # warm-up
         barrier()
         n_done = max(1, min(n_e2e, H - 1))  # the round's first step was the warm-up call
@@ -407,40 +401,118 @@ def main():
                "note": "inner steps through lordo_inner_step_host; the outer step and the refresh take no host input"}
         del G_host
 
+    leg = {
+        "value": value, "ms_per_step": ms_total / steps, "steps": steps, "warmup": warmup,
+        "config": {"workload": wl.name, "matrices": len(wl.mats), "weights": wl.weights, "K": wl.K, "H": H,
+                   "rank": wl.mats[0][2], "variant": variant_name, "qhm": ["none", "low", "full"][hp["form"]],
+                   "outer": "nesterov", "mode": mode, "w_dtype": wl.w_dtype, "g_dtype": wl.g_dtype,
+                   "step": "one round = H inner steps + outer step + subspace refresh",
+                   "l2": "inputs larger than L2 (no flush)" if wl.weight_replicas * 2 > 4e8 else "inputs fit L2",
+                   "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   **({"oversample": oversample} if oversample else {})},
+        "clocks": sampler.summary(t_wall0, t_wall1),
+        "gpu_launches": launches,
+        "inner_step": {"ms": inner_ms, "params_per_s": wl.weight_replicas / (inner_ms * 1e-3) if inner_ms else None,
+                       "tensor_TFLOP_per_s": inner_flops / 1e12 / (inner_ms * 1e-3) if inner_ms else None,
+                       "frac_of_sustained_bf16_peak": (inner_flops / 1e12 / (inner_ms * 1e-3)) / tf_peak if inner_ms else None},
+        "outer_sync": {"ms": outer_ms, "GB_per_s": outer_bytes / 1e9 / (outer_ms * 1e-3) if outer_ms else None,
+                       "frac_of_hbm_peak": (outer_bytes / 1e9 / (outer_ms * 1e-3)) / hbm_peak if outer_ms else None},
+        "refresh": {"ms": classes["refresh"] / per_launch["refresh"]},
+        "kernels": kernels,
+        "roofline": roofline,
+        "e2e": e2e,
+        "device_flags": flags,
+        "memory": {"workspace_bytes": int(opt.workspace_bytes), "peak_allocated_bytes": int(torch.cuda.max_memory_allocated(dev))},
+    }
+    opt.close()
+    del opt, pool
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return leg
+
+
+# The other configurations the path is specified on, timed briefly after the headline workload in the
+# same run: (workload, variant, matrices kept (0 = all), warm-up rounds, timed rounds).
+EXTRA_LEGS = [
+    ("cfg4", "local", 0, 3, 3),
+    ("cfg3", "global", 0, 3, 10),
+    ("cfg3", "local", 0, 3, 10),
+    ("cfg5", "local", 8, 3, 10),   # the first 8 of 32 matrices: all 32 with K = 16 do not fit beside their inputs
+    ("cfg5", "global", 8, 3, 10),
+]
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return reference_main(args)
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = {}
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            peaks = json.load(fh)
+    except Exception:
+        pass
+    where = dict(dev=dev, rank=rank, world=world, local_rank=local_rank, peaks=peaks)
+
+    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
+    main_leg = run_leg(wl, args.variant, args.mode, args.steps, args.warmup, oversample=args.oversample,
+                       e2e_steps=0 if args.no_e2e else args.e2e_steps, **where)
+
+    # ---- the other configurations, briefly (one GPU, default workload only) ----------------------
+    legs = []
+    default_run = (args.workload == "cfg4" and args.variant == "global" and args.mode == "fast" and not args.inner_steps and
+                   not args.layers and not args.matrices and not args.oversample)
+    if world == 1 and default_run and not args.no_legs:
+        for name, variant, matrices, wu, st in EXTRA_LEGS:
+            lw = workload(name, 0, 0, matrices)
+            leg = run_leg(lw, variant, "fast", st, wu, **where)
+            for drop in ("e2e", "memory"):
+                leg.pop(drop, None)
+            legs.append(leg)
+
     # ---- CPU oracle on a bounded sample ---------------------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample, desc = oracle_sample(wl, args.variant)
         dt, p = run_oracle_sample(sample, args.variant)
         cpu = {"value": p / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc, "seconds": dt}
+        one, desc1 = oracle_sample(wl, args.variant, K=2, H=2)
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                dt1, p1 = run_oracle_sample(one, args.variant)
+            cpu["single_thread"] = {"value": p1 / dt1, "unit": UNIT, "cores": 1, "sample": desc1, "seconds": dt1}
+        except Exception as exc:  # threadpoolctl missing: say so instead of reporting a wrong core count
+            cpu["single_thread"] = {"unavailable": str(exc)}
 
     if rank == 0:
         out = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": main_leg["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": main_leg["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if args.mode == "fast" else "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "matrices": len(wl.mats), "weights": wl.weights, "K": wl.K, "H": H,
-                       "rank": wl.mats[0][2], "variant": args.variant, "qhm": ["none", "low", "full"][hp["form"]],
-                       "outer": "nesterov", "mode": args.mode, "w_dtype": wl.w_dtype, "g_dtype": wl.g_dtype,
-                       "step": "one round = H inner steps + outer step + subspace refresh",
-                       "l2": "inputs larger than L2 (no flush)" if wl.weight_replicas * 2 > 4e8 else "inputs fit L2",
-                       "parallelism": "replicas only" if world > 1 else "1 gpu",
-                       **({"oversample": args.oversample} if args.oversample else {})},
-            "clocks": sampler.summary(t_wall0, t_wall1),
-            "gpu_launches": launches,
-            "inner_step": {"ms": inner_ms, "params_per_s": wl.weight_replicas / (inner_ms * 1e-3) if inner_ms else None},
-            "outer_sync": {"ms": outer_ms, "GB_per_s": outer_bytes / 1e9 / (outer_ms * 1e-3) if outer_ms else None,
-                           "frac_of_hbm_peak": (outer_bytes / 1e9 / (outer_ms * 1e-3)) / hbm_peak if outer_ms else None},
-            "refresh": {"ms": classes["refresh"] / per_launch["refresh"]},
-            "kernels": kernels,
-            "roofline": roofline,
-            "e2e": e2e,
-            "cpu_baseline": cpu,
-            "device_flags": flags,
-            "memory": {"workspace_bytes": int(opt.workspace_bytes), "peak_allocated_bytes": int(torch.cuda.max_memory_allocated(dev))},
         }
+        for key in ("config", "clocks", "gpu_launches", "inner_step", "outer_sync", "refresh", "kernels", "roofline", "e2e"):
+            out[key] = main_leg[key]
+        out["gpu_launches"] = main_leg["gpu_launches"] + sum(l["gpu_launches"] for l in legs)
+        out["cpu_baseline"] = cpu
+        out["device_flags"] = main_leg["device_flags"]
+        out["memory"] = main_leg["memory"]
+        out["legs"] = legs
         print(json.dumps(out))
-    opt.close()
     if world > 1:
         dist.destroy_process_group()
     return 0

@@ -22,7 +22,9 @@
  *   - Pointer *tables* (`void* const*`) are host arrays with one device pointer per matrix.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream). Calls enqueue work
  *     and return without synchronising, except lordo_init, lordo_poll_status,
- *     lordo_inner_step_host and lordo_destroy.
+ *     lordo_inner_step_host, lordo_profile_read and lordo_destroy. (A call that is handed new
+ *     gradient pointers stages their table in one of two pinned slots and may wait for the copy
+ *     that left that slot two changes ago, which has normally long finished.)
  *   - Shapes: n and r multiples of 8, 8 <= r <= min(m, n), K >= 1, H >= 1.
  *   - Errors are return codes (lordo_status); nothing throws or aborts. After a non-zero return
  *     from an argument check no device state was modified. Numerical trouble found on the device
@@ -215,7 +217,11 @@ LORDO_API int lordo_selftest_wait_timeout(lordo_ctx* ctx, void* stream);
  * configuration, then call lordo_set_counters (which also makes the library rebuild its internal
  * copies of P before the next step). With time_buffer the low-rank accumulators of a round live in the
  * workspace and are not part of a checkpoint: lordo_set_counters then accepts round boundaries only
- * (in[3] == 0, where the accumulators are zero) and returns LORDO_ERR_UNSUPPORTED otherwise. */
+ * (in[3] == 0, where the accumulators are zero) and returns LORDO_ERR_UNSUPPORTED otherwise.
+ * Global rule: a checkpoint taken between lordo_outer_step and lordo_refresh_subspace (a round boundary
+ * with fewer refreshes than synchronisations) may run that refresh first thing after the restore. The
+ * rotation matrices behind lordo_diagnostics' MSSV are workspace state too: after a restore MSSV returns
+ * LORDO_ERR_STATE until a refresh has run on the new context. */
 LORDO_API int lordo_get_counters(const lordo_ctx* ctx, int64_t out[4]);
 LORDO_API int lordo_set_counters(lordo_ctx* ctx, const int64_t in[4]);
 
@@ -267,11 +273,14 @@ LORDO_API int lordo_fill_random(uint64_t seed, int32_t purpose, int32_t mat, int
  *   G_dev         device pointer, `count` elements of g_dtype (lordo_dtype), 16-byte aligned,
  *                 count a multiple of 8; read only
  *   rho           clipping radius; <= 0 gives c = 1
- *   coef_out_dev  device pointer to one float, written by the call (caller-owned)
+ *   coef_out_dev  device pointer to one float, written by the call (caller-owned); NaN when the
+ *                 sum of squares is NaN or infinite (this entry point has no status word)
  *
  * The call enqueues two kernels on `stream` and returns without synchronising. The first call on
  * each device looks up the device address of the static array (with that device current); make
- * that first call outside any stream capture. All calls on a device share the array: it holds
+ * that first call outside any stream capture (the address is cached for the life of the process
+ * and does not survive a cudaDeviceReset). A CUDA error already pending on the thread makes the
+ * call return LORDO_ERR_CUDA before it launches anything. All calls on a device share the array: it holds
  * whatever the previous call left (every slot a call reads it has written itself, so nothing needs
  * clearing), and two calls whose kernels overlap on the GPU -- different streams, no ordering
  * between them -- race on it. Calls on one stream are safe.

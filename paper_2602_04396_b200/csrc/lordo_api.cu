@@ -110,7 +110,7 @@ struct lordo_ctx {
   int sm_count = 0;
   TmaMatMaps* d_maps = nullptr;
   TmaGradMaps* d_gmaps = nullptr;
-  TmaGradMaps* h_gmaps = nullptr;  // pinned
+  TmaGradMaps* h_gmaps = nullptr;  // pinned, two slots of n_mats entries
   std::vector<TcProblem> h_tc;
   std::vector<TcPrep> h_prep;
   std::vector<long long> h_prep_start;
@@ -137,14 +137,18 @@ struct lordo_ctx {
   std::vector<PlanStep> tb_steps;  // Delta rebuilt from the time buffers (lordo_outer_step with time_buffer)
 
   // pinned host staging
-  const void** h_Gtab = nullptr;  // pinned
+  const void** h_Gtab = nullptr;  // pinned, two slots of n_mats entries
   unsigned* h_status = nullptr;   // pinned
   std::vector<const void*> last_G;
+  cudaEvent_t g_slot_ev[2] = {nullptr, nullptr};  // behind the last copy out of each staging slot
+  bool g_slot_used[2] = {false, false};
+  int g_slot = 0;
 
   // counters and call-order state
   int64_t steps = 0, refreshes = 0, outers = 0, launches = 0;
   int steps_in_round = 0;
   bool after_outer = false;
+  bool rot_valid = false;       // the rotation matrices in the workspace were written by a refresh of this context
   bool p_copies_stale = false;  // the caller may have restored P: the bf16 operand copies are remade before the next use
   std::string err;
 
@@ -923,7 +927,11 @@ int run_plan_step(lordo_ctx* c, const PlanStep& s, GemmScalars sc, cudaStream_t 
   return LORDO_OK;
 }
 
-// Makes the device copy of the gradient pointer table current.
+// Makes the device copy of the gradient pointer table (and of the gradients' tensor maps) current.
+// The pinned staging tables have two slots, each with an event recorded behind its last copy, so a
+// change of pointers waits at most for the copy made two changes ago, never for the whole stream.
+// Nothing of the context is updated until every tensor map has been encoded: a failed call leaves
+// the previous tables in force and is not mistaken for "same pointers" on a retry.
 int set_gradients(lordo_ctx* c, const void* const* G, cudaStream_t st) {
   bool same = true;
   for (int i = 0; i < c->n_mats; ++i) {
@@ -932,19 +940,29 @@ int set_gradients(lordo_ctx* c, const void* const* G, cudaStream_t st) {
     if (G[i] != c->last_G[i]) same = false;
   }
   if (same) return LORDO_OK;
-  // the pinned table may still be read by an earlier copy on another stream: wait for this one
-  CUDA_OK(c, cudaStreamSynchronize(st));
-  for (int i = 0; i < c->n_mats; ++i) { c->h_Gtab[i] = G[i]; c->last_G[i] = G[i]; }
-  CUDA_OK(c, cudaMemcpyAsync(c->d_Gtab, c->h_Gtab, sizeof(void*) * c->n_mats, cudaMemcpyHostToDevice, st));
+  const int slot = c->g_slot ^ 1;
+  if (c->g_slot_used[slot]) CUDA_OK(c, cudaEventSynchronize(c->g_slot_ev[slot]));
+  const void** tab = c->h_Gtab + (size_t)slot * c->n_mats;
+  TmaGradMaps* gm = c->tma ? c->h_gmaps + (size_t)slot * c->n_mats : nullptr;
   if (c->tma) {
     for (int i = 0; i < c->n_mats; ++i) {
       const lordo_mat& a = c->mats[i];
-      if (!encode_map3(c->h_gmaps[i].g_sw, G[i], a.n, a.m, c->K, 64, 64, true) ||
-          !encode_map3(c->h_gmaps[i].g_kb, G[i], a.n, a.m, c->K, 64, 128, true))
+      if (!encode_map3(gm[i].g_sw, G[i], a.n, a.m, c->K, 64, 64, true) || !encode_map3(gm[i].g_kb, G[i], a.n, a.m, c->K, 64, 128, true))
         return fail(c, LORDO_ERR_CUDA, "tensor map encoding failed for a gradient");
     }
-    CUDA_OK(c, cudaMemcpyAsync(c->d_gmaps, c->h_gmaps, sizeof(TmaGradMaps) * c->n_mats, cudaMemcpyHostToDevice, st));
   }
+  for (int i = 0; i < c->n_mats; ++i) tab[i] = G[i];
+  cudaError_t e = cudaMemcpyAsync(c->d_Gtab, tab, sizeof(void*) * c->n_mats, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && c->tma) e = cudaMemcpyAsync(c->d_gmaps, gm, sizeof(TmaGradMaps) * c->n_mats, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaEventRecord(c->g_slot_ev[slot], st);
+  if (e != cudaSuccess) {
+    // the device tables may be half written: force the next call to write them again
+    c->last_G.assign(c->n_mats, nullptr);
+    return fail(c, LORDO_ERR_CUDA, std::string("gradient tables: ") + cudaGetErrorString(e));
+  }
+  c->g_slot = slot;
+  c->g_slot_used[slot] = true;
+  for (int i = 0; i < c->n_mats; ++i) c->last_G[i] = G[i];
   return LORDO_OK;
 }
 
@@ -1020,7 +1038,9 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   if (need > workspace_bytes) { delete c; return LORDO_ERR_NOMEM; }
 
   auto bail = [&](int code) { lordo_destroy(c); return code; };
-  if (cudaHostAlloc((void**)&c->h_Gtab, sizeof(void*) * c->n_mats, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
+  if (cudaHostAlloc((void**)&c->h_Gtab, 2 * sizeof(void*) * c->n_mats, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
+  for (int sl = 0; sl < 2; ++sl)
+    if (cudaEventCreateWithFlags(&c->g_slot_ev[sl], cudaEventDisableTiming) != cudaSuccess) return bail(LORDO_ERR_CUDA);
   if (cudaHostAlloc((void**)&c->h_status, 256, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
 
   std::vector<long long> cs, ms, wb, sb;
@@ -1096,7 +1116,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         INIT_CUDA(cudaMemcpyAsync(c->d_maps, hm.data(), sizeof(TmaMatMaps) * nm, cudaMemcpyHostToDevice, st));
         INIT_CUDA(cudaStreamSynchronize(st));
         INIT_CUDA(tma_configure());
-        if (cudaHostAlloc((void**)&c->h_gmaps, sizeof(TmaGradMaps) * nm, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
+        if (cudaHostAlloc((void**)&c->h_gmaps, 2 * sizeof(TmaGradMaps) * nm, cudaHostAllocDefault) != cudaSuccess) return bail(LORDO_ERR_NOMEM);
       } else {
         return bail(LORDO_ERR_CUDA);  // tensor maps could not be encoded (driver without cuTensorMapEncodeTiled?)
       }
@@ -1338,6 +1358,7 @@ int lordo_refresh_subspace(lordo_ctx* c, const void* const* G, float beta1, void
   }
   c->refreshes += 1;
   c->after_outer = false;
+  c->rot_valid = true;
   return LORDO_OK;
 }
 
@@ -1357,7 +1378,7 @@ int lordo_diagnostics(lordo_ctx* c, float* mssv_dev, float* e_norm_dev, void* st
   if (!mssv_dev && !e_norm_dev) return fail(c, LORDO_ERR_INVALID_ARG, "nothing requested");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (mssv_dev) {
-    if (c->refreshes == 0) return fail(c, LORDO_ERR_STATE, "no refresh has run yet: there is no rotation matrix");
+    if (!c->rot_valid) return fail(c, LORDO_ERR_STATE, "no refresh has run on this context yet: there is no rotation matrix");
     launch_mssv(c->d_diag, (int)c->h_diag.size(), mssv_dev, st);
     c->launches += 1;
   }
@@ -1394,7 +1415,10 @@ int lordo_set_counters(lordo_ctx* c, const int64_t in[4]) {
   if (c->cfg.time_buffer && in[3] != 0)
     return fail(c, LORDO_ERR_UNSUPPORTED, "time_buffer: the accumulators live in the workspace, so a checkpoint can only be restored at a round boundary");
   c->steps = in[0]; c->refreshes = in[1]; c->outers = in[2]; c->steps_in_round = (int)in[3];
-  c->after_outer = false;
+  // Global rule: a checkpoint taken between lordo_outer_step and lordo_refresh_subspace still owes its
+  // refresh; the counters show it (a round boundary with one refresh fewer than synchronisations)
+  c->after_outer = c->cfg.variant == LORDO_GLOBAL && in[3] == 0 && in[2] > 0 && in[1] < in[2];
+  c->rot_valid = false;  // the rotation matrices are workspace state and were not restored
   c->p_copies_stale = true;  // a restored checkpoint brings its own P
   return LORDO_OK;
 }
@@ -1435,6 +1459,8 @@ int lordo_destroy(lordo_ctx* c) {
   if (c->h_Gtab) cudaFreeHost(c->h_Gtab);
   if (c->h_status) cudaFreeHost(c->h_status);
   if (c->h_gmaps) cudaFreeHost(c->h_gmaps);
+  for (int sl = 0; sl < 2; ++sl)
+    if (c->g_slot_ev[sl]) cudaEventDestroy(c->g_slot_ev[sl]);
   for (const lordo_ctx::Span& sp : c->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;

@@ -48,7 +48,12 @@ __global__ void __launch_bounds__(256) static_finalize_kernel(const double* __re
     if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
     __syncthreads();
   }
-  if (threadIdx.x == 0) coef[0] = rho > 0.f ? fminf(1.f, rho / ((float)sqrt(red[0]) + 1e-6f)) : 1.f;
+  if (threadIdx.x == 0) {
+    // a NaN or infinite sum of squares has no coefficient: report NaN instead of fminf's silent 1
+    const double ss = red[0];
+    const bool finite = ss == ss && ss < 1.7e308;
+    coef[0] = !finite ? __int_as_float(0x7fc00000) : (rho > 0.f ? fminf(1.f, rho / ((float)sqrt(ss) + 1e-6f)) : 1.f);
+  }
 }
 
 std::mutex g_setup_mutex;
@@ -56,6 +61,7 @@ double* g_partials_addr[kMaxDevices] = {nullptr};
 
 // Device address of the static array on the current device, looked up once per device.
 // (In host code the array's name is only a handle for this lookup, never a device pointer.)
+// The address is cached for the life of the process: it does not survive a cudaDeviceReset.
 int static_scratch(double** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LORDO_ERR_CUDA;
@@ -90,6 +96,7 @@ int lordo_clip_coefficient_static(const void* G_dev, int g_dtype, int64_t count,
   if (rc != LORDO_OK) return rc;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int chunks = (int)((count + kStaticChunk - 1) / kStaticChunk);
+  if (cudaPeekAtLastError() != cudaSuccess) return LORDO_ERR_CUDA;  // an earlier, unrelated error: not reported as this call's
   static_sumsq_kernel<<<chunks, 256, 0, st>>>(G_dev, g_dtype, count, partial);
   static_finalize_kernel<<<1, 256, 0, st>>>(partial, chunks, rho, coef_out_dev);
   return cudaPeekAtLastError() == cudaSuccess ? LORDO_OK : LORDO_ERR_CUDA;

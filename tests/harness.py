@@ -123,21 +123,74 @@ def sync_oracle_from_gpu(opt, orc: lo.LordoOracle) -> None:
             orc.B[i] = _np_state(opt.B[i])
 
 
-def run_lockstep_refresh(spec: RunSpec):
+def range_finder_bf16_rhs(S: np.ndarray, Omega: Optional[np.ndarray], P_start: Optional[np.ndarray], q: int) -> np.ndarray:
+    """The oracle's range finder (same steps, same Householder QR, fp64) with the right-hand side of every
+    product after the first rounded to bf16 before it is multiplied, which is the one thing the tensor-core
+    refresh does differently from the plain definition (the integer sketch Omega is exact in bf16).
+    Omega given: P' = qr(S Omega), then q iterations; Omega None: q iterations from P_start (warm start)."""
+    P = lo.householder_qr_q(S @ Omega) if Omega is not None else np.asarray(P_start, dtype=np.float64)
+    for _ in range(q):
+        Z = lo.householder_qr_q(S.T @ lo.round_bf16(P))
+        P = lo.householder_qr_q(S @ lo.round_bf16(Z))
+    return P
+
+
+def run_lockstep_refresh(spec: RunSpec, rounded_signal: bool = False, inject_delta=None):
     """Runs both sides through the whole schedule; before every subspace refresh the oracle is given
     the CUDA path's state, so that each refresh is compared on identical inputs (the signal of a
     refresh is itself the product of many rounding-sensitive steps). Returns the worst metrics seen
-    directly after a refresh."""
+    directly after a refresh.
+
+    Besides the state comparison, every refresh that rotates is checked on the CUDA path's own new
+    basis: `rot_u`, `rot_v` compare its rotated moments with the oracle's rotation lines applied to
+    the pre-refresh moments, the pre-refresh basis and the basis the CUDA path itself returned, so
+    that they measure the rotation alone, whatever the two range finders disagree on.
+
+    rounded_signal: the oracle's range finder is fed the signal rounded to bf16, which is what the
+    tensor-core sketch of the CUDA path multiplies (Global: bf16(Delta); Local: bf16 of the fp32
+    value c*G + E), so that `P_angle` shows what the two sides do differently with the same signal.
+    `P_angle_bf16rhs` is then the angle to range_finder_bf16_rhs of that signal: the oracle's steps in
+    the operand precision of the tensor-core products.
+
+    inject_delta(round, matrix) -> [m, n] array: Global rule only; the pseudo-gradient both sides refresh
+    from is replaced by this array after the synchronisation (Delta is a caller-owned buffer), so that
+    the range finder can be tested on a signal of chosen spectrum."""
     wl = spec.wl
     opt, orc = make_gpu(spec), make_oracle(spec)
     lr, b1, om = f32(spec.lr), f32(spec.beta1), f32(spec.omega)
     worst: Dict[str, float] = {}
 
-    def after_refresh(signals=None):
+    def before_refresh():
+        torch.cuda.synchronize()
+        sync_oracle_from_gpu(opt, orc)
+        return {"P": [p.copy() for p in orc.P], "u": [x.copy() for x in orc.u], "v": [x.copy() for x in orc.v], "s": orc.s,
+                "refreshes": orc.refreshes}
+
+    def after_refresh(pre, signals=None):
         torch.cuda.synchronize()
         st = compare_states(opt, orc)
         for k in ("P_angle", "P_orth", "u", "v"):
             worst[k] = max(worst.get(k, 0.0), st[k])
+        if rounded_signal and signals is not None and spec.oversample == 0:
+            q = max(wl.power_iters, 1) if spec.warm_start else wl.power_iters
+            for i, (m, n, r) in enumerate(wl.mats):
+                Pg = _np_state(opt.P[i])
+                for k, S in enumerate(signals[i]):
+                    Om = None if spec.warm_start else lo.random_matrix(spec.seed, lo.PURPOSE_OMEGA, i, pre["refreshes"], k, n, r)
+                    Po = pre["P"][i][k] if Pg.ndim == 3 else pre["P"][i]
+                    want = range_finder_bf16_rhs(S, Om, Po, q)
+                    worst["P_angle_bf16rhs"] = max(worst.get("P_angle_bf16rhs", 0.0),
+                                                   largest_principal_angle(want, Pg[k] if Pg.ndim == 3 else Pg))
+        if pre["s"] > 0:
+            for i in range(len(wl.mats)):
+                Pg = _np_state(opt.P[i])
+                ug, vg = _np_state(opt.u[i]), _np_state(opt.v[i])
+                for k in range(wl.K):
+                    Pn = Pg[k] if Pg.ndim == 3 else Pg
+                    Po = pre["P"][i][k] if Pg.ndim == 3 else pre["P"][i]
+                    un, vn = lo.rotate_moments(pre["u"][i][k], pre["v"][i][k], Pn, Po, b1, orc.cfg.beta2, pre["s"])
+                    worst["rot_u"] = max(worst.get("rot_u", 0.0), scaled_error(ug[k], un))
+                    worst["rot_v"] = max(worst.get("rot_v", 0.0), scaled_error(vg[k], vn))
         if signals is not None:
             # share of the signal's energy that the CUDA path's subspace captures, relative to the
             # oracle's subspace for the same signal and sketch
@@ -153,8 +206,14 @@ def run_lockstep_refresh(spec: RunSpec):
         coef = lo.clip_coefficients(G, orc.cfg.clip_rho, orc.cfg.clip_scope)
         out = []
         for i in range(len(wl.mats)):
-            out.append([coef[i, k] * np.asarray(G[i][k], dtype=np.float64) + (orc.E[i][k] if spec.error_feedback else 0.0)
-                        for k in range(wl.K)])
+            per = []
+            for k in range(wl.K):
+                S = coef[i, k] * np.asarray(G[i][k], dtype=np.float64) + (orc.E[i][k] if spec.error_feedback else 0.0)
+                if rounded_signal:  # c in fp32, one fp32 rounding of c*g + e, then bf16
+                    S = float(np.float32(coef[i, k])) * np.asarray(G[i][k], dtype=np.float64) + (orc.E[i][k] if spec.error_feedback else 0.0)
+                    S = lo.round_bf16(S.astype(np.float32))
+                per.append(S)
+            out.append(per)
         return out
 
     for rnd in range(spec.n_rounds):
@@ -162,23 +221,34 @@ def run_lockstep_refresh(spec: RunSpec):
             G = synth.gradients(wl, spec.seed, rnd, h)
             Gd = device_grads(wl, G)
             if spec.variant == 1 and h == 0:
-                torch.cuda.synchronize()
-                sync_oracle_from_gpu(opt, orc)
+                pre = before_refresh()
                 sig = local_signals(G)
                 opt.refresh_subspace(Gd, spec.beta1)
-                orc.refresh_subspace(G, b1)
-                after_refresh(sig)
+                if rounded_signal:  # hand the oracle the rounded signal as a bare gradient
+                    keep = (orc.cfg.clip_rho, orc.cfg.error_feedback)
+                    orc.cfg.clip_rho, orc.cfg.error_feedback = 0.0, False
+                    orc.refresh_subspace([np.stack(per) for per in sig], b1)
+                    orc.cfg.clip_rho, orc.cfg.error_feedback = keep
+                else:
+                    orc.refresh_subspace(G, b1)
+                after_refresh(pre, sig)
             opt.inner_step(Gd, spec.lr, spec.beta1, spec.omega, spec.form)
             orc.inner_step(G, lr, b1, om, spec.form)
         opt.outer_step()
         orc.outer_step()
         if spec.variant == 0:
-            torch.cuda.synchronize()
-            sync_oracle_from_gpu(opt, orc)
+            if inject_delta is not None:
+                torch.cuda.synchronize()
+                for i in range(len(wl.mats)):
+                    opt.Delta[i].copy_(torch.from_numpy(np.asarray(inject_delta(rnd, i), dtype=np.float32)))
+            pre = before_refresh()
+            if rounded_signal:
+                for i in range(len(wl.mats)):
+                    orc.Delta[i] = lo.round_bf16(orc.Delta[i])
             sig = [[orc.Delta[i].copy()] for i in range(len(wl.mats))]
             opt.refresh_subspace(None, spec.beta1)
             orc.refresh_subspace(None, b1)
-            after_refresh(sig)
+            after_refresh(pre, sig)
     torch.cuda.synchronize()
     return opt, orc, worst
 
@@ -195,6 +265,18 @@ def weight_error(got: np.ndarray, want: np.ndarray) -> float:
     rms = float(np.sqrt(np.mean(want ** 2)))
     den = np.maximum(np.abs(want), rms + 1e-30)
     return float(np.max(np.abs(got - want) / den))
+
+
+def weight_error_strict(got: np.ndarray, want: np.ndarray) -> float:
+    """The same ratio with the floor at 1e-2 * rms(b): tells a 1e-6 from a 1e-3 absolute error on
+    the small weights, which the rms floor cannot."""
+    rms = float(np.sqrt(np.mean(want ** 2)))
+    den = np.maximum(np.abs(want), 1e-2 * rms + 1e-30)
+    return float(np.max(np.abs(got - want) / den))
+
+
+def frobenius_error(got: np.ndarray, want: np.ndarray) -> float:
+    return float(np.linalg.norm(got - want) / (np.linalg.norm(want) + 1e-300))
 
 
 def scaled_error(got: np.ndarray, want: np.ndarray) -> float:
@@ -221,10 +303,13 @@ def bf16_ulp_distance(got: np.ndarray, want: np.ndarray) -> np.ndarray:
 
 def compare_states(opt, orc: lo.LordoOracle) -> Dict[str, float]:
     """Worst-case metrics over all matrices between the CUDA state and the oracle state."""
-    out = {"W": 0.0, "E": 0.0, "u": 0.0, "v": 0.0, "X0": 0.0, "Delta": 0.0, "B": 0.0, "P_angle": 0.0, "P_orth": 0.0,
-           "P_cols": 0.0}
+    out = {"W": 0.0, "W_strict": 0.0, "W_fro": 0.0, "E": 0.0, "u": 0.0, "v": 0.0, "X0": 0.0, "Delta": 0.0, "B": 0.0,
+           "P_angle": 0.0, "P_orth": 0.0, "P_cols": 0.0}
     for i in range(len(orc.cfg.mats)):
-        out["W"] = max(out["W"], weight_error(_np_state(opt.W[i]), orc.W[i]))
+        Wg = _np_state(opt.W[i])
+        out["W"] = max(out["W"], weight_error(Wg, orc.W[i]))
+        out["W_strict"] = max(out["W_strict"], weight_error_strict(Wg, orc.W[i]))
+        out["W_fro"] = max(out["W_fro"], frobenius_error(Wg, orc.W[i]))
         if opt.E[i] is not None:
             out["E"] = max(out["E"], scaled_error(_np_state(opt.E[i]), orc.E[i]))
         out["u"] = max(out["u"], scaled_error(_np_state(opt.u[i]), orc.u[i]))

@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import lordo_oracle as lo
 from paper_2602_04396_b200 import synth
 from tests import harness as hz
 from tests.harness import RunSpec
@@ -39,6 +40,8 @@ def test_static_clip_coefficient_matches_inner_step(dt):
         lordo.clip_coefficient_static(Gd[0], rho, out)
         got = float(out.item())
         assert abs(got - want) <= 1e-6 * max(want, 1e-30), (step, got, want)
+        oracle_c = float(lo.clip_coefficients([np.asarray(hz._np_state(Gd[0]))], rho, 0)[0, 0])  # the definition, on the stored values
+        assert abs(got - oracle_c) <= 2e-6 * oracle_c, (step, got, oracle_c)
     assert want == 1.0  # the second call must not carry the first call's large partial sums
 
 
