@@ -103,7 +103,7 @@ struct lordo_ctx {
   long long* d_prep_start = nullptr;
   char* d_tc_bf16 = nullptr;  // all bf16 operand copies, zeroed once by lordo_init
   size_t tc_bf16_bytes = 0;
-  long long tc_strips = 0, prep_blocks = 0;
+  long long tc_strips = 0, tc_strips_p = 0, prep_blocks = 0;
   int tc_rn_max = 0, tc_rk_max = 0;
   // TMA-fed kernels (bf16 storage): tensor maps per matrix, gradient maps re-encoded per pointer change
   bool tma = false;
@@ -334,7 +334,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   for (int i = 0; i < n_mats; ++i)  // ranks above 512 (above 256 with fp32 storage) run on the fp32 path
     if (cfg.mats[i].r > (cfg.w_dtype == LORDO_BF16 ? 512 : 256)) c->tc = false;
   c->h_tc.clear(); c->h_prep.clear(); c->h_prep_start.assign(1, 0);
-  c->tc_strips = 0; c->tc_rn_max = 0; c->tc_rk_max = 0;
+  c->tc_strips = 0; c->tc_strips_p = 0; c->tc_rn_max = 0; c->tc_rk_max = 0;
   if (c->tc) {
     auto up = [](long long x, long long q) { return (x + q - 1) / q * q; };
     (void)cv.take<char>(0);
@@ -348,6 +348,8 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       const size_t n_pad = (size_t)up(md.n, 128);  // whole strips: the TMA-fed kernels store these per strip
       __nv_bfloat16* gT16 = cv.take<__nv_bfloat16>((size_t)K * n_pad * r_k);
       __nv_bfloat16* uT16 = cv.take<__nv_bfloat16>((size_t)K * n_pad * r_k);
+      const int nsplit = (cfg.w_dtype == LORDO_BF16 && r_n > 256) ? 2 : 1;  // TMA-fed projection: one strip per half of the rank
+      float* dcol2 = nsplit == 2 ? cv.take<float>((size_t)K * md.n) : nullptr;
       if (r_n > c->tc_rn_max) c->tc_rn_max = r_n;
       if (r_k > c->tc_rk_max) c->tc_rk_max = r_k;
       for (int k = 0; k < copies; ++k) {
@@ -378,8 +380,10 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         tp.G_ind = c->d_Gtab + i; tp.G_off = wo;
         tp.cptr = c->d_coef + (size_t)i * K + k;
         tp.mat = i; tp.replica = k; tp.pcopy = pk;
+        tp.strip_start_p = c->tc_strips_p; tp.nsplit = nsplit; tp.dcol2 = dcol2 ? dcol2 + (long long)k * md.n : nullptr;
         c->h_tc.push_back(tp);
         c->tc_strips += (md.n + 127) / 128;
+        c->tc_strips_p += (long long)nsplit * ((md.n + 127) / 128);
       }
     }
     c->d_tc_bf16 = ws ? reinterpret_cast<char*>(ws) + bf16_begin : nullptr;
@@ -1196,7 +1200,7 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
       const int big = c->tc_rn_max > 256;
       {
         ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
-        launch_project_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, big, c->d_status, st);
+        launch_project_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips_p, c->d_maps, c->d_gmaps, ss, c->sm_count, c->d_status, st);
       }
       {
         ProfScope ps(c, st, PC_APPLY);

@@ -92,6 +92,11 @@ struct TcProblem {
   const float* cptr;           // clip coefficient
   int mat, replica, pcopy, pad;  // matrix index, worker index, which copy of P (0 for Global)
   float* tb;                   // [r][n] time buffer of this worker (+= lr * U~ every step), or null
+  // the projection's own strip numbering: nsplit strips per 128 columns (2 when 256 < r <= 512: one per
+  // half of the rank), and the second half's share of the column scale of the full-rank QHM term
+  long long strip_start_p;
+  float* dcol2;                // [n], or null when nsplit == 1
+  int nsplit, pad2;
 };
 
 // Tensor maps (opaque 128-byte objects encoded on the host) of one matrix for the TMA-fed kernels.
@@ -130,8 +135,8 @@ void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips,
 
 // TMA-fed persistent kernels for bf16 storage (lordo_tma.cu).
 cudaError_t tma_configure();
-void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                        const StepScalars& sc, int grid, int big, unsigned* status, cudaStream_t st);
+void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips_p, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
+                        const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
 // mode 0: r <= 256, one sweep; modes 1 and 2: the two sweeps for 256 < r <= 512
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
                       const StepScalars& sc, int grid, int mode, unsigned* status, cudaStream_t st);

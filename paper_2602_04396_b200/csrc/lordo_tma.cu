@@ -5,7 +5,8 @@
 //                       memory, four warps turn the G tile into c*G + E in place (16-byte vector
 //                       operations, layout-agnostic), and the tile is consumed as an MN-major
 //                       operand by tcgen05.mma. Two accumulator buffers in tensor memory let the
-//                       moment-update epilogue of one strip run under the main loop of the next.
+//                       moment-update epilogue of one strip run under the main loop of the next
+//                       (ranks above 256 as two half-rank strips, see the kernel).
 //   apply_tma_kernel    The strip's two low-rank operands (g^T, U~^T) live in tensor memory as the
 //                       A operands; rows of P and the tiles of G, E, W arrive by TMA; the epilogue
 //                       works on the swizzled tiles in shared memory (four neighbouring columns per
@@ -33,6 +34,16 @@ __device__ __forceinline__ int find_problem(const TcProblem* __restrict__ probs,
   return lo;
 }
 
+// the projection numbers its strips on its own: a problem with 256 < r <= 512 has two per 128 columns
+__device__ __forceinline__ int find_problem_p(const TcProblem* __restrict__ probs, int nprobs, long long strip) {
+  int lo = 0, hi = nprobs - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (probs[mid].strip_start_p <= strip) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
 __device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
 
@@ -54,17 +65,20 @@ constexpr int kAThreads = (3 + kAEpiWarps) * 32;  // 608: TMA inputs, MMA, 16 ep
 }  // namespace
 
 // =================================================================================================
-// BIG: 256 < r <= 512. The accumulator then fills all 512 columns of tensor memory (one buffer, no
-// overlap of the epilogue with the next strip) and a stage holds a 64 KB P^T tile (two stages).
-template <bool BIG>
+// 256 < r <= 512: the accumulator of a whole strip would fill all 512 columns of tensor memory and leave
+// no second buffer, so such a problem is dealt out as two strips per 128 columns, one per half of the
+// rank (rows [0, 256) and [256, r) of P^T, of the moments and of the low-rank operands). The two halves
+// are neighbours in the strip list, hence run on neighbouring CTAs at the same time, and the second
+// read of the G and E tiles is served by L2. Each half is then the r <= 256 pipeline: three stages, two
+// accumulator buffers, the moment epilogue of one strip under the main loop of the next.
 __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
                                                                    const TmaMatMaps* __restrict__ maps,
                                                                    const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
                                                                    unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int ST = BIG ? 2 : 3;
-  constexpr uint32_t SB = BIG ? 98304u : kPStageBytes;
+  constexpr int ST = kPStages;
+  constexpr uint32_t SB = kPStageBytes;
   __shared__ uint64_t full_bar[3], xform_bar[3], empty_bar[3], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ float dsum_s[kStrip];
@@ -89,13 +103,14 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       uint32_t it = 0;
       bool ok = true;
       for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
-        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
-        const int n0 = (int)(strip - pr->strip_start) * kStrip;
+        const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
+        const int l = (int)(strip - pr->strip_start_p);
+        const int n0 = (pr->nsplit == 2 ? l >> 1 : l) * kStrip, r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
         const TmaMatMaps* mm = maps + pr->mat;
         const TmaGradMaps* gm = gmaps + pr->mat;
         const int nkb = pr->m_k / 64, rep = pr->replica, pc = pr->pcopy;
         const int pt_rows = pr->r_n < 256 ? pr->r_n : 256;  // rows of one P^T box
-        const uint32_t tx = 16384u + (ef ? 16384u : 0u) + (uint32_t)pt_rows * 128u * (BIG ? 2u : 1u);
+        const uint32_t tx = 16384u + (ef ? 16384u : 0u) + (uint32_t)pt_rows * 128u;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % ST;
           ok = mbar_wait(&empty_bar[s], ((it / ST) & 1u) ^ 1u, status);
@@ -108,8 +123,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
             tma_load_3d(base + 16384, mm->e_sw, n0, kb * 64, rep, &full_bar[s]);
             tma_load_3d(base + 24576, mm->e_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
           }
-          tma_load_3d(base + 32768, mm->pt, kb * 64, 0, pc, &full_bar[s]);
-          if (BIG) tma_load_3d(base + 32768 + pt_rows * 128, mm->pt, kb * 64, 256, pc, &full_bar[s]);
+          tma_load_3d(base + 32768, mm->pt, kb * 64, r_lo, pc, &full_bar[s]);  // rows past r_n arrive as zeros
         }
       }
     }
@@ -119,13 +133,14 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       uint32_t it = 0, si = 0;
       bool ok = true;
       for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
-        const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+        const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
+        const int l = (int)(strip - pr->strip_start_p);
+        const int r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
         const int nkb = pr->m_k / 64;
-        const uint32_t n_lo = pr->r_n < 256 ? (uint32_t)pr->r_n : 256u, n_hi = (uint32_t)pr->r_n - n_lo;
-        const uint32_t idesc = idesc_bf16_f32(128, n_lo) | kIdescAMajorMN;
-        const uint32_t idesc_hi = idesc_bf16_f32(128, n_hi ? n_hi : 16u) | kIdescAMajorMN;
-        const uint32_t buf = BIG ? 0u : (si & 1u);
-        ok = mbar_wait(&acc_empty[buf], ((BIG ? si : (si >> 1)) & 1u) ^ 1u, status);
+        const uint32_t n_h = (uint32_t)(pr->r_n - r_lo < 256 ? pr->r_n - r_lo : 256);
+        const uint32_t idesc = idesc_bf16_f32(128, n_h) | kIdescAMajorMN;
+        const uint32_t buf = si & 1u;
+        ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
         if (!ok) break;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % ST;
@@ -134,11 +149,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           tc_fence_after_sync();
           const uint32_t sA = smem_u32(smem + s * SB), sB = sA + 32768;
 #pragma unroll
-          for (int k16 = 0; k16 < 4; ++k16) {
-            const uint32_t acc = (kb > 0 || k16 > 0) ? 1u : 0u;
-            mma_bf16(tmem + buf * 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc, acc);
-            if (BIG && n_hi) mma_bf16(tmem + 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + 256 * 128 + k16 * 32), idesc_hi, acc);
-          }
+          for (int k16 = 0; k16 < 4; ++k16)
+            mma_bf16(tmem + buf * 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
           mma_commit(&empty_bar[s]);
         }
         if (ok) mma_commit(&acc_full[buf]);
@@ -150,7 +162,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
     uint32_t it = 0;
     bool ok = true;
     for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
-      const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
+      const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
       const int nkb = pr->m_k / 64;
       const float c = *pr->cptr;
       for (int kb = 0; kb < nkb; ++kb, ++it) {
@@ -184,29 +196,32 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
     uint32_t si = 0;
     bool ok = true;
     for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
-      const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
-      const int n = pr->n, r = pr->r, r_n = pr->r_n, r_k = pr->r_k;
-      const long long n0 = (strip - pr->strip_start) * kStrip;
+      const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
+      const int l = (int)(strip - pr->strip_start_p);
+      const int cs = pr->nsplit == 2 ? l >> 1 : l, r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
+      const int n = pr->n, r = pr->r, r_k = pr->r_k;
+      const int rn_h = pr->r_n - r_lo < 256 ? pr->r_n - r_lo : 256;  // rank rows of this strip, padded to 16
+      const long long n0 = (long long)cs * kStrip;
       const long long ecol = n0 + q * 32 + lane;
       const bool e_ok = ecol < n;
       const long long ecolc = e_ok ? ecol : (long long)n - 1;
       float* __restrict__ up_ = pr->u;
       float* __restrict__ vp_ = pr->v;
       float* __restrict__ tb_ = pr->tb;
-      // this column's 16-byte pieces inside the strip's block [r_k/8][128][8]
-      const size_t lr_off = (size_t)(strip - pr->strip_start) * (size_t)r_k * 128 + (size_t)(q * 32 + lane) * 8;
+      // this column's 16-byte pieces inside the strip's block [r_k/8][128][8], from k-chunk r_lo/8 on
+      const size_t lr_off = (size_t)cs * (size_t)r_k * 128 + (size_t)r_lo * 128 + (size_t)(q * 32 + lane) * 8;
       __nv_bfloat16* __restrict__ gT = pr->gT16 + lr_off;
       __nv_bfloat16* __restrict__ uT = pr->uT16 + lr_off;
-      const uint32_t buf = BIG ? 0u : (si & 1u);
-      ok = mbar_wait<64>(&acc_full[buf], (BIG ? si : (si >> 1)) & 1u, status);
+      const uint32_t buf = si & 1u;
+      ok = mbar_wait<64>(&acc_full[buf], (si >> 1) & 1u, status);
       if (!ok) break;
       tc_fence_after_sync();
       float dsum = 0.f;
-      for (int ch = half; ch < r_n / 16; ch += 2) {
+      for (int ch = half; ch < rn_h / 16; ch += 2) {
         float u[16], v[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const size_t idx = (size_t)(unsigned)min(ch * 16 + i, r - 1) * (size_t)n + (size_t)ecolc;
+          const size_t idx = (size_t)(unsigned)min(r_lo + ch * 16 + i, r - 1) * (size_t)n + (size_t)ecolc;
           u[i] = up_[idx];
           v[i] = vp_[idx];
         }
@@ -218,7 +233,7 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           float o[2];
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
-            const int row = ch * 16 + i + t;
+            const int row = r_lo + ch * 16 + i + t;
             const float gg = g[i + t];
             const float un = b1 * u[i + t] + (1.f - b1) * gg;
             const float vn = b2 * v[i + t] + (1.f - b2) * gg * gg;
@@ -247,10 +262,10 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       }
       tc_fence_before_sync();
       mbar_arrive(&acc_empty[buf]);
-      if (sc.form == LORDO_QHM_FULL) {  // mu(D): mean over the rank axis, one value per column
+      if (sc.form == LORDO_QHM_FULL) {  // mu(D): mean over the rank axis, one value per column (a split problem: this half's share)
         if (half == 1) dsum_s[q * 32 + lane] = dsum;
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (half == 0 && e_ok) pr->dcol[ecol] = (dsum + dsum_s[q * 32 + lane]) / (float)r;
+        if (half == 0 && e_ok) (r_lo ? pr->dcol2 : pr->dcol)[ecol] = (dsum + dsum_s[q * 32 + lane]) / (float)r;
         asm volatile("bar.sync 1, 256;" ::: "memory");
       }
     }
@@ -272,11 +287,14 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr uint32_t PSB = MODE ? 65536u : kAPStageBytes;  // one stage of rows of P
-  constexpr int INST = MODE ? 2 : kAInStages;
+  constexpr int INST = kAInStages;
   constexpr bool DO_E = MODE != 2, DO_W = MODE != 1;
   constexpr uint32_t A2COL = MODE ? 0u : 128u;             // first column of the U~^T operand
+  // a stage holds the tiles the mode works on: G | E | W (MODE 0), G | E (MODE 1), G | W (MODE 2)
+  constexpr uint32_t ISB = MODE ? 32768u : kAInStageBytes;
+  constexpr uint32_t EOFF = 16384u, WOFF = MODE == 2 ? 16384u : 32768u;
   unsigned char* sP = smem;                      // kAPStages stages of rows of P
-  unsigned char* sIn = smem + kAPStages * PSB;   // INST stages of G | E | W tiles (48 KB each)
+  unsigned char* sIn = smem + kAPStages * PSB;   // INST stages of tiles
   __shared__ uint64_t p_full[kAPStages], p_empty[kAPStages], in_full[kAInStages], in_free[kAInStages], acc_full[2], acc_empty[2], x_ready;
   __shared__ uint32_t tmem_slot;
 
@@ -314,13 +332,13 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           const int is = jt % INST;
           ok = mbar_wait(&in_free[is], ((jt / INST) & 1u) ^ 1u, status);
           if (!ok) break;
-          unsigned char* base = sIn + is * kAInStageBytes;
+          unsigned char* base = sIn + is * ISB;
           const bool ld_e = DO_E && ef;
           mbar_expect_tx(&in_full[is], 16384u + (ld_e ? 16384u : 0u) + (DO_W ? 16384u : 0u));
           for (int hh = 0; hh < 2; ++hh) {  // two 64-column halves per tile, 8 KB each
             tma_load_3d(base + hh * 8192, gm->g_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
-            if (ld_e) tma_load_3d(base + 16384 + hh * 8192, mm->e_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
-            if (DO_W) tma_load_3d(base + 32768 + hh * 8192, mm->w_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+            if (ld_e) tma_load_3d(base + EOFF + hh * 8192, mm->e_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+            if (DO_W) tma_load_3d(base + WOFF + hh * 8192, mm->w_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
           }
         }
       }
@@ -417,7 +435,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const long long ec = (long long)n0 + ecol0 + j;
-        cd[j] = full ? (1.f - om) * c / pr->dcol[ec < n ? ec : (long long)n - 1] : 0.f;
+        const long long ecc = ec < n ? ec : (long long)n - 1;
+        cd[j] = full ? (1.f - om) * c / (pr->dcol[ecc] + (pr->dcol2 ? pr->dcol2[ecc] : 0.f)) : 0.f;
       }
       // this thread's quarter of its column's low-rank operands -> tensor memory (r_k/8 columns each)
       {
@@ -447,7 +466,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       for (int t = 0; t < nsteps; ++t, ++jt) {
         const int is = jt % INST;
         const uint32_t b = jt & 1u;
-        unsigned char* base = sIn + is * kAInStageBytes;
+        unsigned char* base = sIn + is * ISB;
         ok = mbar_wait<32>(&in_full[is], (jt / INST) & 1u, status);
         if (ok) ok = mbar_wait<32>(&acc_full[b], (jt >> 1) & 1u, status);
         if (!ok) break;
@@ -473,8 +492,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
 #pragma unroll
         for (int ri = 0; ri < 4; ++ri) {
           gv[ri] = *reinterpret_cast<const uint2*>(base + toff[ri]);
-          if (DO_E && ef) ev[ri] = *reinterpret_cast<const uint2*>(base + 16384 + toff[ri]);
-          if (DO_W) wv[ri] = *reinterpret_cast<const uint2*>(base + 32768 + toff[ri]);
+          if (DO_E && ef) ev[ri] = *reinterpret_cast<const uint2*>(base + EOFF + toff[ri]);
+          if (DO_W) wv[ri] = *reinterpret_cast<const uint2*>(base + WOFF + toff[ri]);
         }
 #pragma unroll
         for (int ri = 0; ri < 4; ++ri) {
@@ -485,14 +504,14 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
             const float e1 = (c * g1 + bf_hi(ev[ri].x)) - a1[0][4 * k + 2 + p];
             const float e2 = (c * g2 + bf_lo(ev[ri].y)) - a1[1][4 * k + p];
             const float e3 = (c * g3 + bf_hi(ev[ri].y)) - a1[1][4 * k + 2 + p];
-            *reinterpret_cast<uint2*>(base + 16384 + toff[ri]) = make_uint2(pack2_bf16(e0, e1), pack2_bf16(e2, e3));
+            *reinterpret_cast<uint2*>(base + EOFF + toff[ri]) = make_uint2(pack2_bf16(e0, e1), pack2_bf16(e2, e3));
           }
           if (DO_W) {
             const float w0 = bf_lo(wv[ri].x) - lr * (cd[0] * g0 + a2w * a2[0][4 * k + p]);
             const float w1 = bf_hi(wv[ri].x) - lr * (cd[1] * g1 + a2w * a2[0][4 * k + 2 + p]);
             const float w2 = bf_lo(wv[ri].y) - lr * (cd[2] * g2 + a2w * a2[1][4 * k + p]);
             const float w3 = bf_hi(wv[ri].y) - lr * (cd[3] * g3 + a2w * a2[1][4 * k + 2 + p]);
-            *reinterpret_cast<uint2*>(base + 32768 + toff[ri]) = make_uint2(pack2_bf16(w0, w1), pack2_bf16(w2, w3));
+            *reinterpret_cast<uint2*>(base + WOFF + toff[ri]) = make_uint2(pack2_bf16(w0, w1), pack2_bf16(w2, w3));
           }
         }
         // the four warps of a row group hand their 16 rows to the TMA engine on their own
@@ -503,8 +522,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           const int row = t * kARows + grp * 16;
           for (int hh = 0; hh < 2; ++hh) {
             if (n0 + hh * 64 >= n) break;
-            if (DO_E && ef) tma_store_3d(mm->e_st, n0 + hh * 64, row, rep, sb + 16384 + hh * 8192);
-            if (DO_W) tma_store_3d(mm->w_st, n0 + hh * 64, row, rep, sb + 32768 + hh * 8192);
+            if (DO_E && ef) tma_store_3d(mm->e_st, n0 + hh * 64, row, rep, sb + EOFF + hh * 8192);
+            if (DO_W) tma_store_3d(mm->w_st, n0 + hh * 64, row, rep, sb + WOFF + hh * 8192);
           }
           tma_store_commit();
           tma_store_wait_read();
@@ -525,11 +544,9 @@ cudaError_t sketch_configure();
 cudaError_t tma_configure() {
   cudaError_t e = sketch_configure();
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(project_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
+  e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(project_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
-  if (e != cudaSuccess) return e;
-  const int smem = (int)(kAPStages * 65536 + 2 * kAInStageBytes + 1024);  // the largest of the three modes
+  const int smem = (int)(kAPStages * 65536 + kAInStages * 32768 + 1024);  // the largest of the three modes
   e = cudaFuncSetAttribute(apply_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(apply_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -538,15 +555,14 @@ cudaError_t tma_configure() {
 }
 
 void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                        const StepScalars& sc, int grid, int big, unsigned* status, cudaStream_t st) {
+                        const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
   const long long g = total_strips < grid ? total_strips : grid;
-  if (big) project_tma_kernel<true><<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
-  else project_tma_kernel<false><<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+  project_tma_kernel<<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
 }
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
                       const StepScalars& sc, int grid, int mode, unsigned* status, cudaStream_t st) {
   const unsigned g = (unsigned)(total_strips < grid ? total_strips : grid);
-  const size_t small = kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, large = kAPStages * 65536 + 2 * kAInStageBytes + 1024;
+  const size_t small = kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, large = kAPStages * 65536 + kAInStages * 32768 + 1024;
   if (mode == 0) apply_tma_kernel<0><<<g, kAThreads, small, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
   else if (mode == 1) apply_tma_kernel<1><<<g, kAThreads, large, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
   else apply_tma_kernel<2><<<g, kAThreads, large, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
