@@ -35,6 +35,12 @@ Readings of points the paper leaves open (each is restated where it is used):
       basis is truncated to the top-r left singular subspace of its projection of the signal
       (Rayleigh-Ritz), see compute_projection_rr. Not in the paper: the randomized-SVD refinement of
       R1, closer to the paper's SVD definition of the projection at the same rank.
+  R17 Right-side projection (`sides[i] = 1`; not in the paper, which always projects from the left: the
+      side selection of GaLore-type methods for matrices with more rows than columns): the basis Q is
+      q x r, the low-rank gradient is g = (G^ + E) Q (p x r), the moments are p x r, the update is
+      U~ Q^T, the full-rank QHM scale mu(.) runs over the rank axis and gives one value per row, and
+      ComputeProjection returns the top-r right singular subspace (the range finder applied to the
+      transposed signal, sketch p x r). Everything equals the left-side method applied to W^T.
   R15 Up-link time buffer (App. "Worker Communication", the server-side repacked updates): with
       `time_buffer` every worker accumulates T <- T + eta * alpha, alpha being the low-rank update of
       the step (no QHM or low-rank QHM only), and the pseudo-gradient of the synchronisation is
@@ -283,6 +289,7 @@ class OracleConfig:
     warm_start: bool = False   # refresh by block power iteration from the current P (no sketch)
     time_buffer: bool = False  # R15: pseudo-gradient rebuilt from the accumulated low-rank updates
     oversample: int = 0        # R16: extra sketch columns p, Rayleigh-Ritz truncation back to rank r
+    sides: Optional[Tuple[int, ...]] = None  # R17: per matrix, 0 = project from the left (the paper), 1 = from the right
 
 
 class LordoOracle:
@@ -302,25 +309,31 @@ class LordoOracle:
             w0 = store(W0[i], c.w_dtype)
             self.W.append(np.repeat(w0[None], c.K, axis=0))  # all workers start equal (Alg. 1 Require)
             self.E.append(np.zeros((c.K, m, n)))
-            self.u.append(np.zeros((c.K, r, n)))
-            self.v.append(np.zeros((c.K, r, n)))
-            self.T.append(np.zeros((c.K, r, n)))
+            right = self.side(i) == 1
+            lowrank = (c.K, m, r) if right else (c.K, r, n)  # R17: moments are p x r when projecting from the right
+            self.u.append(np.zeros(lowrank))
+            self.v.append(np.zeros(lowrank))
+            self.T.append(np.zeros(lowrank))
             self.X0.append(store(w0, c.state_dtype))
             self.B.append(np.zeros((m, n)))
             self.Delta.append(np.zeros((m, n)))
+            pm = n if right else m  # rows of the basis
             if P0 is not None:
                 p = np.asarray(P0[i], dtype=np.float64)
             elif c.variant == GLOBAL:
                 # R12: random initial projection, orthonormalised
-                p = householder_qr_q(random_matrix(c.seed, PURPOSE_P0, i, 0, 0, m, r))
+                p = householder_qr_q(random_matrix(c.seed, PURPOSE_P0, i, 0, 0, pm, r))
             else:
-                p = np.eye(m, r)  # R12: Q_0 = identity (Algorithm 2 Require)
+                p = np.eye(pm, r)  # R12: Q_0 = identity (Algorithm 2 Require)
             if c.variant == LOCAL and p.ndim == 2:
                 p = np.repeat(p[None], c.K, axis=0)
             self.P.append(store(p, c.state_dtype))
 
     def _P(self, i: int, k: int) -> np.ndarray:
         return self.P[i][k] if self.cfg.variant == LOCAL else self.P[i]
+
+    def side(self, i: int) -> int:
+        return 0 if self.cfg.sides is None else int(self.cfg.sides[i])
 
     # -- Algorithm 1 / 2, the per-step block ------------------------------------------------------
     def inner_step(self, G: Sequence[np.ndarray], lr: float, beta1: float, omega: float, form: int) -> None:
@@ -339,6 +352,9 @@ class LordoOracle:
                 P = self._P(i, k)
                 Ghat = coef[i, k] * np.asarray(G[i][k], dtype=np.float64)  # clipped gradient
                 A = Ghat + self.E[i][k] if c.error_feedback else Ghat
+                if self.side(i) == 1:
+                    self._inner_right(i, k, P, Ghat, A, lr, beta1, omega, form, bc1, bc2)
+                    continue
                 g = P.T @ A  # low-rank gradient with error feedback
                 if c.error_feedback:
                     self.E[i][k] = store(A - P @ g, c.e_dtype)
@@ -364,6 +380,34 @@ class LordoOracle:
                 if c.time_buffer:
                     self.T[i][k] = store(self.T[i][k] + lr * alpha, c.state_dtype)
 
+    def _inner_right(self, i, k, P, Ghat, A, lr, beta1, omega, form, bc1, bc2) -> None:
+        """R17: the per-step lines of Algorithm 1 with the basis applied from the right (P is q x r)."""
+        c = self.cfg
+        g = A @ P  # p x r
+        if c.error_feedback:
+            self.E[i][k] = store(A - g @ P.T, c.e_dtype)
+        u = beta1 * self.u[i][k] + (1.0 - beta1) * g
+        v = c.beta2 * self.v[i][k] + (1.0 - c.beta2) * g * g
+        self.u[i][k] = store(u, c.state_dtype)
+        self.v[i][k] = store(v, c.state_dtype)
+        u_hat = self.u[i][k] / bc1
+        v_hat = self.v[i][k] / bc2
+        D = np.sqrt(v_hat) + c.eps
+        if form == QHM_NONE:
+            alpha = u_hat / D
+            upd = alpha @ P.T
+        elif form == QHM_LOW:
+            alpha = (omega * u_hat + (1.0 - omega) * g) / D
+            upd = alpha @ P.T
+        elif form == QHM_FULL:
+            d = D.mean(axis=1)  # R6 with R17: mean over the rank axis, one value per row
+            upd = (1.0 - omega) * Ghat / d[:, None] + omega * ((u_hat / D) @ P.T)
+        else:
+            raise ValueError(form)
+        self.W[i][k] = store(self.W[i][k] - lr * upd, c.w_dtype)
+        if c.time_buffer:
+            self.T[i][k] = store(self.T[i][k] + lr * alpha, c.state_dtype)
+
     # -- Algorithm 1, the two state-synchronisation lines on their own (K_u, K_v != K_x) ------------
     def sync_states(self, sync_u: bool, sync_v: bool) -> None:
         c = self.cfg
@@ -382,7 +426,10 @@ class LordoOracle:
             if c.sync_v:
                 self.v[i][:] = store(self.v[i].mean(axis=0), c.state_dtype)[None]
             if c.time_buffer:  # R15: (1/M) sum_m Q^m T^m
-                delta = np.mean([self._P(i, k) @ self.T[i][k] for k in range(c.K)], axis=0)
+                if self.side(i) == 1:
+                    delta = np.mean([self.T[i][k] @ self._P(i, k).T for k in range(c.K)], axis=0)
+                else:
+                    delta = np.mean([self._P(i, k) @ self.T[i][k] for k in range(c.K)], axis=0)
                 self.T[i][:] = 0.0
             else:
                 delta = self.X0[i] - self.W[i].mean(axis=0)  # R9
@@ -407,40 +454,40 @@ class LordoOracle:
             coef = clip_coefficients(G, c.clip_rho, c.clip_scope)
         diag = [[] for _ in c.mats]
         for i, (m, n, r) in enumerate(c.mats):
-            if c.variant == GLOBAL:
-                if c.warm_start:
-                    P_new = store(compute_projection_warm(self.Delta[i], self.P[i], c.power_iters), c.state_dtype)
+            right = self.side(i) == 1
+            for k in range(c.K if c.variant == LOCAL else 1):
+                if c.variant == GLOBAL:
+                    S = self.Delta[i]                                          # Algorithm 1: ComputeProjection(Delta)
+                    P_old = self.P[i]
                 else:
-                    Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, 0, n, r + c.oversample)
-                    if c.oversample:
-                        P_new = store(compute_projection_rr(self.Delta[i], Om, c.power_iters, r), c.state_dtype)
-                    else:
-                        P_new = store(compute_projection(self.Delta[i], Om, c.power_iters), c.state_dtype)
-                diag[i].append(mssv(P_new, self.P[i]))
-                if self.s > 0:
-                    for k in range(c.K):
-                        un, vn = rotate_moments(self.u[i][k], self.v[i][k], P_new, self.P[i], beta1, c.beta2, self.s)
-                        self.u[i][k] = store(un, c.state_dtype)
-                        self.v[i][k] = store(vn, c.state_dtype)
-                self.P[i] = P_new
-            else:
-                for k in range(c.K):
-                    S = coef[i, k] * np.asarray(G[i][k], dtype=np.float64)
+                    S = coef[i, k] * np.asarray(G[i][k], dtype=np.float64)     # Algorithm 2: ComputeProjection(G^ + E)
                     if c.error_feedback:
                         S = S + self.E[i][k]
-                    if c.warm_start:
-                        P_new = store(compute_projection_warm(S, self.P[i][k], c.power_iters), c.state_dtype)
+                    P_old = self.P[i][k]
+                if right:
+                    S = S.T  # R17: the right singular subspace of S is the left one of S^T
+                cols = S.shape[1]
+                if c.warm_start:
+                    P_new = store(compute_projection_warm(S, P_old, c.power_iters), c.state_dtype)
+                else:
+                    Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, cols, r + c.oversample)
+                    if c.oversample:
+                        P_new = store(compute_projection_rr(S, Om, c.power_iters, r), c.state_dtype)
                     else:
-                        Om = random_matrix(c.seed, PURPOSE_OMEGA, i, self.refreshes, k, n, r + c.oversample)
-                        if c.oversample:
-                            P_new = store(compute_projection_rr(S, Om, c.power_iters, r), c.state_dtype)
+                        P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
+                diag[i].append(mssv(P_new, P_old))
+                if self.s > 0:
+                    for kk in (range(c.K) if c.variant == GLOBAL else (k,)):
+                        if right:  # the moments are p x r: their transposes are rotated like left-side moments
+                            un, vn = rotate_moments(self.u[i][kk].T, self.v[i][kk].T, P_new, P_old, beta1, c.beta2, self.s)
+                            un, vn = un.T, vn.T
                         else:
-                            P_new = store(compute_projection(S, Om, c.power_iters), c.state_dtype)
-                    diag[i].append(mssv(P_new, self.P[i][k]))
-                    if self.s > 0:
-                        un, vn = rotate_moments(self.u[i][k], self.v[i][k], P_new, self.P[i][k], beta1, c.beta2, self.s)
-                        self.u[i][k] = store(un, c.state_dtype)
-                        self.v[i][k] = store(vn, c.state_dtype)
+                            un, vn = rotate_moments(self.u[i][kk], self.v[i][kk], P_new, P_old, beta1, c.beta2, self.s)
+                        self.u[i][kk] = store(un, c.state_dtype)
+                        self.v[i][kk] = store(vn, c.state_dtype)
+                if c.variant == GLOBAL:
+                    self.P[i] = P_new
+                else:
                     self.P[i][k] = P_new
         self.last_mssv = diag
         self.refreshes += 1

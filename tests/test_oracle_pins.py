@@ -835,3 +835,66 @@ def test_driver_loop_refreshes_local_before_the_step_and_global_after_the_sync()
     # the error buffer after round 2 is orthogonal to the basis that round 2 projected with
     assert np.abs(P1.T @ o.E[0][0]).max() < 1e-9
     assert np.abs(P0.T @ o.E[0][0]).max() > 1e-3
+
+
+# ---------------------------------------------------------------------------------------------
+# R17: projection from the right (not in the paper). Everything it does is fixed by one identity:
+# right-projecting W is left-projecting W^T. The right-side code path of the oracle (g = A Q,
+# E = A - g Q^T, p x r moments, row-wise mu, range finder on the transposed signal) is written out on
+# its own and compared here with the left-side path, which the tests above pin, on transposed inputs.
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("variant", [GLOBAL, LOCAL])
+@pytest.mark.parametrize("form", [QHM_NONE, QHM_LOW, QHM_FULL])
+@pytest.mark.parametrize("opts", [dict(), dict(power_iters=1), dict(warm_start=True), dict(error_feedback=False), dict(time_buffer=True)])
+def test_right_side_projection_is_left_side_projection_of_the_transpose(variant, form, opts):
+    if opts.get("time_buffer") and form == QHM_FULL:
+        pytest.skip("the full-rank form does not factorise (R15)")
+    rng = np.random.default_rng(41)
+    m, n, r, K, H, rounds = 14, 9, 3, 2, 2, 2
+    kw = dict(K=K, H=H, variant=variant, clip_rho=1.5, outer=OUTER_NESTEROV, outer_lr=0.7, outer_momentum=0.9, beta2=0.95, eps=1e-4, seed=6,
+              state_dtype="f64", w_dtype="f64", e_dtype="f64", **opts)
+    W0 = rng.standard_normal((m, n)) * 0.02
+    right = LordoOracle(OracleConfig(mats=((m, n, r),), sides=(1,), **kw), [W0])
+    left = LordoOracle(OracleConfig(mats=((n, m, r),), sides=(0,), **kw), [W0.T.copy()])
+    assert right.P[0].shape == left.P[0].shape  # the basis is q x r on both sides (same generator stream, same shape)
+    assert right.u[0].shape == (K, m, r) and left.u[0].shape == (K, r, m)
+    grads = [[rng.standard_normal((K, m, n)) * (3.0 if h == 0 else 0.2)] for h in range(H * rounds)]
+    lo.run_rounds(right, lambda rnd, h: grads[rnd * H + h], rounds, 0.01, 0.9, 0.7, form)
+    lo.run_rounds(left, lambda rnd, h: [np.swapaxes(grads[rnd * H + h][0], 1, 2)], rounds, 0.01, 0.9, 0.7, form)
+    T = lambda x: np.swapaxes(x, -1, -2)
+    for name in ("W", "E", "u", "v", "X0", "B", "Delta", "T"):
+        a, b = getattr(right, name)[0], T(getattr(left, name)[0])
+        assert np.abs(a - b).max() <= 1e-12 * max(1.0, np.abs(b).max()), name
+    assert np.abs(right.P[0] - left.P[0]).max() < 1e-12
+    assert right.refreshes == left.refreshes == rounds
+    assert np.abs(right.u[0]).max() > 0 and (not kw.get("error_feedback", True) or np.abs(right.E[0]).max() > 0)
+
+
+def test_right_side_identity_basis_reduces_to_adam():
+    m, n = 11, 6
+    cfg, W0 = make([(m, n, n)], K=1, H=1, variant=LOCAL, eps=1e-8, beta2=0.999, sides=(1,))
+    o = LordoOracle(cfg, W0)  # Local: Q_0 = I, here the n x n identity applied from the right
+    assert o.P[0].shape == (1, n, n)
+    grads = [RNG.standard_normal((m, n)) for _ in range(5)]
+    for g in grads:
+        o.inner_step([g[None]], 3e-3, 0.9, 1.0, QHM_NONE)
+    want = _adam_reference(W0[0], grads, 3e-3, 0.9, 0.999, 1e-8)
+    assert np.abs(o.W[0][0] - want).max() < 1e-13 and np.abs(o.E[0]).max() == 0.0
+
+
+def test_right_side_reconstructs_a_gradient_of_low_row_rank():
+    m, n, r = 40, 24, 5
+    cfg, W0 = make([(m, n, r)], K=1, variant=LOCAL, power_iters=1, sides=(1,))
+    o = LordoOracle(cfg, W0)
+    G = [(RNG.standard_normal((m, r)) @ RNG.standard_normal((r, n)))[None]]
+    o.refresh_subspace(G)
+    P = o.P[0][0]
+    assert P.shape == (n, r) and np.abs(P.T @ P - np.eye(r)).max() < 1e-10
+    assert np.linalg.norm(G[0][0] - (G[0][0] @ P) @ P.T) / np.linalg.norm(G[0][0]) < 1e-6  # the row space is captured
+    o.inner_step(G, 1e-3, 0.9, 0.6, QHM_FULL)
+    assert np.abs(o.E[0]).max() < 1e-10 * np.abs(G[0]).max()
+    # full-rank QHM from the right: one scale per ROW (mean over the rank axis of a p x r array)
+    g = G[0][0] @ P
+    d = (np.abs(g) + cfg.eps).mean(axis=1)
+    upd = 0.4 * G[0][0] / d[:, None] + 0.6 * ((g / (np.abs(g) + cfg.eps)) @ P.T)
+    assert np.abs(o.W[0][0] - (W0[0] - 1e-3 * upd)).max() < 1e-12
