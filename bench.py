@@ -66,6 +66,7 @@ def parse_args():
     ap.add_argument("--inner-steps", type=int, default=0, help="override H (non-standard; recorded in config)")
     ap.add_argument("--layers", type=int, default=0, help="keep only the first N decoder layers (profiling; recorded in config)")
     ap.add_argument("--matrices", type=int, default=0, help="keep only the first N matrices (profiling / memory; recorded in config)")
+    ap.add_argument("--right-side", action="store_true", help="project the matrices with more rows than columns from the right (not in the paper; recorded in config)")
     ap.add_argument("--oversample", type=int, default=0, help="extra sketch columns of the refresh, Rayleigh-Ritz truncation (non-standard; recorded in config)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -74,15 +75,19 @@ def parse_args():
     return ap.parse_args()
 
 
-def workload(name: str, H: int = 0, layers: int = 0, matrices: int = 0):
+def workload(name: str, H: int = 0, layers: int = 0, matrices: int = 0, right_side: bool = False):
     from paper_2602_04396_b200 import synth
     wl = synth.config(int(name[3:]))
+    if right_side:
+        wl = synth.scaled(wl, sides=tuple(1 if m > n else 0 for m, n, _ in wl.mats), name=f"{wl.name}_tall_from_right")
     if H > 0:
         wl = synth.scaled(wl, H=H)
     if layers > 0 and len(wl.mats) >= 7 * layers:
-        wl = synth.scaled(wl, mats=wl.mats[:7 * layers], name=f"{wl.name}_first{layers}layers")
+        wl = synth.scaled(wl, mats=wl.mats[:7 * layers], name=f"{wl.name}_first{layers}layers",
+                          sides=wl.sides[:7 * layers] if wl.sides else None)
     if 0 < matrices < len(wl.mats):
-        wl = synth.scaled(wl, mats=wl.mats[:matrices], name=f"{wl.name}_first{matrices}matrices")
+        wl = synth.scaled(wl, mats=wl.mats[:matrices], name=f"{wl.name}_first{matrices}matrices",
+                          sides=wl.sides[:matrices] if wl.sides else None)
     return wl
 
 
@@ -99,20 +104,21 @@ def algorithmic_bytes(wl, variant: int, form: int, ef: bool = True, fast: bool =
     K = wl.K
     bw, bg, be = bytes_of(wl.w_dtype), bytes_of(wl.g_dtype), bytes_of(wl.e_dtype)
     out = dict(clip=0, project=0, moments=0, apply=0, outer_states=0, outer_weights=0)
-    for m, n, r in wl.mats:
-        mn, rn = m * n, r * n
+    for i, (m, n, r) in enumerate(wl.mats):
+        pm, ln = (n, m) if (wl.sides and wl.sides[i]) else (m, n)  # rows of P, columns of the low-rank arrays
+        mn, rn = m * n, r * ln
         p_copies = K if variant == 1 else 1
-        dcol = K * n * 4 if form == 2 else 0
+        dcol = K * ln * 4 if form == 2 else 0
         out["clip"] += K * mn * bg
         stream_in = K * mn * (bg + (be if ef else 0))
         stream_rw = K * mn * (bg + (2 * be if ef else 0) + 2 * bw)
         if fast:
-            out["project"] += stream_in + p_copies * m * r * 2 + K * rn * (16 + 4) + dcol
-            out["apply"] += stream_rw + p_copies * m * r * 2 + K * rn * 4 + dcol
+            out["project"] += stream_in + p_copies * pm * r * 2 + K * rn * (16 + 4) + dcol
+            out["apply"] += stream_rw + p_copies * pm * r * 2 + K * rn * 4 + dcol
         else:
-            out["project"] += stream_in + p_copies * m * r * 4 + K * rn * 4
+            out["project"] += stream_in + p_copies * pm * r * 4 + K * rn * 4
             out["moments"] += K * rn * 4 * 6 + dcol  # read g,u,v; write u,v,U~
-            out["apply"] += stream_rw + p_copies * m * r * 4 + K * rn * 4 * 2 + dcol
+            out["apply"] += stream_rw + p_copies * pm * r * 4 + K * rn * 4 * 2 + dcol
         out["outer_states"] += 2 * (2 * K * rn * 4)
         out["outer_weights"] += 2 * K * mn * bw + mn * 4 * 5  # X0 r/w, B r/w, Delta w
     return out
@@ -188,7 +194,8 @@ def oracle_sample(wl, variant_name: str, K: int = 0, H: int = 6):
     mat = max(shapes, key=lambda s: (shapes[s], -s[0] * s[1]))
     H = min(wl.H, H)
     Ks = min(wl.K, K) if K > 0 else wl.K
-    sample = synth.scaled(wl, mats=[mat], H=H, rounds=1, K=Ks)
+    side = (wl.sides[wl.mats.index(mat)],) if wl.sides else None
+    sample = synth.scaled(wl, mats=[mat], H=H, rounds=1, K=Ks, sides=side)
     desc = (f"1 matrix {mat[0]}x{mat[1]} r{mat[2]} of {len(wl.mats)}, {'all ' if Ks == wl.K else ''}K={Ks} replicas"
             f"{'' if Ks == wl.K else f' of {wl.K}'}, one round of {H} inner steps + outer step + refresh, {variant_name} rule")
     return sample, desc
@@ -204,7 +211,7 @@ def run_oracle_sample(sample, variant_name: str, seed: int = 0):
                           beta2=float(np.float32(0.999)), eps=float(np.float32(1e-8)), clip_rho=sample.clip_rho,
                           outer=lo.OUTER_NESTEROV, outer_lr=float(np.float32(0.8)), outer_momentum=float(np.float32(0.9)),
                           power_iters=sample.power_iters, seed=seed, w_dtype=sample.w_dtype, e_dtype=sample.e_dtype,
-                          state_dtype="f32")
+                          state_dtype="f32", sides=sample.sides)
     orc = lo.LordoOracle(cfg, synth.init_weights(sample, seed))
     grads = [synth.gradients(sample, seed, 0, h) for h in range(sample.H)]
     t0 = time.perf_counter()
@@ -245,7 +252,7 @@ def reference_main(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
+    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices, args.right_side)
     # one step = one pass of the oracle over the sample; the sample shrinks with the number of passes asked
     # for, so that the whole run stays within a few minutes
     sample, desc = oracle_sample(wl, args.variant, H=6 if args.steps + args.warmup <= 8 else 2)
@@ -290,7 +297,8 @@ def run_leg(wl, variant_name: str, mode: str, steps: int, warmup: int, *, dev, r
     opt = lordo.Lordo(wl.mats, wl.K, H, W0, device=str(dev), g_dtype=synth.torch_dtype(wl.g_dtype),
                       e_dtype=synth.torch_dtype(wl.e_dtype), variant=hp["variant"], error_feedback=True, beta2=0.999,
                       eps=1e-8, clip_rho=wl.clip_rho, outer=lordo.OUTER_NESTEROV, outer_lr=0.8, outer_momentum=0.9,
-                      power_iters=wl.power_iters, seed=seed, check_mode=1 if mode == "check" else 0, oversample=oversample)
+                      power_iters=wl.power_iters, seed=seed, check_mode=1 if mode == "check" else 0, oversample=oversample,
+                      sides=wl.sides)
     del W0
     # two gradient sets (round-level signal + per-replica noise), used alternately
     pool = [synth.gradients_device(wl, seed, 0, s, device=str(dev)) for s in range(2)]
@@ -409,7 +417,8 @@ def run_leg(wl, variant_name: str, mode: str, steps: int, warmup: int, *, dev, r
                    "step": "one round = H inner steps + outer step + subspace refresh",
                    "l2": "inputs larger than L2 (no flush)" if wl.weight_replicas * 2 > 4e8 else "inputs fit L2",
                    "parallelism": "replicas only" if world > 1 else "1 gpu",
-                   **({"oversample": oversample} if oversample else {})},
+                   **({"oversample": oversample} if oversample else {}),
+                   **({"sides": "matrices with m > n projected from the right"} if wl.sides and any(wl.sides) else {})},
         "clocks": sampler.summary(t_wall0, t_wall1),
         "gpu_launches": launches,
         "inner_step": {"ms": inner_ms, "params_per_s": wl.weight_replicas / (inner_ms * 1e-3) if inner_ms else None,
@@ -436,6 +445,7 @@ def run_leg(wl, variant_name: str, mode: str, steps: int, warmup: int, *, dev, r
 # same run: (workload, variant, matrices kept (0 = all), warm-up rounds, timed rounds).
 EXTRA_LEGS = [
     ("cfg4", "local", 0, 3, 3),
+    ("cfg4:right", "global", 0, 3, 3),  # the down projections (m > n) projected from the right
     ("cfg3", "global", 0, 3, 10),
     ("cfg3", "local", 0, 3, 10),
     ("cfg5", "local", 8, 3, 10),   # the first 8 of 32 matrices: all 32 with K = 16 do not fit beside their inputs
@@ -468,17 +478,17 @@ def main():
         pass
     where = dict(dev=dev, rank=rank, world=world, local_rank=local_rank, peaks=peaks)
 
-    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices)
+    wl = workload(args.workload, args.inner_steps, args.layers, args.matrices, args.right_side)
     main_leg = run_leg(wl, args.variant, args.mode, args.steps, args.warmup, oversample=args.oversample,
                        e2e_steps=0 if args.no_e2e else args.e2e_steps, **where)
 
     # ---- the other configurations, briefly (one GPU, default workload only) ----------------------
     legs = []
     default_run = (args.workload == "cfg4" and args.variant == "global" and args.mode == "fast" and not args.inner_steps and
-                   not args.layers and not args.matrices and not args.oversample)
+                   not args.layers and not args.matrices and not args.oversample and not args.right_side)
     if world == 1 and default_run and not args.no_legs:
         for name, variant, matrices, wu, st in EXTRA_LEGS:
-            lw = workload(name, 0, 0, matrices)
+            lw = workload(name.split(":")[0], 0, 0, matrices, right_side=name.endswith(":right"))
             leg = run_leg(lw, variant, "fast", st, wu, **where)
             for drop in ("e2e", "memory"):
                 leg.pop(drop, None)

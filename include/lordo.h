@@ -25,7 +25,8 @@
  *     lordo_inner_step_host, lordo_profile_read and lordo_destroy. (A call that is handed new
  *     gradient pointers stages their table in one of two pinned slots and may wait for the copy
  *     that left that slot two changes ago, which has normally long finished.)
- *   - Shapes: n and r multiples of 8, 8 <= r <= min(m, n), K >= 1, H >= 1.
+ *   - Shapes: n and r multiples of 8 (m too for a matrix projected from the right), 8 <= r <= min(m, n),
+ *     K >= 1, H >= 1.
  *   - Errors are return codes (lordo_status); nothing throws or aborts. After a non-zero return
  *     from an argument check no device state was modified. Numerical trouble found on the device
  *     (non-finite gradient norm, breakdown of the QR) sets a sticky flag word that
@@ -77,7 +78,13 @@ typedef enum { LORDO_OUTER_AVG = 0, LORDO_OUTER_NESTEROV = 1 } lordo_outer;     
 typedef struct {
   int64_t m, n; /* W is m x n */
   int32_t r;    /* P is m x r; moments are r x n (projection from the left, Sec. 2) */
-  int32_t reserved;
+  int32_t side; /* 0: as in the paper, from the left. 1: from the right (not in the paper, which always projects
+                   from the left; the side selection of GaLore-type methods for matrices with m > n): P is n x r,
+                   g = (G^ + E) P, the update is U~ P^T, mu(.) of the full-rank QHM term gives one value per row,
+                   ComputeProjection returns the top-r right singular subspace. It is the left-side method applied
+                   to W^T, and the library keeps that view: the moments u, v of such a matrix are [K][r][m]
+                   (transposed low-rank arrays), P is [n][r] / [K][n][r]. Needs m a multiple of 8; not available
+                   together with time_buffer or oversample. */
 } lordo_mat;
 
 typedef struct {
@@ -123,9 +130,9 @@ typedef struct {
 typedef struct {
   void* const* W;      /* [K][m][n] in w_dtype; on entry to lordo_init replica 0 holds W_0 */
   void* const* E;      /* [K][m][n] in e_dtype; may be NULL when error_feedback == 0 */
-  float* const* P;     /* [m][r] (Global) or [K][m][r] (Local) */
-  float* const* u;     /* [K][r][n] first moment */
-  float* const* v;     /* [K][r][n] second moment */
+  float* const* P;     /* [m][r] (Global) or [K][m][r] (Local); side 1: [n][r] / [K][n][r] */
+  float* const* u;     /* [K][r][n] first moment; side 1: [K][r][m] */
+  float* const* v;     /* [K][r][n] second moment; side 1: [K][r][m] */
   float* const* X0;    /* [m][n] model copy of the last synchronisation */
   float* const* B;     /* [m][n] outer momentum; may be NULL when outer == LORDO_OUTER_AVG */
   float* const* Delta; /* [m][n] aggregated pseudo-gradient of the last lordo_outer_step */

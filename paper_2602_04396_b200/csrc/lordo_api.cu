@@ -99,6 +99,12 @@ struct lordo_ctx {
   // tensor-core path of the inner step (check_mode == 0 and every r <= 256)
   bool tc = false;
   TcProblem* d_tc_probs = nullptr;
+  // the update kernel runs once per side present: its table lists the problems stored as they are
+  // projected first, then the ones stored transposed (matrices projected from the right)
+  TcProblem* d_tc_apply = nullptr;
+  std::vector<TcProblem> h_tc_apply;
+  int tc_n_left = 0;
+  long long tc_strips_left = 0;
   TcPrep* d_tc_prep = nullptr;
   long long* d_prep_start = nullptr;
   char* d_tc_bf16 = nullptr;  // all bf16 operand copies, zeroed once by lordo_init
@@ -132,7 +138,7 @@ struct lordo_ctx {
     __nv_bfloat16 *x16 = nullptr, *rinv16 = nullptr, *phl = nullptr, *rt16 = nullptr, *sq16 = nullptr, *uh16 = nullptr, *wr16 = nullptr;
   };
   std::vector<SketchBufs> h_skbufs;  // per matrix: bf16 right-hand sides of the sketch products (refresh scratch)
-  PlanStep inner_proj, inner_apply;
+  std::vector<PlanStep> inner_proj, inner_apply;  // one launch per side present
   std::vector<PlanStep> refresh_steps, init_steps;
   std::vector<PlanStep> tb_steps;  // Delta rebuilt from the time buffers (lordo_outer_step with time_buffer)
 
@@ -220,6 +226,9 @@ int validate_config(const lordo_config* cfg, std::string& why) {
     const lordo_mat& a = cfg->mats[i];
     if (a.m < 1 || a.n < 1 || a.r < 1) { why = "non-positive shape"; return LORDO_ERR_SHAPE; }
     if (a.n % 8 != 0 || a.r % 8 != 0) { why = "n and r must be multiples of 8"; return LORDO_ERR_ALIGN; }
+    if (a.side != 0 && a.side != 1) { why = "side must be 0 (left) or 1 (right)"; return LORDO_ERR_INVALID_ARG; }
+    if (a.side == 1 && a.m % 8 != 0) { why = "m must be a multiple of 8 for a matrix projected from the right"; return LORDO_ERR_ALIGN; }
+    if (a.side == 1 && (cfg->time_buffer || cfg->oversample > 0)) { why = "projection from the right is not available with time_buffer or oversample"; return LORDO_ERR_UNSUPPORTED; }
     if (a.r > a.m || a.r > a.n) { why = "r must not exceed min(m, n)"; return LORDO_ERR_SHAPE; }
     if (cfg->oversample > 0 && (a.r + cfg->oversample > a.m || a.r + cfg->oversample > a.n || a.r + cfg->oversample > 600)) {
       why = "r + oversample must not exceed min(m, n) nor 600";
@@ -245,9 +254,10 @@ void prefix_arrays(const lordo_config& cfg, std::vector<long long>& chunk_start,
     const lordo_mat& a = cfg.mats[i];
     const long long elems = a.m * a.n;
     chunk_start[i + 1] = chunk_start[i] + (long long)K * ((elems + kSqChunk - 1) / kSqChunk);
-    mom_start[i + 1] = mom_start[i] + (long long)K * ((a.n + 127) / 128);
+    const long long ln = a.side ? a.m : a.n;  // columns of the low-rank arrays
+    mom_start[i + 1] = mom_start[i] + (long long)K * ((ln + 127) / 128);
     wblk[i + 1] = wblk[i] + (elems + 1023) / 1024;
-    sblk[i + 1] = sblk[i] + ((long long)a.r * a.n + 1023) / 1024;
+    sblk[i + 1] = sblk[i] + ((long long)a.r * ln + 1023) / 1024;
   }
 }
 
@@ -285,19 +295,19 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     for (int i = 0; i < n_mats; ++i) {
       const lordo_mat& a = cfg.mats[i];
       const long long maxd = a.m > a.n ? a.m : a.n;
+      const size_t pm = a.side ? a.n : a.m, ln = a.side ? a.m : a.n;  // rows of P, columns of the low-rank arrays
       const size_t nb = local ? K : 1;
       const size_t rs = (size_t)a.r + cfg.oversample;  // columns of the sketch and of everything up to the truncation
-      size_t per = (size_t)a.n * rs + 2 * (size_t)a.m * rs + (size_t)maxd * rs + ((q > 0 || cfg.oversample > 0) ? 2 * (size_t)a.n * rs : 0) +
-                   4 * rs * rs;
+      size_t per = ln * rs + 2 * pm * rs + (size_t)maxd * rs + ((q > 0 || cfg.oversample > 0) ? 2 * ln * rs : 0) + 4 * rs * rs;
       if (cfg.oversample > 0) per += 3 * rs * rs + rs * a.r;  // eigen-solver work and the truncating projector
       // bf16 right-hand sides of the tensor-core sketch products (Omega, P', Z), counted in floats
-      per += ((size_t)a.n * a.r + (q > 0 ? (size_t)a.m * a.r + (size_t)a.n * a.r : 0)) / 2 + 64;
+      per += (ln * a.r + (q > 0 ? pm * a.r + ln * a.r : 0)) / 2 + 64;
       size_t states16 = 0;
       if (cfg.check_mode == 0 && cfg.w_dtype == LORDO_BF16) {
         // bf16 planes of the tensor-core QR and rotation: X and R^-1 in three planes, P, Rot^T, its square
         // (per batch entry) and the two moment operands of every worker in two
-        per += 3 * (size_t)maxd * a.r / 2 + (size_t)a.m * a.r + 7 * (size_t)a.r * a.r / 2 + 128;
-        states16 = 2 * (size_t)K * a.r * a.n + 64;
+        per += 3 * (size_t)maxd * a.r / 2 + pm * a.r + 7 * (size_t)a.r * a.r / 2 + 128;
+        states16 = 2 * (size_t)K * a.r * ln + 64;
       }
       mat_scratch[i] = nb * per + states16;
       if (acc > 0 && acc + mat_scratch[i] > kRefreshScratchFloats) { ++grp; acc = 0; }
@@ -316,12 +326,13 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   for (int i = 0; i < n_mats; ++i) {
     const lordo_mat& a = cfg.mats[i];
     MatDev& md = c->h_mats[i];
-    md.m = a.m; md.n = a.n; md.r = a.r; md.pad = 0; md.Delta16 = nullptr;
-    md.ghat = cv.take<float>((size_t)K * a.r * a.n);
-    md.util = cv.take<float>((size_t)K * a.r * a.n);
-    md.dcol = cv.take<float>((size_t)K * a.n);
-    md.T = cfg.time_buffer ? cv.take<float>((size_t)K * a.r * a.n) : nullptr;
-    md.p_stride = local ? a.m * a.r : 0;
+    md.m = a.m; md.n = a.n; md.r = a.r; md.side = a.side; md.Delta16 = nullptr;
+    md.pm = a.side ? a.n : a.m; md.ln = a.side ? a.m : a.n;
+    md.ghat = cv.take<float>((size_t)K * a.r * md.ln);
+    md.util = cv.take<float>((size_t)K * a.r * md.ln);
+    md.dcol = cv.take<float>((size_t)K * md.ln);
+    md.T = cfg.time_buffer ? cv.take<float>((size_t)K * a.r * md.ln) : nullptr;
+    md.p_stride = local ? md.pm * a.r : 0;
     if (real) {
       md.W = buf->W[i]; md.E = buf->E ? buf->E[i] : nullptr; md.P = buf->P[i]; md.u = buf->u[i]; md.v = buf->v[i];
       md.X0 = buf->X0[i]; md.B = buf->B ? buf->B[i] : nullptr; md.Delta = buf->Delta[i];
@@ -332,7 +343,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   // ---------------- tensor-core operand copies and problem table ----------------
   c->tc = cfg.check_mode == 0 && cfg.g_dtype == cfg.w_dtype && (!cfg.error_feedback || cfg.e_dtype == cfg.w_dtype);
   for (int i = 0; i < n_mats; ++i)  // ranks above 512 (above 256 with fp32 storage) run on the fp32 path
-    if (cfg.mats[i].r > (cfg.w_dtype == LORDO_BF16 ? 512 : 256)) c->tc = false;
+    if (cfg.mats[i].r > (cfg.w_dtype == LORDO_BF16 ? 512 : 256) || (cfg.mats[i].side && cfg.w_dtype != LORDO_BF16)) c->tc = false;
   c->h_tc.clear(); c->h_prep.clear(); c->h_prep_start.assign(1, 0);
   c->tc_strips = 0; c->tc_strips_p = 0; c->tc_rn_max = 0; c->tc_rk_max = 0;
   if (c->tc) {
@@ -341,37 +352,37 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
     const size_t bf16_begin = cv.off;
     for (int i = 0; i < n_mats; ++i) {
       const MatDev& md = c->h_mats[i];
-      const int r_k = (int)up(md.r, 64), r_n = (int)up(md.r, 16), m_k = (int)up(md.m, 64);
+      const int r_k = (int)up(md.r, 64), r_n = (int)up(md.r, 16), m_k = (int)up(md.pm, 64);
       const int copies = local ? K : 1;
       __nv_bfloat16* P16 = cv.take<__nv_bfloat16>((size_t)copies * m_k * r_k);
       __nv_bfloat16* PT16 = cv.take<__nv_bfloat16>((size_t)copies * r_n * m_k);
-      const size_t n_pad = (size_t)up(md.n, 128);  // whole strips: the TMA-fed kernels store these per strip
+      const size_t n_pad = (size_t)up(md.ln, 128);  // whole strips: the TMA-fed kernels store these per strip
       __nv_bfloat16* gT16 = cv.take<__nv_bfloat16>((size_t)K * n_pad * r_k);
       __nv_bfloat16* uT16 = cv.take<__nv_bfloat16>((size_t)K * n_pad * r_k);
       const int nsplit = (cfg.w_dtype == LORDO_BF16 && r_n > 256) ? 2 : 1;  // TMA-fed projection: one strip per half of the rank
-      float* dcol2 = nsplit == 2 ? cv.take<float>((size_t)K * md.n) : nullptr;
+      float* dcol2 = nsplit == 2 ? cv.take<float>((size_t)K * md.ln) : nullptr;
       if (r_n > c->tc_rn_max) c->tc_rn_max = r_n;
       if (r_k > c->tc_rk_max) c->tc_rk_max = r_k;
       for (int k = 0; k < copies; ++k) {
         TcPrep pp;
         std::memset(&pp, 0, sizeof(pp));
-        pp.P = md.P ? md.P + (long long)k * md.m * md.r : nullptr;
+        pp.P = md.P ? md.P + (long long)k * md.pm * md.r : nullptr;
         pp.P16 = P16 + (size_t)k * m_k * r_k; pp.PT16 = PT16 + (size_t)k * r_n * m_k;
-        pp.m = md.m; pp.r = md.r; pp.r_k = r_k; pp.m_k = m_k;
+        pp.m = md.pm; pp.r = md.r; pp.r_k = r_k; pp.m_k = m_k;
         c->h_prep.push_back(pp);
-        c->h_prep_start.push_back(c->h_prep_start.back() + ((md.m + 63) / 64) * ((md.r + 63) / 64));  // 64 x 64 tiles
+        c->h_prep_start.push_back(c->h_prep_start.back() + ((md.pm + 63) / 64) * ((md.r + 63) / 64));  // 64 x 64 tiles
       }
       for (int k = 0; k < K; ++k) {
-        const long long wo = (long long)k * md.m * md.n, so = (long long)k * md.r * md.n;
+        const long long wo = (long long)k * md.m * md.n, so = (long long)k * md.r * md.ln;
         const int pk = local ? k : 0;
         TcProblem tp;
         std::memset(&tp, 0, sizeof(tp));
         tp.strip_start = c->tc_strips;
-        tp.m = (int)md.m; tp.n = (int)md.n; tp.r = md.r; tp.r_k = r_k; tp.r_n = r_n; tp.m_k = m_k;
+        tp.m = (int)md.pm; tp.n = (int)md.ln; tp.tr = md.side; tp.r = md.r; tp.r_k = r_k; tp.r_n = r_n; tp.m_k = m_k;
         tp.PT16 = PT16 + (size_t)pk * r_n * m_k; tp.P16 = P16 + (size_t)pk * m_k * r_k;
         tp.gT16 = gT16 + (size_t)k * n_pad * r_k; tp.uT16 = uT16 + (size_t)k * n_pad * r_k;
         tp.u = md.u ? md.u + so : nullptr; tp.v = md.v ? md.v + so : nullptr;
-        tp.dcol = md.dcol + (long long)k * md.n;
+        tp.dcol = md.dcol + (long long)k * md.ln;
         tp.tb = md.T ? md.T + so : nullptr;
         if (real) {
           tp.W = cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
@@ -380,16 +391,32 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         tp.G_ind = c->d_Gtab + i; tp.G_off = wo;
         tp.cptr = c->d_coef + (size_t)i * K + k;
         tp.mat = i; tp.replica = k; tp.pcopy = pk;
-        tp.strip_start_p = c->tc_strips_p; tp.nsplit = nsplit; tp.dcol2 = dcol2 ? dcol2 + (long long)k * md.n : nullptr;
+        tp.strip_start_p = c->tc_strips_p; tp.nsplit = nsplit; tp.dcol2 = dcol2 ? dcol2 + (long long)k * md.ln : nullptr;
         c->h_tc.push_back(tp);
-        c->tc_strips += (md.n + 127) / 128;
-        c->tc_strips_p += (long long)nsplit * ((md.n + 127) / 128);
+        c->tc_strips += (md.ln + 127) / 128;
+        c->tc_strips_p += (long long)nsplit * ((md.ln + 127) / 128);
       }
     }
     c->d_tc_bf16 = ws ? reinterpret_cast<char*>(ws) + bf16_begin : nullptr;
     c->tc_bf16_bytes = cv.off - bf16_begin;
     c->prep_blocks = c->h_prep_start.back();
     c->d_tc_probs = cv.take<TcProblem>(c->h_tc.size());
+    c->d_tc_apply = cv.take<TcProblem>(c->h_tc.size());
+    c->h_tc_apply.clear();
+    c->tc_n_left = 0; c->tc_strips_left = 0;
+    {
+      long long strips = 0;
+      for (int side = 0; side < 2; ++side) {
+        for (const TcProblem& tp : c->h_tc) {
+          if (tp.tr != side) continue;
+          TcProblem q2 = tp;
+          q2.strip_start = strips;
+          strips += (tp.n + 127) / 128;
+          c->h_tc_apply.push_back(q2);
+        }
+        if (side == 0) { c->tc_n_left = (int)c->h_tc_apply.size(); c->tc_strips_left = strips; }
+      }
+    }
     c->d_tc_prep = cv.take<TcPrep>(c->h_prep.size());
     c->d_prep_start = cv.take<long long>(c->h_prep_start.size());
     c->tma = cfg.w_dtype == LORDO_BF16;
@@ -463,39 +490,48 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   };
 
   // inner step: g = P^T (c G + E)   and   E' = A - P g ; W' = W - lr (...)
-  {
+  c->inner_proj.clear();
+  c->inner_apply.clear();
+  for (int side = 0; side < 2; ++side) {
     SlotBuilder sb;
     for (int i = 0; i < n_mats; ++i) {
       const MatDev& md = c->h_mats[i];
+      if (md.side != side) continue;
       for (int k = 0; k < K; ++k) {
         sb.rewind();
-        const long long wo = (long long)k * md.m * md.n;
-        Operand A = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
-        Operand B = plain(nullptr, md.n, cfg.g_dtype);
-        B.p0_ind = c->d_Gtab + i; B.p0_off = wo;
-        B.s0_ptr = c->d_coef + (size_t)i * K + k;
+        const long long wo = (long long)k * md.m * md.n, so = (long long)k * md.r * md.ln;
+        Operand Pk = plain(md.P ? md.P + k * md.p_stride : nullptr, md.r);
+        Operand S = plain(nullptr, md.n, cfg.g_dtype);  // c G + E, stored [m][n]
+        S.p0_ind = c->d_Gtab + i; S.p0_off = wo;
+        S.s0_ptr = c->d_coef + (size_t)i * K + k;
         if (cfg.error_feedback && real) {
-          B.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + wo) : (const void*)((const unsigned short*)md.E + wo);
-          B.dt1 = cfg.e_dtype;
+          S.p1 = cfg.e_dtype == LORDO_F32 ? (const void*)((const float*)md.E + wo) : (const void*)((const unsigned short*)md.E + wo);
+          S.dt1 = cfg.e_dtype;
         }
-        sb.next(ST_GEMM, 0, 1, 0, 0).g.push_back(gemm_prob(md.r, (int)md.n, (int)md.m, A, B, nullptr, store_epi(md.ghat + (long long)k * md.r * md.n, md.n)));
-        Operand B1 = plain(md.ghat + (long long)k * md.r * md.n, md.n);
-        Operand B2 = plain(md.util + (long long)k * md.r * md.n, md.n);
+        if (!side) {  // g [r][n] = P^T (c G + E)
+          sb.next(ST_GEMM, 0, 1, 0, 0).g.push_back(gemm_prob(md.r, (int)md.n, (int)md.m, Pk, S, nullptr, store_epi(md.ghat + so, md.n)));
+        } else {      // (c G + E) P is [m][r]; kept as its transpose [r][m]
+          Epilogue et = store_epi(md.ghat + so, md.m);
+          et.trans = 1;
+          sb.next(ST_GEMM, 0, 0, 0, 0).g.push_back(gemm_prob((int)md.m, md.r, (int)md.n, S, Pk, nullptr, et));
+        }
+        Operand B1 = plain(md.ghat + so, md.ln);
+        Operand B2 = plain(md.util + so, md.ln);
         Epilogue e;
         std::memset(&e, 0, sizeof(e));
         e.kind = EPI_APPLY;
         e.W = !real ? nullptr : cfg.w_dtype == LORDO_F32 ? (void*)((float*)md.W + wo) : (void*)((unsigned short*)md.W + wo);
         e.E = md.E ? (cfg.e_dtype == LORDO_F32 ? (void*)((float*)md.E + wo) : (void*)((unsigned short*)md.E + wo)) : nullptr;
         e.G_ind = c->d_Gtab + i; e.G_off = wo;
-        e.dcol = md.dcol + (long long)k * md.n;
+        e.dcol = md.dcol + (long long)k * md.ln;
         e.cptr = c->d_coef + (size_t)i * K + k;
-        sb.next(ST_GEMM, 0, 0, 1, 0).g.push_back(gemm_prob((int)md.m, (int)md.n, md.r, A, B1, &B2, e));
+        e.trans = side; e.ldt = md.n;  // side 1: the product P g' is [n][m], element (row, col) is W[col][row]
+        sb.next(ST_GEMM, 0, 0, 1, 0).g.push_back(gemm_prob((int)md.pm, (int)md.ln, md.r, Pk, B1, &B2, e));
       }
     }
     std::vector<PlanStep> two;
     flatten(sb, two);
-    c->inner_proj = two[0];
-    c->inner_apply = two[1];
+    if (two.size() == 2) { c->inner_proj.push_back(two[0]); c->inner_apply.push_back(two[1]); }
   }
 
   // CholeskyQR2 of X (rows x r, batch of nb with stride sx) into O, through T.
@@ -529,13 +565,18 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   c->init_steps.clear();
   const int n_groups = n_mats ? group_of[n_mats - 1] + 1 : 0;
   for (int grp = 0; grp < n_groups; ++grp) {
-    SlotBuilder R, I;
+    // one sequence of launches per side: a launch has one operand-major setting for all its problems
+    SlotBuilder Rs[2], Is[2];
     size_t goff = 0;
     for (int i = 0; i < n_mats; ++i) {
       if (group_of[i] != grp) continue;
-      R.rewind(); I.rewind();
       const MatDev& md = c->h_mats[i];
-      const long long m = md.m, n = md.n;
+      SlotBuilder &R = Rs[md.side], &I = Is[md.side];
+      R.rewind(); I.rewind();
+      // the problem as the refresh sees it: P is m x r, the low-rank arrays have n columns, the signal is
+      // m x n. For a matrix projected from the right that is the transpose of what is stored (sd = 1).
+      const long long m = md.pm, n = md.ln;
+      const int sd = md.side;
       const int r = md.r;
       const int nb = local ? K : 1;
       const long long maxd = m > n ? m : n;
@@ -643,14 +684,15 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SkProblem sp;
           std::memset(&sp, 0, sizeof(sp));
           sp.M = (int)Mo; sp.Kd = (int)Kd; sp.r = r; sp.r_n = (r + 15) / 16 * 16;
-          sp.a_mn = a_mn; sp.a_c2 = local ? b : 0; sp.b_c2 = b;
+          const int st_mn = a_mn ^ sd;  // how the stored signal lies with respect to this product
+          sp.a_mn = st_mn; sp.a_c2 = local ? b : 0; sp.b_c2 = b;
           TmaMatMaps* mm = c->d_maps + i;
           TmaGradMaps* gm = c->d_gmaps + i;
           if (local) {
-            sp.map_a = a_mn ? gm->g_sw : gm->g_kb;
-            if (cfg.error_feedback) { sp.map_e = a_mn ? mm->e_sw : mm->e_kb; sp.cptr = c->d_coef + (size_t)i * K + b; }
+            sp.map_a = st_mn ? gm->g_sw : gm->g_kb;
+            if (cfg.error_feedback) { sp.map_e = st_mn ? mm->e_sw : mm->e_kb; sp.cptr = c->d_coef + (size_t)i * K + b; }
           } else {
-            sp.map_a = a_mn ? mm->d_sw : mm->d_kb;
+            sp.map_a = st_mn ? mm->d_sw : mm->d_kb;
           }
           sp.map_b = map_b;
           sp.C = C + (long long)b * cstride; sp.ldc = r;
@@ -664,9 +706,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         sb.next(ST_CONVERT, PH_SUBSPACE).cv.push_back(cp);
       };
 
-      auto signal = [&](int b) {  // S of problem b: Delta (Global) or c_k G_k + E_k (Local), stored [m][n]
-        if (!local) return plain(md.Delta, n);
-        Operand A = plain(nullptr, n, cfg.g_dtype);
+      auto signal = [&](int b) {  // S of problem b: Delta (Global) or c_k G_k + E_k (Local), as stored: [md.m][md.n]
+        if (!local) return plain(md.Delta, md.n);
+        Operand A = plain(nullptr, md.n, cfg.g_dtype);
         A.p0_ind = c->d_Gtab + i; A.p0_off = (long long)b * m * n;
         A.s0_ptr = c->d_coef + (size_t)i * K + b;
         if (cfg.error_feedback && real) {
@@ -694,7 +736,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           if (!local) convert(R, md.Delta, md.Delta16, (size_t)m * n);  // bf16 copy of the Global signal
           sketch(R, 0, (c->d_maps + i)->om16, Ya, m * r, m, n);
         } else {
-          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, sd, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, rs, (int)n, signal(b), plain(Om + (long long)b * n * rs, rs), nullptr, store_epi(Ya + (long long)b * m * rs, rs)));
         }
         qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs);
@@ -704,7 +746,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           convert(R, Pn, pn16, (size_t)nb * m * r);
           sketch(R, 1, (c->d_maps + i)->pn16, Za, n * r, n, m);
         } else {
-          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1, 0, 0);
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1 - sd, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, rs, (int)m, signal(b), plain(Pn + (long long)b * m * rs, rs), nullptr, store_epi(Za + (long long)b * n * rs, rs)));
         }
         qr2(R, PH_SUBSPACE, Za, n * rs, Yb, maxd * rs, Zq, n * rs, n, rs);
@@ -712,7 +754,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           convert(R, Zq, zq16, (size_t)nb * n * r);
           sketch(R, 0, (c->d_maps + i)->zq16, Ya, m * r, m, n);
         } else {
-          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 0, 0, 0);
+          SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, sd, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, rs, (int)n, signal(b), plain(Zq + (long long)b * n * rs, rs), nullptr, store_epi(Ya + (long long)b * m * rs, rs)));
         }
         qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs);
@@ -815,8 +857,10 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         cholqr2(I, PH_SUBSPACE, Ya, m * r, Yb, maxd * r, md.P, m * r, m, r, 1, gram, lw, rinv);
       }
     }
-    flatten(R, c->refresh_steps);
-    flatten(I, c->init_steps);
+    for (int sd = 0; sd < 2; ++sd) {
+      flatten(Rs[sd], c->refresh_steps);
+      flatten(Is[sd], c->init_steps);
+    }
   }
   // Up-link time buffer: Delta = P T_mean (Global, after the buffers were averaged) or the sum over
   // the workers of P_k T_k (Local; the outer kernel divides by K), one grouped GEMM per term.
@@ -1070,6 +1114,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
     if (!c->tma) INIT_CUDA(tc_configure(c->tc_rn_max, c->tc_rk_max));  // register-staged kernels (fp32 storage)
     INIT_CUDA(cudaMemsetAsync(c->d_tc_bf16, 0, c->tc_bf16_bytes, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_tc_probs, c->h_tc.data(), sizeof(TcProblem) * c->h_tc.size(), cudaMemcpyHostToDevice, st));
+    INIT_CUDA(cudaMemcpyAsync(c->d_tc_apply, c->h_tc_apply.data(), sizeof(TcProblem) * c->h_tc_apply.size(), cudaMemcpyHostToDevice, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_tc_prep, c->h_prep.data(), sizeof(TcPrep) * c->h_prep.size(), cudaMemcpyHostToDevice, st));
     INIT_CUDA(cudaMemcpyAsync(c->d_prep_start, c->h_prep_start.data(), 8 * c->h_prep_start.size(), cudaMemcpyHostToDevice, st));
     if (c->tma) {
@@ -1090,6 +1135,11 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
         }
         good = good && encode_map3(hm[i].w_sw, md.W, md.n, md.m, c->K, 64, 64, true);
         good = good && encode_map3(hm[i].w_st, md.W, md.n, md.m, c->K, 64, 16, true);
+        if (md.side) {  // tiles of 128 stored rows x 64 stored columns, handed back 32 rows at a time
+          good = good && encode_map3(hm[i].w_kb, md.W, md.n, md.m, c->K, 64, 128, true);
+          good = good && encode_map3(hm[i].w_st32, md.W, md.n, md.m, c->K, 64, 32, true);
+          if (md.E) good = good && encode_map3(hm[i].e_st32, md.E, md.n, md.m, c->K, 64, 32, true);
+        }
         good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n < 256 ? tp.r_n : 256, true);
         good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
         // refresh: signal as rows (64 k x 128 rows) and right-hand sides [batch][Kd][r]
@@ -1100,20 +1150,20 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
           good = good && encode_map3(hm[i].d_sw, md.Delta16, md.n, md.m, 1, 64, 64, true);
         }
         const lordo_ctx::SketchBufs& sb = c->h_skbufs[i];
-        good = good && encode_map3(hm[i].om16, sb.om16, md.r, md.n, nbatch, 64, 64, true);
-        if (sb.pn16) good = good && encode_map3(hm[i].pn16, sb.pn16, md.r, md.m, nbatch, 64, 64, true);
-        if (sb.zq16) good = good && encode_map3(hm[i].zq16, sb.zq16, md.r, md.n, nbatch, 64, 64, true);
+        good = good && encode_map3(hm[i].om16, sb.om16, md.r, md.ln, nbatch, 64, 64, true);
+        if (sb.pn16) good = good && encode_map3(hm[i].pn16, sb.pn16, md.r, md.pm, nbatch, 64, 64, true);
+        if (sb.zq16) good = good && encode_map3(hm[i].zq16, sb.zq16, md.r, md.ln, nbatch, 64, 64, true);
         if (sb.x16) {  // hi|lo planes of the tensor-core QR and rotation
-          good = good && encode_map3(hm[i].xm_sw, sb.x16, md.r, md.m, 3 * nbatch, 64, 64, true);
-          good = good && encode_map3(hm[i].xm_kb, sb.x16, md.r, md.m, 3 * nbatch, 64, 128, true);
-          good = good && encode_map3(hm[i].xn_sw, sb.x16, md.r, md.n, 3 * nbatch, 64, 64, true);
-          good = good && encode_map3(hm[i].xn_kb, sb.x16, md.r, md.n, 3 * nbatch, 64, 128, true);
+          good = good && encode_map3(hm[i].xm_sw, sb.x16, md.r, md.pm, 3 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].xm_kb, sb.x16, md.r, md.pm, 3 * nbatch, 64, 128, true);
+          good = good && encode_map3(hm[i].xn_sw, sb.x16, md.r, md.ln, 3 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].xn_kb, sb.x16, md.r, md.ln, 3 * nbatch, 64, 128, true);
           good = good && encode_map3(hm[i].rinv_sw, sb.rinv16, md.r, md.r, 3 * nbatch, 64, 64, true);
-          good = good && encode_map3(hm[i].phl_sw, sb.phl, md.r, md.m, 2 * nbatch, 64, 64, true);
+          good = good && encode_map3(hm[i].phl_sw, sb.phl, md.r, md.pm, 2 * nbatch, 64, 64, true);
           good = good && encode_map3(hm[i].rt_sw, sb.rt16, md.r, md.r, 2 * nbatch, 64, 64, true);
           good = good && encode_map3(hm[i].sq_sw, sb.sq16, md.r, md.r, 2 * nbatch, 64, 64, true);
-          good = good && encode_map3(hm[i].uh_sw, sb.uh16, md.n, md.r, 2 * c->K, 64, 64, true);
-          good = good && encode_map3(hm[i].wr_sw, sb.wr16, md.n, md.r, 2 * c->K, 64, 64, true);
+          good = good && encode_map3(hm[i].uh_sw, sb.uh16, md.ln, md.r, 2 * c->K, 64, 64, true);
+          good = good && encode_map3(hm[i].wr_sw, sb.wr16, md.ln, md.r, 2 * c->K, 64, 64, true);
         }
       }
       if (good) {
@@ -1135,7 +1185,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
   c->launches += 2;
   for (int i = 0; i < nm; ++i) {
     const MatDev& md = c->h_mats[i];
-    const size_t wn = (size_t)md.m * md.n, sn = (size_t)c->K * md.r * md.n;
+    const size_t wn = (size_t)md.m * md.n, sn = (size_t)c->K * md.r * md.ln;
     if (md.E) INIT_CUDA(cudaMemsetAsync(md.E, 0, (size_t)c->K * wn * (c->cfg.e_dtype == LORDO_F32 ? 4 : 2), st));
     INIT_CUDA(cudaMemsetAsync(md.u, 0, sn * 4, st));
     INIT_CUDA(cudaMemsetAsync(md.v, 0, sn * 4, st));
@@ -1143,7 +1193,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
     if (md.B) INIT_CUDA(cudaMemsetAsync(md.B, 0, wn * 4, st));
     INIT_CUDA(cudaMemsetAsync(md.Delta, 0, wn * 4, st));
     if (c->cfg.variant == LORDO_LOCAL) {
-      launch_identity_projection(md.P, md.m, md.r, c->K, st);
+      launch_identity_projection(md.P, md.pm, md.r, c->K, st);
       c->launches += 1;
     }
   }
@@ -1204,16 +1254,26 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
       }
       {
         ProfScope ps(c, st, PC_APPLY);
-        if (!big) {
-          launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, 0, c->d_status, st);
-        } else {  // 256 < r <= 512: the error-feedback sweep, then the model-update sweep
-          if (c->cfg.error_feedback) {
-            launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, 1, c->d_status, st);
+        const int n_all = (int)c->h_tc_apply.size();
+        for (int side = 0; side < 2; ++side) {  // problems stored as projected, then the ones stored transposed
+          const TcProblem* pb = c->d_tc_apply + (side ? c->tc_n_left : 0);
+          const int np = side ? n_all - c->tc_n_left : c->tc_n_left;
+          const long long s0 = side ? c->tc_strips_left : 0, s1 = side ? c->tc_strips : c->tc_strips_left;
+          if (np == 0) continue;
+          if (!big) {
+            launch_apply_tma(pb, np, s0, s1, c->d_maps, c->d_gmaps, ss, c->sm_count, 0, side, c->d_status, st);
+            c->launches += 1;
+          } else {  // 256 < r <= 512: the error-feedback sweep, then the model-update sweep
+            if (c->cfg.error_feedback) {
+              launch_apply_tma(pb, np, s0, s1, c->d_maps, c->d_gmaps, ss, c->sm_count, 1, side, c->d_status, st);
+              c->launches += 1;
+            }
+            launch_apply_tma(pb, np, s0, s1, c->d_maps, c->d_gmaps, ss, c->sm_count, 2, side, c->d_status, st);
             c->launches += 1;
           }
-          launch_apply_tma(c->d_tc_probs, (int)c->h_tc.size(), c->tc_strips, c->d_maps, c->d_gmaps, ss, c->sm_count, 2, c->d_status, st);
         }
       }
+      c->launches -= 1;  // the common tail below counts one update launch
     } else {
     {
       ProfScope ps(c, st, PC_PROJECT);  // includes the moment update (fused epilogue)
@@ -1236,7 +1296,10 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
   }
   {
     ProfScope ps(c, st, PC_PROJECT);
-    rc = run_plan_step(c, c->inner_proj, gs, st);
+    for (const PlanStep& s : c->inner_proj) {
+      rc = run_plan_step(c, s, gs, st);
+      if (rc != LORDO_OK) break;
+    }
   }
   if (rc != LORDO_OK) return rc;
   {
@@ -1248,7 +1311,10 @@ int lordo_inner_step(lordo_ctx* c, const void* const* G, float lr, float beta1, 
   if (rc != LORDO_OK) return rc;
   {
     ProfScope ps(c, st, PC_APPLY);
-    rc = run_plan_step(c, c->inner_apply, gs, st);
+    for (const PlanStep& s : c->inner_apply) {
+      rc = run_plan_step(c, s, gs, st);
+      if (rc != LORDO_OK) break;
+    }
   }
   if (rc != LORDO_OK) return rc;
   c->steps = s;
@@ -1304,7 +1370,7 @@ int lordo_outer_step(lordo_ctx* c, void* stream) {
   if (rc != LORDO_OK) return rc;
   if (tb)
     for (int i = 0; i < c->n_mats; ++i)
-      CUDA_OK(c, cudaMemsetAsync(c->h_mats[i].T, 0, sizeof(float) * (size_t)c->K * c->h_mats[i].r * c->h_mats[i].n, st));
+      CUDA_OK(c, cudaMemsetAsync(c->h_mats[i].T, 0, sizeof(float) * (size_t)c->K * c->h_mats[i].r * c->h_mats[i].ln, st));
   c->steps_in_round = 0;
   c->outers += 1;
   c->after_outer = true;

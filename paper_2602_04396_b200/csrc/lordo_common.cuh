@@ -12,23 +12,24 @@ namespace lordo {
 // Per-matrix device record, built once by lordo_init and kept in the workspace.
 // ---------------------------------------------------------------------------------------------
 struct MatDev {
-  long long m, n;
+  long long m, n;     // storage shape of W, G, E, X0, B, Delta
   int r;
-  int pad;
+  int side;           // 1: projected from the right, handled as the left-side problem on the transpose
+  long long pm, ln;   // rows of P and columns of the low-rank arrays: (m, n), or (n, m) for side 1
   void* W;            // [K][m][n] w_dtype
   void* E;            // [K][m][n] e_dtype
-  float* P;           // [m][r] or [K][m][r]
-  float* u;           // [K][r][n]
-  float* v;           // [K][r][n]
+  float* P;           // [pm][r] or [K][pm][r]
+  float* u;           // [K][r][ln]
+  float* v;           // [K][r][ln]
   float* X0;          // [m][n]
   float* B;           // [m][n]
   float* Delta;       // [m][n]
-  float* ghat;        // [K][r][n] low-rank gradient (workspace)
-  float* util;        // [K][r][n] normalised low-rank update U~ (workspace)
-  float* dcol;        // [K][n]    column scale of the full-rank QHM term (workspace)
+  float* ghat;        // [K][r][ln] low-rank gradient (workspace)
+  float* util;        // [K][r][ln] normalised low-rank update U~ (workspace)
+  float* dcol;        // [K][ln]   column scale of the full-rank QHM term (workspace)
   long long p_stride; // elements between the P of consecutive replicas (0 for Global)
   __nv_bfloat16* Delta16;  // [m][n] bf16 copy of Delta, made at the start of a Global refresh for the tensor-core sketch (workspace; may be null)
-  float* T;           // [K][r][n] up-link time buffer: sum over the round of lr * U~ (workspace; null unless enabled)
+  float* T;           // [K][r][ln] up-link time buffer: sum over the round of lr * U~ (workspace; null unless enabled)
 };
 
 // Scalars of one inner step (Algorithm 1, per-step lines).

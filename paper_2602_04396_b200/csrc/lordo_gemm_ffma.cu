@@ -176,7 +176,14 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
   for (int i = 0; i < 4; ++i) {
     const long long row = m0 + ty * 4 + i;
     if (row >= M) break;
-    if (ep.kind == EPI_STORE) {
+    if (ep.kind == EPI_STORE && ep.trans) {  // C[col][row]
+      const float o[4] = {acc[i][0], acc[i][1], acc[i][2], acc[i][3]};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float* cp = ep.C + (col + j) * ep.ldc + row;
+        *cp = ep.pad ? *cp + o[j] : o[j];
+      }
+    } else if (ep.kind == EPI_STORE) {
       float4* cp = reinterpret_cast<float4*>(ep.C + row * ep.ldc + col);
       float4 o = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
       if (ep.pad) {  // accumulate into C
@@ -184,6 +191,22 @@ __global__ void __launch_bounds__(256) gemm_ffma_kernel(const GemmProblem* __res
         o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
       }
       *cp = o;
+    } else if (ep.kind == EPI_APPLY && ep.trans) {
+      // the product was formed for the transposed problem: output (row, col) is weight element (col, row),
+      // and the full-rank QHM scale belongs to the output column = the weight's row
+      if constexpr (DUAL) {
+        const float c = *ep.cptr;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const long long idx = (col + j) * ep.ldt + row;
+          const float g = load1(*ep.G_ind, sc.g_dt, ep.G_off + idx);
+          const float w = load1(ep.W, sc.w_dt, idx);
+          float upd = acc2[i][j];
+          if (sc.form == LORDO_QHM_FULL) upd = (1.f - sc.omega) * (c * g) / ep.dcol[col + j] + sc.omega * upd;
+          if (sc.ef) store1(ep.E, sc.e_dt, idx, (c * g + load1(ep.E, sc.e_dt, idx)) - acc[i][j]);
+          store1(ep.W, sc.w_dt, idx, w - sc.lr * upd);
+        }
+      }
     } else if (ep.kind == EPI_APPLY) {
       if constexpr (DUAL) {
         const long long idx = row * (long long)N + col;

@@ -47,6 +47,10 @@ struct Epilogue {
   // ROTATE (Algorithm 1: moment-rotation lines)
   float* u_out;
   float* v_out;
+  // STORE and APPLY, a matrix projected from the right: output element (row, col) belongs to memory
+  // element col * ldt + row (the product is formed for the transposed problem). STORE: ldt = ldc.
+  int trans, pad2;
+  long long ldt;
 };
 
 struct GemmProblem {
@@ -90,7 +94,9 @@ struct TcProblem {
   const void* const* G_ind;    // entry of the per-call gradient pointer table
   long long G_off;             // element offset of this worker inside it
   const float* cptr;           // clip coefficient
-  int mat, replica, pcopy, pad;  // matrix index, worker index, which copy of P (0 for Global)
+  int mat, replica, pcopy;     // matrix index, worker index, which copy of P (0 for Global)
+  int tr;                      // 1: W, G, E are stored transposed with respect to this problem (a matrix projected from the
+                               // right): m counts their columns, n their rows
   float* tb;                   // [r][n] time buffer of this worker (+= lr * U~ every step), or null
   // the projection's own strip numbering: nsplit strips per 128 columns (2 when 256 < r <= 512: one per
   // half of the rank), and the second half's share of the column scale of the full-rank QHM term
@@ -104,6 +110,8 @@ struct TcProblem {
 // epilogue reads and writes in place); "st": 64 x 16 boxes with the same swizzle.
 struct alignas(128) TmaMatMaps {
   unsigned char e_sw[128], pt[128], p16[128], w_sw[128];
+  // a matrix projected from the right: W as 64 x 128 boxes, and stores of 32 rows of a 64-column tile
+  unsigned char w_kb[128], e_st32[128], w_st32[128];
   // refresh: E and Delta16 as 64 x 128 swizzled boxes ("kb", rows of S as MMA rows), Delta16 as
   // 64 x 64 swizzled boxes, and the three bf16 right-hand sides [batch][Kd][r]
   unsigned char e_kb[128], d_kb[128], d_sw[128], om16[128], pn16[128], zq16[128];
@@ -137,9 +145,10 @@ void launch_apply_tc(const TcProblem* probs, int nprobs, long long total_strips,
 cudaError_t tma_configure();
 void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips_p, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
                         const StepScalars& sc, int grid, unsigned* status, cudaStream_t st);
-// mode 0: r <= 256, one sweep; modes 1 and 2: the two sweeps for 256 < r <= 512
-void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                      const StepScalars& sc, int grid, int mode, unsigned* status, cudaStream_t st);
+// mode 0: r <= 256, one sweep; modes 1 and 2: the two sweeps for 256 < r <= 512. The launch covers the strips
+// [strip_begin, strip_end) of `probs` (problems of one side only: tr = 0 stored as the problem, tr = 1 transposed).
+void launch_apply_tma(const TcProblem* probs, int nprobs, long long strip_begin, long long strip_end, const TmaMatMaps* maps,
+                      const TmaGradMaps* gmaps, const StepScalars& sc, int grid, int mode, int tr, unsigned* status, cudaStream_t st);
 
 void launch_selftest_wait(unsigned* status, cudaStream_t st);
 

@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(256) moments_kernel(const MatDev* __restrict__
   const long long blk = blockIdx.x;
   const int i = find_segment(tile_start, n_mats, blk);
   const MatDev md = mats[i];
-  const long long n = md.n;
+  const long long n = md.ln;  // columns of the low-rank arrays
   const int r = md.r;
   const long long ctiles = (n + 127) / 128;
   const long long local = blk - tile_start[i];
@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(256) outer_states_kernel(const MatDev* __restr
   const long long blk = blockIdx.x;
   const int i = find_segment(blk_start, n_mats, blk);
   const MatDev md = mats[i];
-  const long long elems = (long long)md.r * md.n;
+  const long long elems = (long long)md.r * md.ln;
   const long long e = ((blk - blk_start[i]) * 256 + threadIdx.x) * 4;
   if (e >= elems) return;
   const float inv_k = 1.f / (float)K;

@@ -117,11 +117,16 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           if (!ok) break;
           unsigned char* base = smem + s * SB;
           mbar_expect_tx(&full_bar[s], tx);
-          tma_load_3d(base, gm->g_sw, n0, kb * 64, rep, &full_bar[s]);
-          tma_load_3d(base + 8192, gm->g_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
-          if (ef) {
-            tma_load_3d(base + 16384, mm->e_sw, n0, kb * 64, rep, &full_bar[s]);
-            tma_load_3d(base + 24576, mm->e_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
+          if (pr->tr) {  // stored transposed: the strip's 128 elements are stored rows, the k-block 64 stored columns
+            tma_load_3d(base, gm->g_kb, kb * 64, n0, rep, &full_bar[s]);
+            if (ef) tma_load_3d(base + 16384, mm->e_kb, kb * 64, n0, rep, &full_bar[s]);
+          } else {
+            tma_load_3d(base, gm->g_sw, n0, kb * 64, rep, &full_bar[s]);
+            tma_load_3d(base + 8192, gm->g_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
+            if (ef) {
+              tma_load_3d(base + 16384, mm->e_sw, n0, kb * 64, rep, &full_bar[s]);
+              tma_load_3d(base + 24576, mm->e_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
+            }
           }
           tma_load_3d(base + 32768, mm->pt, kb * 64, r_lo, pc, &full_bar[s]);  // rows past r_n arrive as zeros
         }
@@ -138,7 +143,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
         const int r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
         const int nkb = pr->m_k / 64;
         const uint32_t n_h = (uint32_t)(pr->r_n - r_lo < 256 ? pr->r_n - r_lo : 256);
-        const uint32_t idesc = idesc_bf16_f32(128, n_h) | kIdescAMajorMN;
+        const bool tr = pr->tr != 0;  // the tile then lies as [128 strip elements][64 k]: a K-major operand
+        const uint32_t idesc = idesc_bf16_f32(128, n_h) | (tr ? 0u : kIdescAMajorMN);
         const uint32_t buf = si & 1u;
         ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
         if (!ok) break;
@@ -150,7 +156,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           const uint32_t sA = smem_u32(smem + s * SB), sB = sA + 32768;
 #pragma unroll
           for (int k16 = 0; k16 < 4; ++k16)
-            mma_bf16(tmem + buf * 256, smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            mma_bf16(tmem + buf * 256, tr ? smem_desc_k128(sA + k16 * 32) : smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc,
+                     (kb > 0 || k16 > 0) ? 1u : 0u);
           mma_commit(&empty_bar[s]);
         }
         if (ok) mma_commit(&acc_full[buf]);
@@ -279,9 +286,13 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
 // MODE 0: r <= 256, both products in one sweep. For 256 < r <= 512 one low-rank operand alone fills
 // 256 columns of tensor memory, so the update is two sweeps of the same kernel: MODE 1 does the
 // error-feedback line (operand g^T, tiles G and E), MODE 2 the model update (operand U~^T, tiles G, W).
-template <int MODE>
-__global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
-                                                                 const TmaMatMaps* __restrict__ maps,
+// TR: the problems of this launch are matrices projected from the right, whose W, G, E are stored
+// transposed with respect to the problem: a strip is 128 stored rows, a step 64 stored columns, and the
+// accumulator tile (lane = strip element, column = step element) already lies the way the tiles are
+// stored, so a thread works on 16 neighbouring stored columns of its own row.
+template <int MODE, bool TR>
+__global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long strip_begin,
+                                                                 long long strip_end, const TmaMatMaps* __restrict__ maps,
                                                                  const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
                                                                  unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
@@ -321,7 +332,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
     if (lane == 0) {
       uint32_t jt = 0;
       bool ok = true;
-      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+      for (long long strip = strip_begin + blockIdx.x; strip < strip_end && ok; strip += gridDim.x) {
         const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
         const int n0 = (int)(strip - pr->strip_start) * kStrip;
         const TmaMatMaps* mm = maps + pr->mat;
@@ -335,10 +346,16 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
           unsigned char* base = sIn + is * ISB;
           const bool ld_e = DO_E && ef;
           mbar_expect_tx(&in_full[is], 16384u + (ld_e ? 16384u : 0u) + (DO_W ? 16384u : 0u));
-          for (int hh = 0; hh < 2; ++hh) {  // two 64-column halves per tile, 8 KB each
-            tma_load_3d(base + hh * 8192, gm->g_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
-            if (ld_e) tma_load_3d(base + EOFF + hh * 8192, mm->e_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
-            if (DO_W) tma_load_3d(base + WOFF + hh * 8192, mm->w_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+          if (TR) {  // one box of 128 stored rows x 64 stored columns per tile
+            tma_load_3d(base, gm->g_kb, t * kARows, n0, rep, &in_full[is]);
+            if (ld_e) tma_load_3d(base + EOFF, mm->e_kb, t * kARows, n0, rep, &in_full[is]);
+            if (DO_W) tma_load_3d(base + WOFF, mm->w_kb, t * kARows, n0, rep, &in_full[is]);
+          } else {
+            for (int hh = 0; hh < 2; ++hh) {  // two 64-column halves per tile, 8 KB each
+              tma_load_3d(base + hh * 8192, gm->g_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+              if (ld_e) tma_load_3d(base + EOFF + hh * 8192, mm->e_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+              if (DO_W) tma_load_3d(base + WOFF + hh * 8192, mm->w_sw, n0 + hh * 64, t * kARows, rep, &in_full[is]);
+            }
           }
         }
       }
@@ -348,7 +365,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
     if (lane == 0) {
       uint32_t jt = 0;
       bool ok = true;
-      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+      for (long long strip = strip_begin + blockIdx.x; strip < strip_end && ok; strip += gridDim.x) {
         const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
         const TmaMatMaps* mm = maps + pr->mat;
         const int nkb = pr->r_k / 64, pc = pr->pcopy;
@@ -368,7 +385,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       const uint32_t idesc = idesc_bf16_f32(128, kARows);
       uint32_t jt = 0, si = 0;
       bool ok = true;
-      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+      for (long long strip = strip_begin + blockIdx.x; strip < strip_end && ok; strip += gridDim.x, ++si) {
         const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
         const int nkb = pr->r_k / 64;
         const int nsteps = (pr->m + kARows - 1) / kARows;
@@ -405,7 +422,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
     // 2(t%4), +1, +8, +9 of its row group: 8-byte accesses to the swizzled tiles, free of conflicts.
     const int ew = warp - 2;
     const int q = warp & 3, grp = ew >> 2;  // lane quarter (fixed by the hardware), row group 0..3
-    const int colq = q * 32 + 4 * (lane & 7) + (lane >> 3);  // column this lane's operands belong to
+    const int colq = TR ? q * 32 + lane : q * 32 + 4 * (lane & 7) + (lane >> 3);  // strip element this lane's operands belong to
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
     const int tb = lane >> 2, tr = lane & 3;
     const int ecol0 = q * 32 + 4 * tb;  // first of this thread's four epilogue columns
@@ -422,7 +439,7 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
     const float a2w = full ? om : 1.f;
     uint32_t jt = 0, si = 0;
     bool ok = true;
-    for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+    for (long long strip = strip_begin + blockIdx.x; strip < strip_end && ok; strip += gridDim.x, ++si) {
       const TcProblem* __restrict__ pr = probs + find_problem(probs, nprobs, strip);
       const int n = pr->n, r_k = pr->r_k;
       const int n0 = (int)(strip - pr->strip_start) * kStrip;
@@ -434,7 +451,8 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
       float cd[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const long long ec = (long long)n0 + ecol0 + j;
+        // TR: one strip element per thread (its own row); else the four columns of the thread's epilogue block
+        const long long ec = TR ? col : (long long)n0 + ecol0 + j;
         const long long ecc = ec < n ? ec : (long long)n - 1;
         cd[j] = full ? (1.f - om) * c / (pr->dcol[ecc] + (pr->dcol2 ? pr->dcol2[ecc] : 0.f)) : 0.f;
       }
@@ -471,67 +489,118 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
         if (ok) ok = mbar_wait<32>(&acc_full[b], (jt >> 1) & 1u, status);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
-        // both accumulators come out of tensor memory together and the buffer goes back to the MMA
-        // warp before any arithmetic. a?[h][4k + 2jj + p]: column 2h + jj, row 8k + 2(t%4) + p.
-        float a1[2][8], a2[2][8];
+        if constexpr (TR) {
+          // this thread: stored row 32q + lane of the strip, stored columns 16 grp .. +15 of the step
+          const int row = q * 32 + lane;
+          const uint32_t o0 = swz_chunk(row, 2 * grp), o1 = swz_chunk(row, 2 * grp + 1);
+          float a1[16], a2[16];
+          const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
+          if (DO_E && DO_W) tmem_ld16x2(taddr, taddr + 64, a1, a2);
+          else if (DO_E) tmem_ld16(taddr, a1);
+          else tmem_ld16(taddr + 64, a2);
+          tc_fence_before_sync();
+          mbar_arrive(&acc_empty[b]);
+          const uint4 gq[2] = {*reinterpret_cast<const uint4*>(base + o0), *reinterpret_cast<const uint4*>(base + o1)};
+          const float cdv = cd[0];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (DO_E) tmem_ld_16x256b_x2(taddr + ((uint32_t)(h * 16) << 16), a1[h]);       // (P g)^T
-          if (DO_W) tmem_ld_16x256b_x2(taddr + 64 + ((uint32_t)(h * 16) << 16), a2[h]);  // (P U~)^T
-        }
-        tmem_ld_wait();
+          for (int h = 0; h < 2; ++h) {
+            const uint32_t off = h ? o1 : o0;
+            const uint32_t gw[4] = {gq[h].x, gq[h].y, gq[h].z, gq[h].w};
+            if (DO_E && ef) {
+              const uint4 eq = *reinterpret_cast<const uint4*>(base + EOFF + off);
+              const uint32_t ew4[4] = {eq.x, eq.y, eq.z, eq.w};
+              uint32_t o[4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (DO_E) tmem_ld_pin8(a1[h]);
-          if (DO_W) tmem_ld_pin8(a2[h]);
-        }
-        tc_fence_before_sync();
-        mbar_arrive(&acc_empty[b]);
-        uint2 gv[4], ev[4], wv[4];
+              for (int j = 0; j < 4; ++j)
+                o[j] = pack2_bf16((c * bf_lo(gw[j]) + bf_lo(ew4[j])) - a1[8 * h + 2 * j], (c * bf_hi(gw[j]) + bf_hi(ew4[j])) - a1[8 * h + 2 * j + 1]);
+              *reinterpret_cast<uint4*>(base + EOFF + off) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            if (DO_W) {
+              const uint4 wq = *reinterpret_cast<const uint4*>(base + WOFF + off);
+              const uint32_t ww[4] = {wq.x, wq.y, wq.z, wq.w};
+              uint32_t o[4];
 #pragma unroll
-        for (int ri = 0; ri < 4; ++ri) {
-          gv[ri] = *reinterpret_cast<const uint2*>(base + toff[ri]);
-          if (DO_E && ef) ev[ri] = *reinterpret_cast<const uint2*>(base + EOFF + toff[ri]);
-          if (DO_W) wv[ri] = *reinterpret_cast<const uint2*>(base + WOFF + toff[ri]);
-        }
-#pragma unroll
-        for (int ri = 0; ri < 4; ++ri) {
-          const int k = ri >> 1, p = ri & 1;
-          const float g0 = bf_lo(gv[ri].x), g1 = bf_hi(gv[ri].x), g2 = bf_lo(gv[ri].y), g3 = bf_hi(gv[ri].y);
-          if (DO_E && ef) {
-            const float e0 = (c * g0 + bf_lo(ev[ri].x)) - a1[0][4 * k + p];
-            const float e1 = (c * g1 + bf_hi(ev[ri].x)) - a1[0][4 * k + 2 + p];
-            const float e2 = (c * g2 + bf_lo(ev[ri].y)) - a1[1][4 * k + p];
-            const float e3 = (c * g3 + bf_hi(ev[ri].y)) - a1[1][4 * k + 2 + p];
-            *reinterpret_cast<uint2*>(base + EOFF + toff[ri]) = make_uint2(pack2_bf16(e0, e1), pack2_bf16(e2, e3));
+              for (int j = 0; j < 4; ++j)
+                o[j] = pack2_bf16(bf_lo(ww[j]) - lr * (cdv * bf_lo(gw[j]) + a2w * a2[8 * h + 2 * j]),
+                                  bf_hi(ww[j]) - lr * (cdv * bf_hi(gw[j]) + a2w * a2[8 * h + 2 * j + 1]));
+              *reinterpret_cast<uint4*>(base + WOFF + off) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
           }
-          if (DO_W) {
-            const float w0 = bf_lo(wv[ri].x) - lr * (cd[0] * g0 + a2w * a2[0][4 * k + p]);
-            const float w1 = bf_hi(wv[ri].x) - lr * (cd[1] * g1 + a2w * a2[0][4 * k + 2 + p]);
-            const float w2 = bf_lo(wv[ri].y) - lr * (cd[2] * g2 + a2w * a2[1][4 * k + p]);
-            const float w3 = bf_hi(wv[ri].y) - lr * (cd[3] * g3 + a2w * a2[1][4 * k + 2 + p]);
-            *reinterpret_cast<uint2*>(base + WOFF + toff[ri]) = make_uint2(pack2_bf16(w0, w1), pack2_bf16(w2, w3));
+          // the four warps that share 32 stored rows hand them to the TMA engine on their own
+          fence_async_smem();
+          asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");
+          if (grp == 0 && lane == 0) {
+            if (n0 + q * 32 < n) {
+              if (DO_E && ef) tma_store_3d(mm->e_st32, t * kARows, n0 + q * 32, rep, base + EOFF + q * 4096);
+              if (DO_W) tma_store_3d(mm->w_st32, t * kARows, n0 + q * 32, rep, base + WOFF + q * 4096);
+            }
+            tma_store_commit();
+            tma_store_wait_read();
+            mbar_arrive(&in_free[is]);
           }
-        }
-        // the four warps of a row group hand their 16 rows to the TMA engine on their own
-        fence_async_smem();
-        asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory");
-        if ((ew & 3) == 0 && lane == 0) {
-          unsigned char* sb = base + grp * 2048;
-          const int row = t * kARows + grp * 16;
-          for (int hh = 0; hh < 2; ++hh) {
-            if (n0 + hh * 64 >= n) break;
-            if (DO_E && ef) tma_store_3d(mm->e_st, n0 + hh * 64, row, rep, sb + EOFF + hh * 8192);
-            if (DO_W) tma_store_3d(mm->w_st, n0 + hh * 64, row, rep, sb + WOFF + hh * 8192);
+        } else {
+          const uint32_t taddr = tmem + lane_base + 256 + b * 128 + (uint32_t)(grp * 16);
+          // both accumulators come out of tensor memory together and the buffer goes back to the MMA
+          // warp before any arithmetic. a?[h][4k + 2jj + p]: column 2h + jj, row 8k + 2(t%4) + p.
+          float a1[2][8], a2[2][8];
+  #pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if (DO_E) tmem_ld_16x256b_x2(taddr + ((uint32_t)(h * 16) << 16), a1[h]);       // (P g)^T
+            if (DO_W) tmem_ld_16x256b_x2(taddr + 64 + ((uint32_t)(h * 16) << 16), a2[h]);  // (P U~)^T
           }
-          tma_store_commit();
-          tma_store_wait_read();
-          mbar_arrive(&in_free[is]);
+          tmem_ld_wait();
+  #pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if (DO_E) tmem_ld_pin8(a1[h]);
+            if (DO_W) tmem_ld_pin8(a2[h]);
+          }
+          tc_fence_before_sync();
+          mbar_arrive(&acc_empty[b]);
+          uint2 gv[4], ev[4], wv[4];
+  #pragma unroll
+          for (int ri = 0; ri < 4; ++ri) {
+            gv[ri] = *reinterpret_cast<const uint2*>(base + toff[ri]);
+            if (DO_E && ef) ev[ri] = *reinterpret_cast<const uint2*>(base + EOFF + toff[ri]);
+            if (DO_W) wv[ri] = *reinterpret_cast<const uint2*>(base + WOFF + toff[ri]);
+          }
+  #pragma unroll
+          for (int ri = 0; ri < 4; ++ri) {
+            const int k = ri >> 1, p = ri & 1;
+            const float g0 = bf_lo(gv[ri].x), g1 = bf_hi(gv[ri].x), g2 = bf_lo(gv[ri].y), g3 = bf_hi(gv[ri].y);
+            if (DO_E && ef) {
+              const float e0 = (c * g0 + bf_lo(ev[ri].x)) - a1[0][4 * k + p];
+              const float e1 = (c * g1 + bf_hi(ev[ri].x)) - a1[0][4 * k + 2 + p];
+              const float e2 = (c * g2 + bf_lo(ev[ri].y)) - a1[1][4 * k + p];
+              const float e3 = (c * g3 + bf_hi(ev[ri].y)) - a1[1][4 * k + 2 + p];
+              *reinterpret_cast<uint2*>(base + EOFF + toff[ri]) = make_uint2(pack2_bf16(e0, e1), pack2_bf16(e2, e3));
+            }
+            if (DO_W) {
+              const float w0 = bf_lo(wv[ri].x) - lr * (cd[0] * g0 + a2w * a2[0][4 * k + p]);
+              const float w1 = bf_hi(wv[ri].x) - lr * (cd[1] * g1 + a2w * a2[0][4 * k + 2 + p]);
+              const float w2 = bf_lo(wv[ri].y) - lr * (cd[2] * g2 + a2w * a2[1][4 * k + p]);
+              const float w3 = bf_hi(wv[ri].y) - lr * (cd[3] * g3 + a2w * a2[1][4 * k + 2 + p]);
+              *reinterpret_cast<uint2*>(base + WOFF + toff[ri]) = make_uint2(pack2_bf16(w0, w1), pack2_bf16(w2, w3));
+            }
+          }
+          // the four warps of a row group hand their 16 rows to the TMA engine on their own
+          fence_async_smem();
+          asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory");
+          if ((ew & 3) == 0 && lane == 0) {
+            unsigned char* sb = base + grp * 2048;
+            const int row = t * kARows + grp * 16;
+            for (int hh = 0; hh < 2; ++hh) {
+              if (n0 + hh * 64 >= n) break;
+              if (DO_E && ef) tma_store_3d(mm->e_st, n0 + hh * 64, row, rep, sb + EOFF + hh * 8192);
+              if (DO_W) tma_store_3d(mm->w_st, n0 + hh * 64, row, rep, sb + WOFF + hh * 8192);
+            }
+            tma_store_commit();
+            tma_store_wait_read();
+            mbar_arrive(&in_free[is]);
+          }
         }
       }
     }
-    if ((ew & 3) == 0 && lane == 0) tma_store_wait_all();
+    if ((TR ? grp == 0 : (ew & 3) == 0) && lane == 0) tma_store_wait_all();
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -547,11 +616,17 @@ cudaError_t tma_configure() {
   e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
   if (e != cudaSuccess) return e;
   const int smem = (int)(kAPStages * 65536 + kAInStages * 32768 + 1024);  // the largest of the three modes
-  e = cudaFuncSetAttribute(apply_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  e = cudaFuncSetAttribute(apply_tma_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(apply_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  e = cudaFuncSetAttribute(apply_tma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(apply_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  e = cudaFuncSetAttribute(apply_tma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(apply_tma_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(apply_tma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(apply_tma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
 void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
@@ -559,13 +634,23 @@ void launch_project_tma(const TcProblem* probs, int nprobs, long long total_stri
   const long long g = total_strips < grid ? total_strips : grid;
   project_tma_kernel<<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
 }
-void launch_apply_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
-                      const StepScalars& sc, int grid, int mode, unsigned* status, cudaStream_t st) {
-  const unsigned g = (unsigned)(total_strips < grid ? total_strips : grid);
+void launch_apply_tma(const TcProblem* probs, int nprobs, long long strip_begin, long long strip_end, const TmaMatMaps* maps,
+                      const TmaGradMaps* gmaps, const StepScalars& sc, int grid, int mode, int tr, unsigned* status, cudaStream_t st) {
+  const long long total = strip_end - strip_begin;
+  if (total <= 0) return;
+  const unsigned g = (unsigned)(total < grid ? total : grid);
   const size_t small = kAPStages * kAPStageBytes + kAInStages * kAInStageBytes + 1024, large = kAPStages * 65536 + kAInStages * 32768 + 1024;
-  if (mode == 0) apply_tma_kernel<0><<<g, kAThreads, small, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
-  else if (mode == 1) apply_tma_kernel<1><<<g, kAThreads, large, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
-  else apply_tma_kernel<2><<<g, kAThreads, large, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+#define LORDO_APPLY(M, T, SM) apply_tma_kernel<M, T><<<g, kAThreads, SM, st>>>(probs, nprobs, strip_begin, strip_end, maps, gmaps, sc, status)
+  if (!tr) {
+    if (mode == 0) LORDO_APPLY(0, false, small);
+    else if (mode == 1) LORDO_APPLY(1, false, large);
+    else LORDO_APPLY(2, false, large);
+  } else {
+    if (mode == 0) LORDO_APPLY(0, true, small);
+    else if (mode == 1) LORDO_APPLY(1, true, large);
+    else LORDO_APPLY(2, true, large);
+  }
+#undef LORDO_APPLY
 }
 
 }  // namespace lordo

@@ -36,7 +36,7 @@ class LordoError(RuntimeError):
 
 
 class _Mat(C.Structure):
-    _fields_ = [("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int32), ("reserved", C.c_int32)]
+    _fields_ = [("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int32), ("side", C.c_int32)]
 
 
 class _Config(C.Structure):
@@ -123,11 +123,12 @@ def _stream_handle(stream: Optional[torch.cuda.Stream]) -> C.c_void_p:
 
 def make_config(mats: Sequence[Tuple[int, int, int]], K: int, H: int, *, w_dtype=F32, g_dtype=F32, e_dtype=F32,
                 variant=GLOBAL, error_feedback=True, beta2=0.999, eps=1e-8, clip_rho=0.0, clip_scope=0, sync_u=True,
-                sync_v=True, outer=OUTER_AVG, outer_lr=1.0, outer_momentum=0.0, power_iters=0, seed=0, check_mode=1, warm_start=0, time_buffer=0, oversample=0):
-    """Returns (config struct, keep-alive matrix array)."""
+                sync_v=True, outer=OUTER_AVG, outer_lr=1.0, outer_momentum=0.0, power_iters=0, seed=0, check_mode=1, warm_start=0, time_buffer=0, oversample=0,
+                sides: Optional[Sequence[int]] = None):
+    """Returns (config struct, keep-alive matrix array). sides[i] = 1 projects matrix i from the right."""
     arr = (_Mat * len(mats))()
     for i, (m, n, r) in enumerate(mats):
-        arr[i] = _Mat(m, n, r, 0)
+        arr[i] = _Mat(m, n, r, int(sides[i]) if sides is not None else 0)
     cfg = _Config(len(mats), arr, K, H, w_dtype, g_dtype, e_dtype, variant, int(error_feedback), beta2, eps, clip_rho,
                   clip_scope, int(sync_u), int(sync_v), outer, outer_lr, outer_momentum, power_iters, seed, check_mode, int(warm_start), int(time_buffer), int(oversample))
     return cfg, arr
@@ -181,19 +182,21 @@ class Lordo:
         self.variant = kw.get("variant", GLOBAL)
         self.error_feedback = bool(kw.get("error_feedback", True))
         self.outer = kw.get("outer", OUTER_AVG)
+        self.sides = [int(x) for x in kw["sides"]] if kw.get("sides") is not None else [0] * len(self.mats)
         self.cfg, self._mats_keep = make_config(self.mats, K, H, w_dtype=_dtype_code(w_dt), g_dtype=_dtype_code(g_dtype),
                                                 e_dtype=_dtype_code(e_dtype), **kw)
         dev = self.device
         z = lambda shape, dt=torch.float32: torch.empty(shape, device=dev, dtype=dt)
         self.W, self.E, self.P, self.u, self.v, self.X0, self.B, self.Delta = [], [], [], [], [], [], [], []
-        for (m, n, r), w0 in zip(self.mats, W0):
+        for (m, n, r), w0, side in zip(self.mats, W0, self.sides):
             w = z((K, m, n), w_dt)
             w[0].copy_(w0.to(dev))
             self.W.append(w)
             self.E.append(z((K, m, n), e_dtype) if self.error_feedback else None)
-            self.P.append(z((K, m, r)) if self.variant == LOCAL else z((m, r)))
-            self.u.append(z((K, r, n)))
-            self.v.append(z((K, r, n)))
+            pm, ln = (n, m) if side else (m, n)  # rows of the basis, columns of the low-rank moments
+            self.P.append(z((K, pm, r)) if self.variant == LOCAL else z((pm, r)))
+            self.u.append(z((K, r, ln)))
+            self.v.append(z((K, r, ln)))
             self.X0.append(z((m, n)))
             self.B.append(z((m, n)) if self.outer == OUTER_NESTEROV else None)
             self.Delta.append(z((m, n)))

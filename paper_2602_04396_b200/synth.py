@@ -50,6 +50,7 @@ class Workload:
     clip_rho: float = 1.0
     signal_rank: int = 32
     noise: float = 0.1
+    sides: Tuple[int, ...] | None = None  # per matrix: 1 = the basis is applied from the right (default: all from the left)
 
     @property
     def weights(self) -> int:

@@ -52,6 +52,13 @@ def _np_state(x) -> np.ndarray:
     return x.detach().to(torch.float32).cpu().numpy().astype(np.float64)
 
 
+def _moments(x, orc: lo.LordoOracle, i: int) -> np.ndarray:
+    """Moments of matrix i as the oracle holds them: the CUDA path keeps [K][r][.] for either side, the
+    oracle's right-side moments are [K][rows][r]."""
+    a = _np_state(x)
+    return np.swapaxes(a, 1, 2) if orc.side(i) == 1 else a
+
+
 def f32(x: float) -> float:
     """The value a C `float` argument carries: both sides are fed the same fp32 hyper-parameters."""
     return float(np.float32(x))
@@ -74,7 +81,8 @@ def make_gpu(spec: RunSpec):
                        beta2=spec.beta2, eps=spec.eps, clip_rho=wl.clip_rho, clip_scope=spec.clip_scope,
                        sync_u=spec.sync_u, sync_v=spec.sync_v, outer=spec.outer, outer_lr=spec.outer_lr,
                        outer_momentum=spec.outer_momentum, power_iters=wl.power_iters, seed=spec.seed,
-                       check_mode=spec.check_mode, warm_start=int(spec.warm_start), time_buffer=int(spec.time_buffer), oversample=spec.oversample)
+                       check_mode=spec.check_mode, warm_start=int(spec.warm_start), time_buffer=int(spec.time_buffer), oversample=spec.oversample,
+                       sides=wl.sides)
 
 
 def device_grads(wl: synth.Workload, G: List[np.ndarray]) -> List[torch.Tensor]:
@@ -104,7 +112,8 @@ def make_oracle(spec: RunSpec) -> lo.LordoOracle:
                           beta2=f32(spec.beta2), eps=f32(spec.eps), clip_rho=f32(wl.clip_rho), clip_scope=spec.clip_scope,
                           sync_u=spec.sync_u, sync_v=spec.sync_v, outer=spec.outer, outer_lr=f32(spec.outer_lr),
                           outer_momentum=f32(spec.outer_momentum), power_iters=wl.power_iters, seed=spec.seed,
-                          w_dtype=wl.w_dtype, e_dtype=wl.e_dtype, state_dtype="f32", warm_start=spec.warm_start, time_buffer=spec.time_buffer, oversample=spec.oversample)
+                          w_dtype=wl.w_dtype, e_dtype=wl.e_dtype, state_dtype="f32", warm_start=spec.warm_start, time_buffer=spec.time_buffer, oversample=spec.oversample,
+                          sides=wl.sides)
     return lo.LordoOracle(cfg, synth.init_weights(wl, spec.seed))
 
 
@@ -115,8 +124,8 @@ def sync_oracle_from_gpu(opt, orc: lo.LordoOracle) -> None:
         if opt.E[i] is not None:
             orc.E[i] = _np_state(opt.E[i])
         orc.P[i] = _np_state(opt.P[i])
-        orc.u[i] = _np_state(opt.u[i])
-        orc.v[i] = _np_state(opt.v[i])
+        orc.u[i] = _moments(opt.u[i], orc, i)
+        orc.v[i] = _moments(opt.v[i], orc, i)
         orc.X0[i] = _np_state(opt.X0[i])
         orc.Delta[i] = _np_state(opt.Delta[i])
         if opt.B[i] is not None:
@@ -176,7 +185,9 @@ def run_lockstep_refresh(spec: RunSpec, rounded_signal: bool = False, inject_del
             for i, (m, n, r) in enumerate(wl.mats):
                 Pg = _np_state(opt.P[i])
                 for k, S in enumerate(signals[i]):
-                    Om = None if spec.warm_start else lo.random_matrix(spec.seed, lo.PURPOSE_OMEGA, i, pre["refreshes"], k, n, r)
+                    if orc.side(i) == 1:
+                        S = S.T
+                    Om = None if spec.warm_start else lo.random_matrix(spec.seed, lo.PURPOSE_OMEGA, i, pre["refreshes"], k, S.shape[1], r)
                     Po = pre["P"][i][k] if Pg.ndim == 3 else pre["P"][i]
                     want = range_finder_bf16_rhs(S, Om, Po, q)
                     worst["P_angle_bf16rhs"] = max(worst.get("P_angle_bf16rhs", 0.0),
@@ -184,11 +195,13 @@ def run_lockstep_refresh(spec: RunSpec, rounded_signal: bool = False, inject_del
         if pre["s"] > 0:
             for i in range(len(wl.mats)):
                 Pg = _np_state(opt.P[i])
-                ug, vg = _np_state(opt.u[i]), _np_state(opt.v[i])
+                ug, vg = _np_state(opt.u[i]), _np_state(opt.v[i])  # [K][r][.] for either side
+                right = orc.side(i) == 1
                 for k in range(wl.K):
                     Pn = Pg[k] if Pg.ndim == 3 else Pg
                     Po = pre["P"][i][k] if Pg.ndim == 3 else pre["P"][i]
-                    un, vn = lo.rotate_moments(pre["u"][i][k], pre["v"][i][k], Pn, Po, b1, orc.cfg.beta2, pre["s"])
+                    u0, v0 = (pre["u"][i][k].T, pre["v"][i][k].T) if right else (pre["u"][i][k], pre["v"][i][k])
+                    un, vn = lo.rotate_moments(u0, v0, Pn, Po, b1, orc.cfg.beta2, pre["s"])
                     worst["rot_u"] = max(worst.get("rot_u", 0.0), scaled_error(ug[k], un))
                     worst["rot_v"] = max(worst.get("rot_v", 0.0), scaled_error(vg[k], vn))
         if signals is not None:
@@ -199,6 +212,8 @@ def run_lockstep_refresh(spec: RunSpec, rounded_signal: bool = False, inject_del
                 if Pg.ndim == 2:
                     Pg, Po = Pg[None], Po[None]
                 for k, S in enumerate(per_rep):
+                    if orc.side(i) == 1:
+                        S = S.T
                     ratio = float(np.sum((Pg[k].T @ S) ** 2) / max(np.sum((Po[k].T @ S) ** 2), 1e-300))
                     worst["energy"] = min(worst.get("energy", 1e9), ratio)
 
@@ -312,8 +327,8 @@ def compare_states(opt, orc: lo.LordoOracle) -> Dict[str, float]:
         out["W_fro"] = max(out["W_fro"], frobenius_error(Wg, orc.W[i]))
         if opt.E[i] is not None:
             out["E"] = max(out["E"], scaled_error(_np_state(opt.E[i]), orc.E[i]))
-        out["u"] = max(out["u"], scaled_error(_np_state(opt.u[i]), orc.u[i]))
-        out["v"] = max(out["v"], scaled_error(_np_state(opt.v[i]), orc.v[i]))
+        out["u"] = max(out["u"], scaled_error(_moments(opt.u[i], orc, i), orc.u[i]))
+        out["v"] = max(out["v"], scaled_error(_moments(opt.v[i], orc, i), orc.v[i]))
         out["X0"] = max(out["X0"], weight_error(_np_state(opt.X0[i]), orc.X0[i]))
         out["Delta"] = max(out["Delta"], scaled_error(_np_state(opt.Delta[i]), orc.Delta[i]))
         if opt.B[i] is not None:

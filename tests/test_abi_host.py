@@ -51,6 +51,10 @@ def test_workspace_query_and_validation(lib):
         ([(256, 256, 16)], dict(oversample=8, warm_start=1), 8),    # needs a fresh sketch
         ([(256, 24, 16)], dict(oversample=16), 2),                  # r + p > n
         ([(1024, 1024, 512)], dict(oversample=96), 2),              # r + p > 600
+        ([(252, 256, 16)], dict(sides=[1]), 3),                     # projected from the right: m not a multiple of 8
+        ([(256, 256, 16)], dict(sides=[2]), 1),                     # no such side
+        ([(256, 256, 16)], dict(sides=[1], time_buffer=1), 8),      # not available from the right
+        ([(256, 256, 16)], dict(sides=[1], oversample=8), 8),
     ]
     for mats, kw, code in bad:
         cfg, _k = lordo.make_config(mats, 2, 4, **kw)
@@ -67,6 +71,10 @@ def test_workspace_query_and_validation(lib):
     cfg, _k = lordo.make_config([(256, 256, 16)], 65, 4)
     with pytest.raises(lordo.LordoError):
         lordo.query_workspace(cfg)
+    # projected from the right, the low-rank arrays of a tall matrix have m columns instead of n
+    tall_l, _kl = lordo.make_config([(1024, 128, 16)], 2, 4, check_mode=1)
+    tall_r, _kr = lordo.make_config([(1024, 128, 16)], 2, 4, check_mode=1, sides=[1])
+    assert lordo.query_workspace(tall_r) > lordo.query_workspace(tall_l)
 
 
 def test_null_arguments_are_rejected(lib):

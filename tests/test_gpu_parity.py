@@ -819,3 +819,98 @@ def test_checkpoint_between_sync_and_global_refresh():
     assert torch.equal(mssv_a, mssv_b)
     with pytest.raises(lordo.LordoError):
         b.refresh_subspace(None, 0.9)  # the refresh that was owed has been run
+
+
+# ------------------------------------------------------------------ projection from the right (not in the paper)
+
+def _right(m, n, r, **kw):
+    return synth.scaled(_small(m=m, n=n, r=r, **kw), sides=(1,))
+
+
+@pytest.mark.parametrize("form", [0, 1, 2])
+@pytest.mark.parametrize("ef", [True, False])
+@pytest.mark.parametrize("variant", [0, 1])
+def test_right_side_inner_steps_ragged(form, ef, variant):
+    """A matrix with more rows than columns projected from the right (P is n x r, moments kept as [r][m]),
+    fp32 arithmetic, against the oracle's right-side path; shapes with ragged tiles in both directions."""
+    wl = _right(264, 136, 24, K=3, H=3, rounds=1, clip_rho=30.0)
+    spec = RunSpec(wl, variant=variant, form=form, error_feedback=ef, refresh=(variant == 1), lr=0.01, omega=0.9)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    assert tuple(opt.P[0].shape)[-2:] == (136, 24) and tuple(opt.u[0].shape) == (3, 24, 264)
+    st = hz.compare_states(opt, orc)
+    assert st["W"] < W_TOL and st["u"] < 1e-4 and st["v"] < 1e-4 and st["E"] < 1e-4 and st["P_orth"] < 1e-5, st
+    assert opt.poll_status() == 0
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("q", [0, 2])
+def test_right_side_refresh_and_rotation(variant, q):
+    """Every refresh compared on the CUDA path's own state (the sketch of a rank-8 signal with r = 32 has a
+    condition number of a few thousand, which two free-running fp32 / fp64 trajectories turn into an angle
+    of about 1e-3 between their signals' trailing directions)."""
+    wl = _right(264, 200, 32, K=2, H=2, rounds=2, grad="lowrank", power_iters=q, signal_rank=8)
+    spec = RunSpec(wl, variant=variant, form=2, lr=0.01, outer=1)
+    opt, orc, worst = hz.run_lockstep_refresh(spec)
+    st = hz.compare_states(opt, orc)
+    assert worst["P_orth"] < 1e-5 and worst["P_angle"] < ANGLE_TOL and worst["u"] < 1e-3 and worst["v"] < 1e-3, worst
+    assert worst["rot_u"] < 1e-4 and worst["rot_v"] < 1e-4, worst
+    assert st["W"] < W_TOL and st["X0"] < W_TOL, st
+    assert opt.poll_status() == 0
+
+
+def test_mixed_sides_in_one_context():
+    """The usual arrangement: wide matrices from the left, tall ones from the right, one context, both rules,
+    warm-started refresh included."""
+    wl = synth.Workload("mixed", ((136, 264, 24), (264, 136, 24), (200, 200, 16)), K=2, H=2, rounds=2, grad="lowrank", signal_rank=8,
+                        clip_rho=30.0, power_iters=1, sides=(0, 1, 1))
+    for variant, form, warm in ((0, 2, False), (1, 1, False), (0, 2, True)):
+        spec = RunSpec(wl, variant=variant, form=form, lr=0.01, outer=1, warm_start=warm)
+        opt, orc, worst = hz.run_lockstep_refresh(spec)
+        st = hz.compare_states(opt, orc)
+        assert opt.poll_status() == 0
+        assert worst["P_angle"] < ANGLE_TOL and worst["P_orth"] < 1e-5 and worst["u"] < 1e-3 and worst["v"] < 1e-3, worst
+        assert worst["rot_u"] < 1e-4 and worst["rot_v"] < 1e-4 and st["W"] < W_TOL, (worst, st)
+
+
+@pytest.mark.parametrize("shape", [(264, 136, 24), (392, 200, 72), (2048, 384, 256), (520, 600, 320), (1032, 704, 512), (64, 64, 8), (1032, 136, 24)])
+@pytest.mark.parametrize("form,variant,ef", [(2, 0, True), (1, 1, True), (0, 0, False)])
+def test_right_side_fast_mode_inner_steps_bf16(shape, form, variant, ef):
+    """bf16 storage in fast mode: the TMA-fed kernels with the tiles taken the other way round (the strip is
+    128 stored rows, a step 64 stored columns), at the tolerances of the left-side fast path."""
+    m, n, r = shape
+    wl = _right(m, n, r, K=2, H=3, rounds=1, clip_rho=30.0, w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    spec = RunSpec(wl, variant=variant, form=form, error_feedback=ef, refresh=False, lr=0.01, omega=0.9, check_mode=0, eps=0.05)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    st = hz.compare_states(opt, orc)
+    assert opt.poll_status() == 0
+    assert st["u"] < FAST_TOL and st["v"] < 2 * FAST_TOL and st["E"] < 2 * FAST_TOL, st
+    assert _update_error(opt, orc, spec) < 0.05, _update_error(opt, orc, spec)
+    d = hz.bf16_ulp_distance(hz._np_state(opt.W[0]), orc.W[0])
+    assert (d <= 1).mean() > 0.99 and d.max() <= 8, ((d <= 1).mean(), d.max())
+
+
+@pytest.mark.parametrize("variant,form,q", [(0, 2, 0), (0, 2, 2), (1, 1, 2)])
+def test_right_side_fast_mode_refresh_on_tensor_cores(variant, form, q):
+    m, n, r = 520, 392, 136
+    wl = _right(m, n, r, K=2, H=2, rounds=2, grad="lowrank" if q else "gauss", signal_rank=r, noise=0.005, clip_rho=30.0, power_iters=q,
+                w_dtype="bf16", g_dtype="bf16", e_dtype="bf16")
+    spec = RunSpec(wl, variant=variant, form=form, lr=0.01, check_mode=0, eps=0.05)
+    inject = (lambda rnd, i: 1e-2 * synth.gradients(wl, 77, rnd, 0)[i][0]) if variant == 0 else None
+    opt, orc, worst = hz.run_lockstep_refresh(spec, rounded_signal=True, inject_delta=inject)
+    assert opt.poll_status() == 0
+    assert worst["P_angle"] < ANGLE_TOL and worst["P_angle_bf16rhs"] < ANGLE_TOL and worst["P_orth"] < TC_ORTH_TOL, worst
+    assert worst["rot_u"] < ROT_TOL and worst["rot_v"] < 2 * ROT_TOL, worst
+
+
+def test_right_side_config3_down_projection():
+    """The down projection of the 125M-shaped stack (3072 x 768, r = 128, K = 8, bf16) projected from the right,
+    check mode, with the lockstep form of the refresh comparison; and the same in fast mode."""
+    wl = synth.scaled(synth.config(3, 128), mats=[(3072, 768, 128)], H=3, rounds=2, sides=(1,))
+    spec = RunSpec(wl, variant=0, form=2, beta1=0.999)
+    opt, orc = hz.run_gpu(spec), hz.run_oracle(spec)
+    _bf16_check(opt, orc)
+    _lockstep_refresh_check(spec)
+    fast = RunSpec(wl, variant=0, form=2, beta1=0.999, check_mode=0, eps=0.05)
+    opt, orc, worst = hz.run_lockstep_refresh(fast, rounded_signal=True)
+    assert opt.poll_status() == 0
+    assert worst["P_orth"] < TC_ORTH_TOL and worst["rot_u"] < ROT_TOL and worst["rot_v"] < 2 * ROT_TOL, worst
