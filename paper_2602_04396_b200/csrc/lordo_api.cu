@@ -644,12 +644,19 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
       // CholeskyQR2 with the Gram matrices and the products with R^-1 on tensor cores, operands in three
       // planes: the Gram matrix then carries fp32's rounding noise, which the breakdown threshold of the
       // Cholesky step assumes
-      auto cholqr2_tc = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows) {
+      // `last` = false: the result only serves as the right-hand side of the next product of the subspace
+      // iteration. Such a basis has to span the same subspace and be well conditioned, no more: one pass
+      // instead of two, which leaves it orthonormal to cond(X)^2 * 1e-7. Both products keep their three
+      // planes: with fewer, the rounding of X (relative 2^-9 or 2^-17) times cond(X) would enter the
+      // weak directions of the span (measured: angles of 0.03..0.1 rad with one plane on a sketch of
+      // condition 1e3).
+      auto cholqr2_tc = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows,
+                            bool last) {
         const bool by_m = rows == m;
         const unsigned char* x_sw = by_m ? mmi->xm_sw : mmi->xn_sw;
         const unsigned char* x_kb = by_m ? mmi->xm_kb : mmi->xn_kb;
         float* src = X; long long ss = sx;
-        for (int pass = 0; pass < 2; ++pass) {
+        for (int pass = last ? 0 : 1; pass < 2; ++pass) {
           float* dst = pass == 0 ? T : O;
           const long long sd = pass == 0 ? st : so;
           conv_split(sb, phase, src, ss, x16, rows * r, 3);
@@ -666,6 +673,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           for (int b = 0; b < nb; ++b) sk_split(ap, 0, x_kb, b, nb, mmi->rinv_sw, b, nb, rows, r, dst + b * sd, r, 0, 3);
           src = dst; ss = sd;
         }
+        if (!last) return;
         SlotBuilder::Slot& nr = sb.next(ST_NORM, phase);  // the columns of Q back to unit length
         for (int b = 0; b < nb; ++b) {
           NormProblem np;
@@ -673,8 +681,9 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           nr.nm.push_back(np);
         }
       };
-      auto qr2 = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows, int w) {
-        if (tc_sketch) cholqr2_tc(sb, phase, X, sx, T, st, O, so, rows);
+      auto qr2 = [&](SlotBuilder& sb, int phase, float* X, long long sx, float* T, long long st, float* O, long long so, long long rows, int w,
+                     bool last = true) {
+        if (tc_sketch) cholqr2_tc(sb, phase, X, sx, T, st, O, so, rows, last);
         else cholqr2(sb, phase, X, sx, T, st, O, so, rows, w, nb, gram, lw, rinv);
       };
       // S * B on tensor cores: a_mn = 0 -> S rows are the output rows (Y = S B), 1 -> S^T B
@@ -739,7 +748,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, sd, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, rs, (int)n, signal(b), plain(Om + (long long)b * n * rs, rs), nullptr, store_epi(Ya + (long long)b * m * rs, rs)));
         }
-        qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs);
+        qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs, q == 0 || rr);
       }
       for (int it = 0; it < q; ++it) {
         if (tc_sketch) {  // Z = S^T P'
@@ -749,7 +758,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, 1 - sd, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)n, rs, (int)m, signal(b), plain(Pn + (long long)b * m * rs, rs), nullptr, store_epi(Za + (long long)b * n * rs, rs)));
         }
-        qr2(R, PH_SUBSPACE, Za, n * rs, Yb, maxd * rs, Zq, n * rs, n, rs);
+        qr2(R, PH_SUBSPACE, Za, n * rs, Yb, maxd * rs, Zq, n * rs, n, rs, rr);
         if (tc_sketch) {  // Y = S Z
           convert(R, Zq, zq16, (size_t)nb * n * r);
           sketch(R, 0, (c->d_maps + i)->zq16, Ya, m * r, m, n);
@@ -757,7 +766,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
           SlotBuilder::Slot& g = R.next(ST_GEMM, PH_SUBSPACE, sd, 0, 0);
           for (int b = 0; b < nb; ++b) g.g.push_back(gemm_prob((int)m, rs, (int)n, signal(b), plain(Zq + (long long)b * n * rs, rs), nullptr, store_epi(Ya + (long long)b * m * rs, rs)));
         }
-        qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs);
+        qr2(R, PH_SUBSPACE, Ya, m * rs, Yb, maxd * rs, Pn, m * rs, m, rs, it == q - 1 || rr);
       }
       if (rr) {
         // Rayleigh-Ritz truncation of the (r + p)-column basis Q (in Pn): Z = S^T Q, C = Z^T Z, the
