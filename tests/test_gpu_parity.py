@@ -613,6 +613,59 @@ def test_config4_full_size_fast_mode_sampled_columns():
     opt.close()
 
 
+def test_config5_full_shape_fast_mode_sampled_columns():
+    """One matrix of the refresh-stress configuration at its stated shape (4096 x 11008, r = 512, bf16,
+    Student-t gradients scaled to unit RMS), four workers, fast mode: the projection as two half-rank strips
+    per 128 columns and the update in its two sweeps, in the launch configuration the benchmark times for
+    this configuration. The inner step is separable by column, so the oracle recomputes sampled columns
+    (first, last, and some in between) from the same basis; then the outer step and a refresh with two
+    power iterations are held to the properties that do not need the oracle at this size."""
+    from paper_2602_04396_b200 import lordo
+    wl = synth.scaled(synth.config(5), mats=[(4096, 11008, 512)], K=4, H=2)
+    seed, lr, beta1, omega, form = 13, 0.004, 0.999, 0.97, 2
+    m, n, r = wl.mats[0]
+    W0 = synth.init_weights_device(wl, seed)
+    rng = np.random.default_rng(6)
+    cols = np.unique(np.concatenate([rng.integers(0, n, 6), [0, 127, 128, n - 1]]))
+    jj = torch.from_numpy(cols).cuda()
+    w0 = W0[0][:, jj].float().cpu().numpy().astype(np.float64)
+    opt = lordo.Lordo(wl.mats, wl.K, wl.H, W0, g_dtype=torch.bfloat16, e_dtype=torch.bfloat16, variant=0, error_feedback=True,
+                      beta2=0.999, eps=0.05, clip_rho=wl.clip_rho, outer=lordo.OUTER_NESTEROV, outer_lr=0.8, outer_momentum=0.9,
+                      power_iters=2, seed=seed, check_mode=0)
+    del W0
+    cfg = lo.OracleConfig(mats=((m, len(cols), r),), K=wl.K, H=wl.H, variant=0, beta2=hz.f32(0.999), eps=hz.f32(0.05), clip_rho=0.0,
+                          w_dtype="bf16", e_dtype="bf16", state_dtype="f32")
+    P0 = lo.store(lo.householder_qr_q(lo.random_matrix(seed, lo.PURPOSE_P0, 0, 0, 0, m, r)), "f32")
+    assert hz.largest_principal_angle(P0, hz._np_state(opt.P[0])) < ANGLE_TOL  # both sides start from the same basis
+    orc = lo.LordoOracle(cfg, [w0], P0=[hz._np_state(opt.P[0])])
+    G = None
+    for h in range(2):
+        G = synth.gradients_device(wl, seed, 0, h, out=G)
+        sq = G[0].float().pow(2).sum(dim=(1, 2), dtype=torch.float64)
+        c_want = np.minimum(1.0, wl.clip_rho / (np.sqrt(sq.cpu().numpy()) + 1e-6))
+        opt.inner_step(G, lr, beta1, omega, form)
+        c_got = opt.clip_coefficients().cpu().numpy()
+        assert np.abs(c_got - c_want[None, :]).max() <= 2e-6 * c_want.max()
+        gj = G[0][:, :, jj].float().cpu().numpy().astype(np.float64)
+        orc.inner_step([gj * c_want[:, None, None]], hz.f32(lr), hz.f32(beta1), hz.f32(omega), form)
+    assert opt.poll_status() == 0
+    got = {name: getattr(opt, name)[0][:, :, jj].float().cpu().numpy().astype(np.float64) for name in ("W", "E", "u", "v")}
+    assert hz.scaled_error(got["u"], orc.u[0]) < FAST_TOL and hz.scaled_error(got["v"], orc.v[0]) < 2 * FAST_TOL
+    assert hz.scaled_error(got["E"], orc.E[0]) < 2 * FAST_TOL
+    d = hz.bf16_ulp_distance(got["W"], orc.W[0])
+    assert (d <= 1).mean() > 0.99 and d.max() <= 8, ((d <= 1).mean(), d.max())
+    opt.outer_step()
+    opt.refresh_subspace(None, beta1)
+    assert opt.poll_status() == 0
+    W = opt.W[0]
+    assert bool((W == W[0:1]).all())
+    P = opt.P[0].double()
+    assert float((P.T @ P - torch.eye(r, device="cuda", dtype=torch.float64)).abs().max()) < TC_ORTH_TOL
+    for t in (opt.u[0], opt.v[0]):
+        assert bool(torch.isfinite(t).all())
+    opt.close()
+
+
 def _fold(t):
     """Order-sensitive 64-bit fold of a tensor's bit pattern (computed on the device)."""
     v = t.contiguous().view(-1)
