@@ -285,7 +285,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
   prefix_arrays(cfg, chunk_start, mom_start, wblk, sblk);
   // Refresh scratch: matrices are processed in groups whose scratch fits kRefreshScratchFloats;
   // every step of the refresh is one launch over a whole group.
-  constexpr size_t kRefreshScratchFloats = size_t(1) << 32;  // 16 GiB
+  constexpr size_t kRefreshScratchFloats = size_t(1) << 33;  // 32 GiB: fewer, fuller launches (a launch of the factorisation kernel takes as long for 64 matrices as for 148)
   std::vector<size_t> mat_scratch(n_mats);
   std::vector<int> group_of(n_mats);
   size_t scratch_floats = 0;
