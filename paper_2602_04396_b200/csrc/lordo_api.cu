@@ -394,7 +394,7 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         tp.strip_start_p = c->tc_strips_p; tp.nsplit = nsplit; tp.dcol2 = dcol2 ? dcol2 + (long long)k * md.ln : nullptr;
         c->h_tc.push_back(tp);
         c->tc_strips += (md.ln + 127) / 128;
-        c->tc_strips_p += (long long)nsplit * ((md.ln + 127) / 128);
+        c->tc_strips_p += (long long)nsplit * ((md.ln + 255) / 256);  // the projection runs as CTA pairs: two strips each
       }
     }
     c->d_tc_bf16 = ws ? reinterpret_cast<char*>(ws) + bf16_begin : nullptr;
@@ -466,7 +466,8 @@ size_t build(lordo_ctx* c, const lordo_buffers* buf, void* ws) {
         for (RandProblem& x : sl.rn) { x.blk_start = st.tiles; st.tiles += (x.count + 2047) / 2048; c->h_rands.push_back(x); }  // 8 per thread
       } else if (st.type == ST_SKETCH) {
         st.first = (long long)c->h_sks.size(); st.count = (int)sl.sk.size(); st.tiles = 0;
-        for (SkProblem& x : sl.sk) { x.tile_start = st.tiles; st.tiles += (x.M + 127) / 128; c->h_sks.push_back(x); }
+        // the kernel runs as CTA pairs: tiles of 256 rows, 128 per CTA
+        for (SkProblem& x : sl.sk) { x.tile_start = st.tiles; st.tiles += (x.M + 255) / 256; c->h_sks.push_back(x); }
       } else if (st.type == ST_CONVERT) {
         st.first = (long long)c->h_convs.size(); st.count = (int)sl.cv.size(); st.tiles = 0;
         for (ConvProblem& x : sl.cv) { x.blk_start = st.tiles; st.tiles += (x.count + 1023) / 1024; c->h_convs.push_back(x); }
@@ -1149,7 +1150,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
           good = good && encode_map3(hm[i].w_st32, md.W, md.n, md.m, c->K, 64, 32, true);
           if (md.E) good = good && encode_map3(hm[i].e_st32, md.E, md.n, md.m, c->K, 64, 32, true);
         }
-        good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n < 256 ? tp.r_n : 256, true);
+        good = good && encode_map3(hm[i].pt, tp.PT16, tp.m_k, tp.r_n, copies, 64, tp.r_n <= 256 ? tp.r_n / 2 : 128, true);  // a CTA's half of an MMA's rows
         good = good && encode_map3(hm[i].p16, tp.P16, tp.r_k, tp.m_k, copies, 64, 64, true);
         // refresh: signal as rows (64 k x 128 rows) and right-hand sides [batch][Kd][r]
         const int nbatch = loc ? c->K : 1;

@@ -98,8 +98,8 @@ struct TcProblem {
   int tr;                      // 1: W, G, E are stored transposed with respect to this problem (a matrix projected from the
                                // right): m counts their columns, n their rows
   float* tb;                   // [r][n] time buffer of this worker (+= lr * U~ every step), or null
-  // the projection's own strip numbering: nsplit strips per 128 columns (2 when 256 < r <= 512: one per
-  // half of the rank), and the second half's share of the column scale of the full-rank QHM term
+  // the projection's own numbering, in CTA pairs: nsplit pairs per 256 columns (2 when 256 < r <= 512: one
+  // per half of the rank), and the second half's share of the column scale of the full-rank QHM term
   long long strip_start_p;
   float* dcol2;                // [n], or null when nsplit == 1
   int nsplit, pad2;
@@ -238,7 +238,7 @@ void launch_colnorm_grouped(const NormProblem* probs, int nprobs, long long tota
 // signal matrix S streamed by TMA as bf16 (optionally formed as c*G + E in shared memory) and
 // B [Kd][r] in bf16. a_mn = 1: S is stored [Kd][M] (the product S^T P'); 0: stored [M][Kd].
 struct SkProblem {
-  long long tile_start;      // first 128-row tile of this problem within the launch
+  long long tile_start;      // first 256-row tile (128 rows per CTA of a pair) of this problem within the launch
   int M, Kd, r, r_n;
   int a_mn, a_c2, b_c2;      // third TMA coordinate (worker / batch index) of A and of B
   int split;                 // 0: one product; 2 or 3: operands split in that many bf16 planes, 3 or 6 passes over k

@@ -48,8 +48,8 @@ __device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x <<
 __device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
 
 // ---- projection ---------------------------------------------------------------------------------
-constexpr int kPStages = 3;
-constexpr uint32_t kPStageBytes = 65536;  // G 16 KB | E 16 KB | P^T tile up to 32 KB
+constexpr int kPStages = 4;
+constexpr uint32_t kPStageBytes = 49152;  // G 16 KB | E 16 KB | this CTA's rows of the P^T tile, up to 16 KB
 constexpr int kPXformWarps = 4, kPEpiWarps = 8;
 constexpr int kPThreads = (2 + kPXformWarps + kPEpiWarps) * 32;  // 448
 
@@ -69,47 +69,65 @@ constexpr int kAThreads = (3 + kAEpiWarps) * 32;  // 608: TMA inputs, MMA, 16 ep
 // no second buffer, so such a problem is dealt out as two strips per 128 columns, one per half of the
 // rank (rows [0, 256) and [256, r) of P^T, of the moments and of the low-rank operands). The two halves
 // are neighbours in the strip list, hence run on neighbouring CTAs at the same time, and the second
-// read of the G and E tiles is served by L2. Each half is then the r <= 256 pipeline: three stages, two
+// read of the G and E tiles is served by L2. Each half is then the r <= 256 pipeline: four stages, two
 // accumulator buffers, the moment epilogue of one strip under the main loop of the next.
-__global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_strips,
-                                                                   const TmaMatMaps* __restrict__ maps,
-                                                                   const TmaGradMaps* __restrict__ gmaps, StepScalars sc,
-                                                                   unsigned* __restrict__ status) {
+//
+// The kernel runs as CTA pairs (clusters of two, tcgen05 cta_group::2): a pair works on two neighbouring
+// strips of a problem (and the same half of the rank), one per CTA, and every MMA spans both (M = 256),
+// so each CTA fetches and keeps only half of the rows of the P^T tile. Each CTA's loads complete on
+// its own barrier; its transform warps pass the stage on to the MMA thread of the pair's first CTA.
+// strip_start_p and total_pairs count such pairs; a problem with an odd number of strips ends in a
+// pair whose second CTA reads zeros and stores nothing.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPThreads, 1)
+    project_tma_kernel(const TcProblem* __restrict__ probs, int nprobs, long long total_pairs, const TmaMatMaps* __restrict__ maps,
+                       const TmaGradMaps* __restrict__ gmaps, StepScalars sc, unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int ST = kPStages;
   constexpr uint32_t SB = kPStageBytes;
-  __shared__ uint64_t full_bar[3], xform_bar[3], empty_bar[3], acc_full[2], acc_empty[2];
+  // xform_bar and acc_empty are waited on by the MMA thread of the pair's first CTA only and fed by the
+  // warps of both CTAs; empty_bar and acc_full are signalled in both CTAs by that thread's commits
+  __shared__ uint64_t full_bar[kPStages], xform_bar[kPStages], empty_bar[kPStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ float dsum_s[kStrip];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool ef = sc.ef != 0;
+  const uint32_t rank = cluster_rank();
+  const long long pair_first = blockIdx.x >> 1, pair_step = gridDim.x >> 1;
 
   if (tid == 0) {
-    for (int s = 0; s < ST; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], kPXformWarps * 32); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kPEpiWarps * 32); }
+    for (int s = 0; s < ST; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], 2 * kPXformWarps); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 2 * kPEpiWarps); }
     mbar_init_fence();
   }
-  if (warp == 1) tmem_alloc(&tmem_slot, 512);
+  if (warp == 1) tmem_alloc_pair(&tmem_slot, 512);
   tc_fence_before_sync();
-  __syncthreads();
+  cluster_sync();  // both CTAs' barriers exist before either reaches into the other
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
+  // pair lp of a problem -> this CTA's 128 columns and its half of the rank (split problems: the two
+  // halves of a column pair are neighbouring pairs)
+#define LORDO_PAIR_COORDS(pr, pp)                                                              \
+  const int lp = (int)((pp) - (pr)->strip_start_p);                                            \
+  const int cs = 2 * ((pr)->nsplit == 2 ? lp >> 1 : lp) + (int)rank;                          \
+  const int r_lo = (pr)->nsplit == 2 ? (lp & 1) * 256 : 0;
 
   if (warp == 0) {
     // ---------------- TMA producer ------------------------------------------------------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+      for (long long strip = pair_first; strip < total_pairs && ok; strip += pair_step) {
         const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
-        const int l = (int)(strip - pr->strip_start_p);
-        const int n0 = (pr->nsplit == 2 ? l >> 1 : l) * kStrip, r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
+        LORDO_PAIR_COORDS(pr, strip)
+        const int n0 = cs * kStrip;
         const TmaMatMaps* mm = maps + pr->mat;
         const TmaGradMaps* gm = gmaps + pr->mat;
         const int nkb = pr->m_k / 64, rep = pr->replica, pc = pr->pcopy;
-        const int pt_rows = pr->r_n < 256 ? pr->r_n : 256;  // rows of one P^T box
+        const int pt_rows = pr->r_n <= 256 ? pr->r_n / 2 : 128;  // rows of one P^T box: a CTA's half of an MMA's N
+        const int n_h = pr->r_n - r_lo < 256 ? pr->r_n - r_lo : 256;
+        const int pt_row0 = r_lo + (int)rank * (n_h / 2);
         const uint32_t tx = 16384u + (ef ? 16384u : 0u) + (uint32_t)pt_rows * 128u;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % ST;
@@ -128,23 +146,25 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
               tma_load_3d(base + 24576, mm->e_sw, n0 + 64, kb * 64, rep, &full_bar[s]);
             }
           }
-          tma_load_3d(base + 32768, mm->pt, kb * 64, r_lo, pc, &full_bar[s]);  // rows past r_n arrive as zeros
+          tma_load_3d(base + 32768, mm->pt, kb * 64, pt_row0, pc, &full_bar[s]);  // rows past r_n arrive as zeros
         }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issue ---------------------------------------------------------------
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       uint32_t it = 0, si = 0;
       bool ok = true;
-      for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+      // the barriers the commits arrive on, in this CTA and in the other (8 bytes apart within an array)
+      const uint32_t eb0 = cluster_addr(&empty_bar[0], 0), eb1 = cluster_addr(&empty_bar[0], 1);
+      const uint32_t af0 = cluster_addr(&acc_full[0], 0), af1 = cluster_addr(&acc_full[0], 1);
+      for (long long strip = pair_first; strip < total_pairs && ok; strip += pair_step, ++si) {
         const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
-        const int l = (int)(strip - pr->strip_start_p);
-        const int r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
+        const int r_lo = pr->nsplit == 2 ? ((int)(strip - pr->strip_start_p) & 1) * 256 : 0;
         const int nkb = pr->m_k / 64;
         const uint32_t n_h = (uint32_t)(pr->r_n - r_lo < 256 ? pr->r_n - r_lo : 256);
         const bool tr = pr->tr != 0;  // the tile then lies as [128 strip elements][64 k]: a K-major operand
-        const uint32_t idesc = idesc_bf16_f32(128, n_h) | (tr ? 0u : kIdescAMajorMN);
+        const uint32_t idesc = idesc_bf16_f32(256, n_h) | (tr ? 0u : kIdescAMajorMN);
         const uint32_t buf = si & 1u;
         ok = mbar_wait(&acc_empty[buf], ((si >> 1) & 1u) ^ 1u, status);
         if (!ok) break;
@@ -156,11 +176,11 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           const uint32_t sA = smem_u32(smem + s * SB), sB = sA + 32768;
 #pragma unroll
           for (int k16 = 0; k16 < 4; ++k16)
-            mma_bf16(tmem + buf * 256, tr ? smem_desc_k128(sA + k16 * 32) : smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32), idesc,
-                     (kb > 0 || k16 > 0) ? 1u : 0u);
-          mma_commit(&empty_bar[s]);
+            mma_bf16_pair(tmem + buf * 256, tr ? smem_desc_k128(sA + k16 * 32) : smem_desc_mn128(sA + k16 * 2048), smem_desc_k128(sB + k16 * 32),
+                          idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+          mma_commit_pair(eb0 + 8u * s); mma_commit_pair(eb1 + 8u * s);
         }
-        if (ok) mma_commit(&acc_full[buf]);
+        if (ok) { mma_commit_pair(af0 + 8u * buf); mma_commit_pair(af1 + 8u * buf); }
       }
     }
   } else if (warp < 2 + kPXformWarps) {
@@ -168,7 +188,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
     const int xt = tid - 64;
     uint32_t it = 0;
     bool ok = true;
-    for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x) {
+    const uint32_t xf = cluster_addr(&xform_bar[0], 0);
+    for (long long strip = pair_first; strip < total_pairs && ok; strip += pair_step) {
       const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
       const int nkb = pr->m_k / 64;
       const float c = *pr->cptr;
@@ -192,7 +213,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
           G[idx] = a;
         }
         fence_async_smem();
-        mbar_arrive(&xform_bar[s]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(xf + 8u * s);  // this CTA's half of the stage is ready for the pair's MMAs
       }
     }
   } else {
@@ -202,10 +224,10 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
     const bool low = sc.form == LORDO_QHM_LOW;
     uint32_t si = 0;
     bool ok = true;
-    for (long long strip = blockIdx.x; strip < total_strips && ok; strip += gridDim.x, ++si) {
+    const uint32_t ae = cluster_addr(&acc_empty[0], 0);
+    for (long long strip = pair_first; strip < total_pairs && ok; strip += pair_step, ++si) {
       const TcProblem* __restrict__ pr = probs + find_problem_p(probs, nprobs, strip);
-      const int l = (int)(strip - pr->strip_start_p);
-      const int cs = pr->nsplit == 2 ? l >> 1 : l, r_lo = pr->nsplit == 2 ? (l & 1) * 256 : 0;
+      LORDO_PAIR_COORDS(pr, strip)
       const int n = pr->n, r = pr->r, r_k = pr->r_k;
       const int rn_h = pr->r_n - r_lo < 256 ? pr->r_n - r_lo : 256;  // rank rows of this strip, padded to 16
       const long long n0 = (long long)cs * kStrip;
@@ -268,7 +290,8 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
         }
       }
       tc_fence_before_sync();
-      mbar_arrive(&acc_empty[buf]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(ae + 8u * buf);
       if (sc.form == LORDO_QHM_FULL) {  // mu(D): mean over the rank axis, one value per column (a split problem: this half's share)
         if (half == 1) dsum_s[q * 32 + lane] = dsum;
         asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -277,9 +300,11 @@ __global__ void __launch_bounds__(kPThreads, 1) project_tma_kernel(const TcProbl
       }
     }
   }
+#undef LORDO_PAIR_COORDS
   tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 1) tmem_free(tmem, 512);
+  __syncwarp();
+  cluster_sync();  // neither CTA leaves while the other may still signal one of its barriers
+  if (warp == 1) tmem_free_pair(tmem, 512);
 }
 
 // =================================================================================================
@@ -629,10 +654,11 @@ cudaError_t tma_configure() {
   return cudaFuncSetAttribute(apply_tma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
-void launch_project_tma(const TcProblem* probs, int nprobs, long long total_strips, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
+void launch_project_tma(const TcProblem* probs, int nprobs, long long total_pairs, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
                         const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
-  const long long g = total_strips < grid ? total_strips : grid;
-  project_tma_kernel<<<(unsigned)g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_strips, maps, gmaps, sc, status);
+  if (total_pairs <= 0 || grid < 2) return;
+  const unsigned g = 2u * (unsigned)(total_pairs < grid / 2 ? total_pairs : grid / 2);
+  project_tma_kernel<<<g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_pairs, maps, gmaps, sc, status);
 }
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long strip_begin, long long strip_end, const TmaMatMaps* maps,
                       const TmaGradMaps* gmaps, const StepScalars& sc, int grid, int mode, int tr, unsigned* status, cudaStream_t st) {
@@ -658,13 +684,22 @@ void launch_apply_tma(const TcProblem* probs, int nprobs, long long strip_begin,
 // =================================================================================================
 // Sketch products of the refresh: C = S * B (fp32 out), S streamed by TMA. Same pipeline as the
 // projection: TMA -> (optional c*G + E in place) -> tcgen05.mma -> epilogue out of tensor memory,
-// two accumulator buffers, one CTA per SM walking the tile list.
+// two accumulator buffers.
+//
+// The kernel runs as CTA pairs (clusters of two, tcgen05 cta_group::2): a pair works on 256 rows of
+// S, 128 per CTA, and every MMA spans both CTAs (M = 256), so each CTA fetches and keeps only half of
+// the columns of B. With both operands in shared memory an MMA of one CTA reads 4 KB of A and 8 KB of B
+// per 16-deep step at r = 256, more than the shared memory can feed at the tensor cores' rate; the
+// pair halves B's share and its L2 traffic, and the freed shared memory holds one more stage. Each
+// CTA's loads complete on its own barrier; its transform warps (which form c*G + E where asked) pass
+// the stage on to the MMA thread of the pair's first CTA. The table counts tiles in pairs; a problem
+// with an odd number of 128-row tiles ends in a pair whose second CTA reads zeros and stores nothing.
 // =================================================================================================
 namespace lordo {
 using namespace umma;
 namespace {
-constexpr int kSStages = 3;
-constexpr uint32_t kSStageBytes = 65536;  // A 16 KB | E 16 KB | B up to 32 KB
+constexpr int kSMaxStages = 4;
+constexpr uint32_t kSSmemBytes = 196608 + 1024;  // 4 stages of A 16 KB | E 16 KB | B 16 KB, or 3 with 32 KB of B
 constexpr int kSThreads = (2 + 4 + 4) * 32;  // TMA, MMA, 4 transform warps, 4 epilogue warps
 constexpr uint32_t kIdescBMajorMN = 1u << 16;
 __device__ __forceinline__ int sk_passes(int split) { return split == 3 ? 6 : (split == 2 ? 3 : 1); }
@@ -680,24 +715,29 @@ __device__ __forceinline__ int find_sk(const SkProblem* __restrict__ probs, int 
 }  // namespace
 
 template <bool BIG>
-__global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProblem* __restrict__ probs, int nprobs, long long total_tiles,
-                                                                  unsigned* __restrict__ status) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSThreads, 1)
+    sketch_tma_kernel(const SkProblem* __restrict__ probs, int nprobs, long long total_tiles, unsigned* __restrict__ status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int ST = BIG ? 2 : 3;
-  constexpr uint32_t SB = BIG ? 98304u : kSStageBytes;
-  __shared__ uint64_t full_bar[3], xform_bar[3], empty_bar[3], acc_full[2], acc_empty[2];
+  constexpr int ST = BIG ? 3 : 4;
+  constexpr uint32_t SB = BIG ? 65536u : 49152u;  // A 16 KB | E 16 KB | this CTA's columns of B: up to 2 (+ 2) boxes of 8 KB
+  static_assert(ST * SB + 1024 <= kSSmemBytes, "stages do not fit the shared memory asked for");
+  // xform_bar and acc_empty are waited on by the MMA thread of the pair's first CTA only and fed by the
+  // warps of both CTAs; empty_bar and acc_full are signalled in both CTAs by that thread's commits
+  __shared__ uint64_t full_bar[kSMaxStages], xform_bar[kSMaxStages], empty_bar[kSMaxStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_slot;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();
+  const long long tile_first = blockIdx.x >> 1, tile_step = gridDim.x >> 1;  // tiles of 256 rows, one per pair
 
   if (tid == 0) {
-    for (int s = 0; s < ST; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], 128); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+    for (int s = 0; s < ST; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&xform_bar[s], 8); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 8); }
     mbar_init_fence();
   }
-  if (warp == 1) tmem_alloc(&tmem_slot, 512);
+  if (warp == 1) tmem_alloc_pair(&tmem_slot, 512);
   tc_fence_before_sync();
-  __syncthreads();
+  cluster_sync();  // both CTAs' barriers exist before either reaches into the other
   tc_fence_after_sync();
   const uint32_t tmem = tmem_slot;
 
@@ -705,13 +745,17 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (long long tile = tile_first; tile < total_tiles && ok; tile += tile_step) {
         const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
-        const int m0 = (int)(tile - pr->tile_start) * 128;
-        const int nkb1 = (pr->Kd + 63) / 64, nbox = (pr->r_n + 63) / 64;
+        const int m0 = (2 * (int)(tile - pr->tile_start) + (int)rank) * 128;
+        const int nkb1 = (pr->Kd + 63) / 64;
+        // this CTA's columns of B: half of the first 256 (one MMA) and half of the rest (a second MMA)
+        const int n_lo = pr->r_n < 256 ? pr->r_n : 256, n_hi = pr->r_n - n_lo;
+        const int c_lo = (int)rank * (n_lo / 2), c_hi = 256 + (int)rank * (n_hi / 2);
+        const int nbox_lo = (n_lo / 2 + 63) / 64, nbox_hi = (n_hi / 2 + 63) / 64;
         const int nkb = nkb1 * sk_passes(pr->split);
         const bool has_e = pr->map_e != nullptr;
-        const uint32_t tx = 16384u + (has_e ? 16384u : 0u) + (uint32_t)nbox * 8192u;
+        const uint32_t tx = 16384u + (has_e ? 16384u : 0u) + (uint32_t)(nbox_lo + nbox_hi) * 8192u;
         for (int j = 0; j < nkb; ++j, ++it) {
           const int seg = j / nkb1, kb = j - seg * nkb1;  // plane pairs (0,0) (0,1) (1,0) (1,1) (0,2) (2,0)
           const int a_c2 = pr->a_c2 + ((0x201100 >> (4 * seg)) & 3) * pr->a_pl, b_c2 = pr->b_c2 + ((0x021010 >> (4 * seg)) & 3) * pr->b_pl;
@@ -731,21 +775,25 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
             tma_load_3d(base, pr->map_a, kb * 64, m0, a_c2, &full_bar[s]);
             if (has_e) tma_load_3d(base + 16384, pr->map_e, kb * 64, m0, a_c2, &full_bar[s]);
           }
-          for (int x = 0; x < nbox; ++x) tma_load_3d(base + 32768 + x * 8192, pr->map_b, x * 64, kb * 64, b_c2, &full_bar[s]);
+          for (int x = 0; x < nbox_lo; ++x) tma_load_3d(base + 32768 + x * 8192, pr->map_b, c_lo + x * 64, kb * 64, b_c2, &full_bar[s]);
+          for (int x = 0; x < nbox_hi; ++x) tma_load_3d(base + 49152 + x * 8192, pr->map_b, c_hi + x * 64, kb * 64, b_c2, &full_bar[s]);
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       uint32_t it = 0, si = 0;
       bool ok = true;
-      for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++si) {
+      // the barriers the commits arrive on, in this CTA and in the other (8 bytes apart within an array)
+      const uint32_t eb0 = cluster_addr(&empty_bar[0], 0), eb1 = cluster_addr(&empty_bar[0], 1);
+      const uint32_t af0 = cluster_addr(&acc_full[0], 0), af1 = cluster_addr(&acc_full[0], 1);
+      for (long long tile = tile_first; tile < total_tiles && ok; tile += tile_step, ++si) {
         const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
         const int nkb = ((pr->Kd + 63) / 64) * sk_passes(pr->split);
         const bool a_mn = pr->a_mn != 0;
         const uint32_t n_lo = pr->r_n < 256 ? (uint32_t)pr->r_n : 256u, n_hi = (uint32_t)pr->r_n - n_lo;
         const uint32_t majors = kIdescBMajorMN | (a_mn ? kIdescAMajorMN : 0u);
-        const uint32_t idesc = idesc_bf16_f32(128, n_lo) | majors, idesc_hi = idesc_bf16_f32(128, n_hi ? n_hi : 16u) | majors;
+        const uint32_t idesc = idesc_bf16_f32(256, n_lo) | majors, idesc_hi = idesc_bf16_f32(256, n_hi ? n_hi : 16u) | majors;
         const uint32_t buf = BIG ? 0u : (si & 1u);
         ok = mbar_wait(&acc_empty[buf], ((BIG ? si : (si >> 1)) & 1u) ^ 1u, status);
         if (!ok) break;
@@ -758,19 +806,20 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
 #pragma unroll
           for (int k16 = 0; k16 < 4; ++k16) {
             const uint64_t ad = a_mn ? smem_desc_mn128(sA + k16 * 2048) : smem_desc_k128(sA + k16 * 32);
-            mma_bf16(tmem + buf * 256, ad, smem_desc_mn128(sB + k16 * 2048), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
-            if (BIG && n_hi) mma_bf16(tmem + 256, ad, smem_desc_mn128(sB + 4 * 8192 + k16 * 2048), idesc_hi, (kb > 0 || k16 > 0) ? 1u : 0u);
+            mma_bf16_pair(tmem + buf * 256, ad, smem_desc_mn128(sB + k16 * 2048), idesc, (kb > 0 || k16 > 0) ? 1u : 0u);
+            if (BIG && n_hi) mma_bf16_pair(tmem + 256, ad, smem_desc_mn128(sB + 2 * 8192 + k16 * 2048), idesc_hi, (kb > 0 || k16 > 0) ? 1u : 0u);
           }
-          mma_commit(&empty_bar[s]);
+          mma_commit_pair(eb0 + 8u * s); mma_commit_pair(eb1 + 8u * s);
         }
-        if (ok) mma_commit(&acc_full[buf]);
+        if (ok) { mma_commit_pair(af0 + 8u * buf); mma_commit_pair(af1 + 8u * buf); }
       }
     }
   } else if (warp < 6) {
     const int xt = tid - 64;
     uint32_t it = 0;
     bool ok = true;
-    for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+    const uint32_t xf = cluster_addr(&xform_bar[0], 0);
+    for (long long tile = tile_first; tile < total_tiles && ok; tile += tile_step) {
       const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
       const int nkb = ((pr->Kd + 63) / 64) * sk_passes(pr->split);
       const bool has_e = pr->map_e != nullptr;
@@ -795,7 +844,8 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
           }
           fence_async_smem();
         }
-        mbar_arrive(&xform_bar[s]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(xf + 8u * s);  // this CTA's half of the stage is ready for the pair's MMAs
       }
     }
   } else {
@@ -803,9 +853,10 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
     const int q = warp & 3;
     uint32_t si = 0;
     bool ok = true;
-    for (long long tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++si) {
+    const uint32_t ae = cluster_addr(&acc_empty[0], 0);
+    for (long long tile = tile_first; tile < total_tiles && ok; tile += tile_step, ++si) {
       const SkProblem* __restrict__ pr = probs + find_sk(probs, nprobs, tile);
-      const long long row = (tile - pr->tile_start) * 128 + q * 32 + lane;
+      const long long row = (2 * (tile - pr->tile_start) + rank) * 128 + q * 32 + lane;
       const bool row_ok = row < pr->M;
       float* __restrict__ crow = pr->C + (row_ok ? row : 0) * pr->ldc;
       const int r = pr->r, r_n = pr->r_n;
@@ -827,23 +878,27 @@ __global__ void __launch_bounds__(kSThreads, 1) sketch_tma_kernel(const SkProble
         }
       }
       tc_fence_before_sync();
-      mbar_arrive(&acc_empty[buf]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(ae + 8u * buf);
     }
   }
   tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 1) tmem_free(tmem, 512);
+  __syncwarp();
+  cluster_sync();  // neither CTA leaves while the other may still signal one of its barriers
+  if (warp == 1) tmem_free_pair(tmem, 512);
 }
 
 cudaError_t sketch_configure() {
-  cudaError_t e = cudaFuncSetAttribute(sketch_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSStages * kSStageBytes + 1024));
+  cudaError_t e = cudaFuncSetAttribute(sketch_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSSmemBytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(sketch_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSStages * kSStageBytes + 1024));
+  return cudaFuncSetAttribute(sketch_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSSmemBytes);
 }
+// total_tiles counts tiles of 256 rows (tile_start in `probs` does too); a CTA pair per SM pair.
 void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, int big, unsigned* status, cudaStream_t st) {
-  const long long g = total_tiles < grid ? total_tiles : grid;
-  if (big) sketch_tma_kernel<true><<<(unsigned)g, kSThreads, kSStages * kSStageBytes + 1024, st>>>(probs, nprobs, total_tiles, status);
-  else sketch_tma_kernel<false><<<(unsigned)g, kSThreads, kSStages * kSStageBytes + 1024, st>>>(probs, nprobs, total_tiles, status);
+  if (total_tiles <= 0 || grid < 2) return;
+  const unsigned g = 2u * (unsigned)(total_tiles < grid / 2 ? total_tiles : grid / 2);
+  if (big) sketch_tma_kernel<true><<<g, kSThreads, kSSmemBytes, st>>>(probs, nprobs, total_tiles, status);
+  else sketch_tma_kernel<false><<<g, kSThreads, kSSmemBytes, st>>>(probs, nprobs, total_tiles, status);
 }
 
 }  // namespace lordo
