@@ -149,7 +149,7 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint4& lo, const 
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // TMA: 3-d tiled load into shared memory completing on an mbarrier, 3-d tiled store from shared
-// memory in a bulk group. No multicast anywhere. `map` is a 128-byte tensor map in global memory.
+// memory in a bulk group. Every load goes to the issuing CTA's shared memory alone. `map` is a 128-byte tensor map in global memory.
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
@@ -241,25 +241,10 @@ __device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, u
                "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
                : "memory");
 }
-// A in tensor memory (128 rows per CTA), B in shared memory (N/2 rows per CTA), M = 256.
-__device__ __forceinline__ void mma_bf16_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
-               "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-               : "memory");
-}
 // Arrives on one barrier (of either CTA) once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit_pair(uint32_t bar_cluster_addr) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
-// 3-d tiled load into this CTA's shared memory that completes on a barrier of either CTA of the pair.
-__device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const void* map, int c0, int c1, int c2, uint32_t bar_cluster_addr) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
-          smem_u32(smem_dst)),
-      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster_addr)
-      : "memory");
-}
-
 // Byte offset of the 16-byte chunk `ch` (0..7) of row `i` inside a swizzled tile.
 __device__ __forceinline__ uint32_t swz_chunk(int i, int ch) {
   return (uint32_t)((i >> 3) * 1024 + (i & 7) * 128 + ((ch ^ (i & 7)) << 4));
