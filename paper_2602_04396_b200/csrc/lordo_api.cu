@@ -1131,6 +1131,7 @@ int lordo_init(const lordo_config* cfg, const lordo_buffers* buf, void* workspac
       int dev = 0;
       INIT_CUDA(cudaGetDevice(&dev));
       INIT_CUDA(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev));
+      if (c->sm_count < 2) return bail(LORDO_ERR_UNSUPPORTED);  // the projection and the refresh products run as CTA pairs
       std::vector<TmaMatMaps> hm(nm);
       bool good = tmap_encoder() != nullptr;
       const bool loc = c->cfg.variant == LORDO_LOCAL;
