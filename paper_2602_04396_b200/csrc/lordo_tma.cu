@@ -6,14 +6,17 @@
 //                       operations, layout-agnostic), and the tile is consumed as an MN-major
 //                       operand by tcgen05.mma. Two accumulator buffers in tensor memory let the
 //                       moment-update epilogue of one strip run under the main loop of the next
-//                       (ranks above 256 as two half-rank strips, see the kernel).
+//                       (ranks above 256 as two half-rank strips, see the kernel). Runs as CTA
+//                       pairs (clusters of two, tcgen05 cta_group::2): one strip per CTA, each CTA
+//                       holding half of the rows of the P^T tile.
 //   apply_tma_kernel    The strip's two low-rank operands (g^T, U~^T) live in tensor memory as the
 //                       A operands; rows of P and the tiles of G, E, W arrive by TMA; the epilogue
 //                       works on the swizzled tiles in shared memory (four neighbouring columns per
 //                       thread, 8-byte accesses) and the updated E and W tiles leave by TMA stores.
 //
-// One CTA per SM; a CTA walks the list of 128-column strips with stride gridDim.x. Every role walks
-// the same list, so stage and phase counters stay in step without further communication.
+// One CTA per SM; a CTA (the update kernel) or a CTA pair (the projection) walks the list of 128-column
+// strips, or of pairs of strips, with the stride of the grid. Every role walks the same list, so stage
+// and phase counters stay in step without further communication.
 #include "lordo_kernels.h"
 #include "lordo_umma.cuh"
 
