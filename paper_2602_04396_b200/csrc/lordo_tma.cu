@@ -638,10 +638,26 @@ __global__ void __launch_bounds__(kAThreads, 1) apply_tma_kernel(const TcProblem
 // =================================================================================================
 cudaError_t sketch_configure();
 
+// How many CTA pairs of `kernel` the device holds at once. A persistent kernel that launched more would
+// still be correct (no pair waits for another pair), but the pairs that start late would double its time.
+template <typename Kernel>
+static cudaError_t max_resident_pairs(Kernel kernel, int threads, size_t smem, int* pairs) {
+  cudaLaunchConfig_t lc = {};
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeClusterDimension;
+  at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+  lc.gridDim = dim3(2048, 1, 1); lc.blockDim = dim3((unsigned)threads, 1, 1); lc.dynamicSmemBytes = smem;
+  lc.attrs = &at; lc.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(pairs, kernel, &lc);
+}
+static int g_project_pairs = 0, g_sketch_pairs = 0;  // set by tma_configure, per process (one device model per process)
+
 cudaError_t tma_configure() {
   cudaError_t e = sketch_configure();
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(project_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kPStages * kPStageBytes + 1024));
+  if (e != cudaSuccess) return e;
+  e = max_resident_pairs(project_tma_kernel, kPThreads, kPStages * kPStageBytes + 1024, &g_project_pairs);
   if (e != cudaSuccess) return e;
   const int smem = (int)(kAPStages * 65536 + kAInStages * 32768 + 1024);  // the largest of the three modes
   e = cudaFuncSetAttribute(apply_tma_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -660,7 +676,9 @@ cudaError_t tma_configure() {
 void launch_project_tma(const TcProblem* probs, int nprobs, long long total_pairs, const TmaMatMaps* maps, const TmaGradMaps* gmaps,
                         const StepScalars& sc, int grid, unsigned* status, cudaStream_t st) {
   if (total_pairs <= 0 || grid < 2) return;
-  const unsigned g = 2u * (unsigned)(total_pairs < grid / 2 ? total_pairs : grid / 2);
+  long long pairs = grid / 2;
+  if (g_project_pairs > 0 && pairs > g_project_pairs) pairs = g_project_pairs;
+  const unsigned g = 2u * (unsigned)(total_pairs < pairs ? total_pairs : pairs);
   project_tma_kernel<<<g, kPThreads, kPStages * kPStageBytes + 1024, st>>>(probs, nprobs, total_pairs, maps, gmaps, sc, status);
 }
 void launch_apply_tma(const TcProblem* probs, int nprobs, long long strip_begin, long long strip_end, const TmaMatMaps* maps,
@@ -894,12 +912,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSThreads, 1)
 cudaError_t sketch_configure() {
   cudaError_t e = cudaFuncSetAttribute(sketch_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSSmemBytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(sketch_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSSmemBytes);
+  e = cudaFuncSetAttribute(sketch_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSSmemBytes);
+  if (e != cudaSuccess) return e;
+  return max_resident_pairs(sketch_tma_kernel<true>, kSThreads, kSSmemBytes, &g_sketch_pairs);
 }
 // total_tiles counts tiles of 256 rows (tile_start in `probs` does too); a CTA pair per SM pair.
 void launch_sketch_tma(const SkProblem* probs, int nprobs, long long total_tiles, int grid, int big, unsigned* status, cudaStream_t st) {
   if (total_tiles <= 0 || grid < 2) return;
-  const unsigned g = 2u * (unsigned)(total_tiles < grid / 2 ? total_tiles : grid / 2);
+  long long pairs = grid / 2;
+  if (g_sketch_pairs > 0 && pairs > g_sketch_pairs) pairs = g_sketch_pairs;
+  const unsigned g = 2u * (unsigned)(total_tiles < pairs ? total_tiles : pairs);
   if (big) sketch_tma_kernel<true><<<g, kSThreads, kSSmemBytes, st>>>(probs, nprobs, total_tiles, status);
   else sketch_tma_kernel<false><<<g, kSThreads, kSSmemBytes, st>>>(probs, nprobs, total_tiles, status);
 }
